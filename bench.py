@@ -1,0 +1,363 @@
+#!/usr/bin/env python
+"""Benchmark of the fused eviction path (score + select + compact) on synthetic Llama-3.1-8B-shaped inputs.
+
+One step = one call of restkv_evict over one layer of the long-context workload (batch 1, 32 query / 8 KV
+heads, head_dim 128, n = 131072 prefix rows, window 32, budget 2048, bf16).  Metric: prefix tokens scored and
+evicted per second per layer.  Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg4]
+
+N > 1 (under torchrun): every rank runs an independent replica of the layer on its own GPU -- the path has no
+exchange step, so there is no data-path collective; NCCL is used only for the barrier and the max over ranks.
+`--impl reference` times the CPU oracle (test infrastructure) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "prefix tokens/sec scored+evicted per layer at 128k"
+UNIT = "tokens/s"
+L2_FLUSH_BYTES = 256 << 20
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
+
+
+def algorithmic_bytes(case, keep):
+    """K and V read once plus the compacted cache written (bytes per step)."""
+    es = 2 if case.dtype == "bf16" else 4
+    kv = 2 * case.batch * case.n_kv_heads * case.n_kv * case.head_dim * es
+    out = 2 * case.batch * case.n_kv_heads * keep * case.head_dim * es
+    return kv, out
+
+
+def algorithmic_flops(case):
+    """Three dense contractions per prefix token and KV head: Q K^T, P V, V O^T."""
+    R = case.w * case.group
+    return 3 * 2 * R * case.head_dim * case.batch * case.n_kv_heads * case.n
+
+
+class ClockSampler:
+    """Samples nvidia-smi SM clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) >= 8:
+                self.rows.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm = sorted(float(r[0]) for r in self.rows if r[0].replace(".", "").isdigit())
+        mx = [float(r[1]) for r in self.rows if r[1].replace(".", "").isdigit()]
+        reasons = set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            for name, val in zip(names, r[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(self.rows)}
+
+
+# ------------------------------------------------------------------------------------------------
+def time_oracle(inp, heads, budget, repeats=1):
+    """Wall time of the oracle's score + select + compact on the given KV heads of the workload."""
+    import numpy as np
+    import oracle
+    c = inp.case
+    G = c.group
+    qh = np.concatenate([np.arange(h * G, (h + 1) * G) for h in heads])
+    Q, K, V = (np.ascontiguousarray(x) for x in (inp.Q[:, qh], inp.K[:, heads], inp.V[:, heads]))
+    best = None
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        res = oracle.score(Q, K, V, causal_tail=c.causal_tail, ema_decay=c.ema_decay, width=c.width, shift=c.shift,
+                           want_I_hat=False)
+        idx = oracle.select(res.scores, budget)
+        oracle.compact(K, idx)
+        oracle.compact(V, idx)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return best
+
+
+def cpu_baseline(inp, budget, target_seconds=12.0):
+    """The oracle as it stands on the host cores, on a bounded sample: whole KV heads of the workload."""
+    import oracle
+    c = inp.case
+    t1 = time_oracle(inp, [0], budget)
+    heads = max(1, min(c.n_kv_heads, int(target_seconds / max(t1, 1e-3))))
+    t = t1 if heads == 1 else time_oracle(inp, list(range(heads)), budget)
+    tokens = c.batch * c.n * heads / c.n_kv_heads     # layer-equivalent prefix tokens in the sample
+    return {"value": tokens / t, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": "%d of %d KV heads of the workload at full length n=%d (score+select+compact), %.2f s"
+                      % (heads, c.n_kv_heads, c.n, t)}
+
+
+def run_reference(args, case):
+    """--impl reference: the CPU oracle, as it stands, on a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2605_08840_b200.inputs import make_inputs
+    inp = make_inputs(case)
+    budget = case.budget
+    t1 = time_oracle(inp, [0], budget)
+    per_step_budget = 150.0 / max(1, args.steps + args.warmup)
+    heads = max(1, min(case.n_kv_heads, int(per_step_budget / max(t1, 1e-3))))
+    sel = list(range(heads))
+    for _ in range(args.warmup):
+        time_oracle(inp, sel, budget)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time_oracle(inp, sel, budget)
+    dt = (time.perf_counter() - t0) / args.steps
+    tokens = case.batch * case.n * heads / case.n_kv_heads
+    value = tokens / dt
+    sample = "%d of %d KV heads at full length n=%d per step" % (heads, case.n_kv_heads, case.n)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(case, l2="n/a (CPU)"),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def workload_config(case, l2):
+    return {"workload": "%s: one layer, batch %d, %d query / %d KV heads, head_dim %d, n=%d prefix rows, window %d, "
+                        "budget %d, pool width %d, ema_decay %.2f, %s, planted heavy hitters + sinks"
+                        % (case.name, case.batch, case.n_q_heads, case.n_kv_heads, case.head_dim, case.n, case.w,
+                           case.budget, case.width, case.ema_decay, case.dtype),
+            "global_batch": case.batch, "seq_len": case.n, "parallelism": "replicas", "l2": l2}
+
+
+# ------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg4")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--path", type=int, default=0, help="0 auto, 1 force SIMT, 2 require tensor cores")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    from paper_2605_08840_b200.inputs import CONFIGS, make_inputs
+    case = CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, case)
+        return
+
+    import numpy as np
+    import torch
+    from paper_2605_08840_b200 import binding as rk
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # every rank: an independent replica of the layer (per-rank seed so the replicas are not identical)
+    inp = make_inputs(case, seed=case.seed + 1000 * rank)
+    q_np, k_np, v_np = inp.device_arrays()
+    tdt = torch.bfloat16 if case.dtype == "bf16" else torch.float32
+
+    def dev(a):
+        t = torch.from_numpy(np.ascontiguousarray(a)).cuda()
+        return t.view(tdt) if case.dtype == "bf16" else t
+
+    Q, K, V = dev(q_np), dev(k_np), dev(v_np)
+    handle = rk.Handle()
+    handle.set_kernel_path(args.path)
+    shape = rk.make_shape(case.batch, case.n_q_heads, case.n_kv_heads, case.head_dim, case.n_kv, case.w,
+                          case.causal_tail, rk.BF16 if case.dtype == "bf16" else rk.F32)
+    pool = rk.fixed_pool(case.width, case.shift)
+    keep = min(case.budget, case.n_kv)
+    BH = (case.batch, case.n_kv_heads)
+    indices = torch.empty(BH + (keep,), dtype=torch.int32, device="cuda")
+    K_out = torch.empty(BH + (keep, case.head_dim), dtype=tdt, device="cuda")
+    V_out = torch.empty_like(K_out)
+    ws = torch.empty(handle.workspace_bytes(shape, case.budget), dtype=torch.uint8, device="cuda")
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+
+    def step():
+        handle.evict(shape, Q, K, V, case.ema_decay, pool, case.budget, indices, K_out, V_out, ws)
+
+    kernel_ids = {"pass1": rk.KERNEL_PASS1, "combine": rk.KERNEL_COMBINE, "pass2": rk.KERNEL_PASS2,
+                  "pool": rk.KERNEL_POOL, "select": rk.KERNEL_SELECT, "compact": rk.KERNEL_COMPACT}
+    prof = {}
+    for name, kid in kernel_ids.items():
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); b.record()
+        prof[name] = (a, b)
+    torch.cuda.synchronize()
+    for name, kid in kernel_ids.items():
+        handle.set_profile_events(kid, *prof[name])
+
+    for _ in range(args.warmup):
+        flush.zero_()
+        step()
+    barrier()
+    launches0 = handle.launch_count()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    step_ms, kern_ms = [], {k: [] for k in kernel_ids}
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(args.steps):
+        flush.zero_()                       # evict the previous step's lines from L2 (not timed)
+        ev0.record()
+        step()
+        ev1.record()
+        torch.cuda.synchronize()
+        step_ms.append(ev0.elapsed_time(ev1))
+        for name in kernel_ids:
+            kern_ms[name].append(prof[name][0].elapsed_time(prof[name][1]))
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    launches = handle.launch_count() - launches0
+    for kid in kernel_ids.values():
+        handle.set_profile_events(kid, None, None)
+    assert handle.poll_status() == rk.RESTKV_OK
+
+    total_ms = float(sum(step_ms))
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    tokens_per_step = world * case.batch * case.n
+    value = tokens_per_step * args.steps / (total_ms / 1e3)
+    ms_per_step = total_ms / args.steps
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----
+    e2e = None
+    if not args.no_e2e:
+        hQ, hK, hV = (torch.from_numpy(np.ascontiguousarray(a)).pin_memory() for a in (q_np, k_np, v_np))
+        h_idx = torch.empty(BH + (keep,), dtype=torch.int32).pin_memory()
+        h_Ko = torch.empty(BH + (keep, case.head_dim), dtype=torch.int16 if case.dtype == "bf16" else torch.float32)
+        h_Ko = h_Ko.pin_memory()
+        h_Vo = torch.empty_like(h_Ko).pin_memory()
+        e2e_steps = max(2, min(args.steps, 5))
+
+        def e2e_step():
+            handle.evict_host(shape, hQ, hK, hV, case.ema_decay, pool, case.budget, h_idx, h_Ko, h_Vo, Q, K, V,
+                              indices, K_out, V_out, ws)
+        e2e_step()
+        barrier()
+        ms = 0.0
+        for _ in range(e2e_steps):
+            ev0.record()
+            e2e_step()
+            ev1.record()
+            torch.cuda.synchronize()
+            ms += ev0.elapsed_time(ev1)
+        barrier()
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        h2d = sum(x.numel() * x.element_size() for x in (hQ, hK, hV))
+        d2h = sum(x.numel() * x.element_size() for x in (h_idx, h_Ko, h_Vo))
+        e2e = {"value": tokens_per_step * e2e_steps / (ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    kv_bytes, out_bytes = algorithmic_bytes(case, keep)
+    flops = algorithmic_flops(case)
+    kmean = {k: float(np.mean(v)) for k, v in kern_ms.items()}
+    dominant = max(("pass1", "pass2"), key=lambda k: kmean[k])
+    # the dominant kernel streams K and V once (pass 2 also writes 4 B of score per token and head)
+    dom_bytes = kv_bytes + (4 * case.batch * case.n_kv_heads * case.n if dominant == "pass2" else 0)
+    achieved = dom_bytes / (kmean[dominant] * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                "algorithmic_bytes_per_launch": dom_bytes, "ms_per_launch": kmean[dominant]}
+    t_roof_ms = max((kv_bytes + out_bytes) / (peaks["hbm_gbs"] * 1e9), flops / (peaks["bf16_tflops"] * 1e12)) * 1e3
+    path_roofline = {"t_roof_ms": t_roof_ms, "ms_per_step": ms_per_step / 1.0, "frac": t_roof_ms / ms_per_step,
+                     "bytes": kv_bytes + out_bytes, "flops": flops, "peak_source": peaks["source"],
+                     "note": "fused path against max(bytes/HBM peak, flops/bf16 peak); K,V read once + compacted write"}
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": case.dtype, "data": "synthetic",
+        "config": workload_config(case, l2="flushed between steps (256 MiB write); inputs 537 MB > 126 MB L2"),
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+        "roofline": roofline, "path_roofline": path_roofline, "kernels_ms": kmean,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = cpu_baseline(inp, case.budget)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,186 @@
+/*
+ * restkv.h -- C ABI of librestkv.so: the ReST-KV eviction-scoring hot path on one B200 (sm_100a).
+ *
+ * For one transformer layer, after prefill attention, the library scores every prefix
+ * KV pair of every KV head with the layer-wise output-reconstruction indicator, smooths
+ * the scores over the observation-window queries (EMA) and along the token axis (box
+ * pooling), selects the B best pairs per head and gathers their K/V rows into a
+ * compacted cache.  A split-K decode-attention kernel over such a cache is included so
+ * that decode latency over the compacted and the full cache can be timed.
+ *
+ * Conventions that hold for every entry point unless it says otherwise
+ *  - Tensor pointers are DEVICE pointers owned by the caller.  Nothing is allocated,
+ *    freed or synchronised by the library after restkv_create(); every call only enqueues
+ *    work on the given stream and returns.
+ *  - Layouts: Q_obs [batch, n_q_heads, w, head_dim] contiguous, oldest window query first.
+ *    K, V [batch, n_kv_heads, n_kv, head_dim] addressed through the element strides in
+ *    restkv_shape (head_dim is contiguous).  Query head hq reads KV head hq / (n_q_heads / n_kv_heads).
+ *    All base pointers must be 16-byte aligned and all strides multiples of 8 elements.
+ *  - n_kv = n + causal_tail.  causal_tail = 0: K,V hold only the n scored prefix rows and every
+ *    window query sees every row.  causal_tail = w: the last w rows of K,V are the window tokens'
+ *    own pairs; window query i sees trailing row j' only if j' <= i, and those rows receive
+ *    the score +inf (the paper's Omega, Eq. 8) so they are always kept.
+ *  - Errors are return codes.  A call that returns anything but RESTKV_OK has enqueued nothing.
+ *    Conditions detected on the device (a bounded wait that ran out) set a sticky status word
+ *    that restkv_poll_status() reads; kernels never trap.
+ *  - Calls on one handle must not overlap on the GPU if they share a workspace.
+ */
+#ifndef RESTKV_H_
+#define RESTKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  RESTKV_OK = 0,
+  RESTKV_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, misaligned pointer or stride, bad mode */
+  RESTKV_ERR_UNSUPPORTED = 2, /* a shape or mode no kernel covers (stated per entry point) */
+  RESTKV_ERR_WORKSPACE = 3,   /* workspace null, misaligned (256 B) or smaller than restkv_workspace_bytes() */
+  RESTKV_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed; restkv_last_cuda_error() has the code */
+  RESTKV_ERR_TIMEOUT = 5      /* a bounded device-side wait expired (reported by restkv_poll_status) */
+} restkv_status;
+
+typedef enum { RESTKV_BF16 = 0, RESTKV_F32 = 1 } restkv_dtype;
+
+typedef struct restkv_handle restkv_handle;
+
+/* The stream argument is a cudaStream_t passed as an opaque pointer (NULL = legacy default stream). */
+typedef void* restkv_stream;
+
+typedef struct {
+  int batch, n_q_heads, n_kv_heads, head_dim;
+  int n_kv;            /* rows in K and V (= scored prefix rows n + causal_tail) */
+  int w;               /* observation-window queries per head (the paper's S_w) */
+  int causal_tail;     /* 0 or w, see above */
+  restkv_dtype dtype;  /* element type of Q_obs, K, V and of the compacted outputs */
+  float softmax_scale; /* 0 => 1/sqrt(head_dim) (Eq. 3) */
+  long long k_stride_b, k_stride_h, k_stride_n; /* element strides of K; 0,0,0 => contiguous */
+  long long v_stride_b, v_stride_h, v_stride_n; /* element strides of V; 0,0,0 => contiguous */
+} restkv_shape;
+
+typedef enum { RESTKV_POOL_FIXED = 0, RESTKV_POOL_ADAPTIVE = 1 } restkv_pool_mode;
+
+typedef struct {
+  int mode;       /* restkv_pool_mode */
+  int width;      /* FIXED: odd box width W >= 1 (the kernel size k of Appendix B) */
+  int shift;      /* FIXED: gamma_shift */
+  float beta;     /* ADAPTIVE: scaling factor of Eq. 11-12 (paper: 2000) */
+  int base_width; /* ADAPTIVE: odd fixed kernel k; the box has width W_s + k - 1, centre shift gamma_shift */
+  int budget;     /* ADAPTIVE: B of Eq. 10 (per-query top-B whose mean index gives D_front / D_rear) */
+} restkv_pool_params;
+
+/* Creates a handle for the CURRENT device: queries its properties and allocates a 256-byte
+ * device status block (the only allocation the library ever makes).  Host pointer out. */
+restkv_status restkv_create(restkv_handle** out);
+restkv_status restkv_destroy(restkv_handle* h);
+
+/* Bytes of device workspace that score / select / evict / decode need for this shape and budget
+ * (256-byte aligned pointer required).  Returns 0 on invalid arguments.  `budget` may be 0 when
+ * only restkv_score / restkv_decode are used.  ADAPTIVE pooling needs the larger size reported by
+ * restkv_workspace_bytes_adaptive (it stores the per-query indicator, 4*batch*n_q_heads*w*n bytes). */
+size_t restkv_workspace_bytes(const restkv_shape* shape, int budget);
+size_t restkv_workspace_bytes_adaptive(const restkv_shape* shape, int budget);
+
+/*
+ * restkv_score -- Eq. 3 (attention weights and outputs of the window queries), Eq. 7 (indicator
+ * A/(1-A) * ||z - v_n||_2 with W_O = identity), Eq. 8-9 (EMA over the w window queries, oldest
+ * first, alpha = 1 - ema_decay, seeded with the oldest query), mean over the query heads of each
+ * KV head, Eq. 10-12 (ADAPTIVE window) and Eq. 13 (box mean, zero outside the scored rows, divisor
+ * always the box width).
+ *   Q_obs, K, V  device, dtype per shape->dtype
+ *   scores       device float [batch, n_kv_heads, n_kv]; rows >= n receive +inf
+ *   pool_used    optional device int32 [batch, n_kv_heads, 2] receiving (W, gamma) per head, or NULL
+ * RESTKV_BF16 with head_dim 128 and w * (n_q_heads/n_kv_heads) == 128 runs on the tcgen05 tensor-core
+ * kernels; every other supported shape (head_dim <= 256 and a multiple of 8, w*group <= 256) runs on
+ * fp32 SIMT kernels.  RESTKV_ERR_UNSUPPORTED otherwise.
+ */
+restkv_status restkv_score(restkv_handle* h, const restkv_shape* shape, const void* Q_obs, const void* K,
+                           const void* V, float ema_decay, const restkv_pool_params* pool, float* scores,
+                           int32_t* pool_used, void* workspace, size_t workspace_bytes, restkv_stream stream);
+
+/*
+ * restkv_select -- Eq. 14's argmax_B: per (batch, KV head) the min(budget, n_kv) largest scores,
+ * ties to the lower index, indices written in ascending order.
+ *   scores   device float [batch, n_kv_heads, n_kv] (+inf allowed, NaN not)
+ *   indices  device int32 [batch, n_kv_heads, min(budget, n_kv)]
+ */
+restkv_status restkv_select(restkv_handle* h, const restkv_shape* shape, const float* scores, int budget,
+                            int32_t* indices, void* workspace, size_t workspace_bytes, restkv_stream stream);
+
+/*
+ * restkv_compact -- Eq. 14's gather: K_out[b,h,s,:] = K[b,h,indices[b,h,s],:], same for V; bit-exact.
+ *   indices       device int32 [batch, n_kv_heads, n_sel], each in [0, n_kv) (out-of-range entries are
+ *                 skipped and set the sticky status word)
+ *   K_out, V_out  device [batch, n_kv_heads, n_sel, head_dim] contiguous, dtype per shape->dtype
+ */
+restkv_status restkv_compact(restkv_handle* h, const restkv_shape* shape, const void* K, const void* V,
+                             const int32_t* indices, int n_sel, void* K_out, void* V_out, restkv_stream stream);
+
+/*
+ * restkv_evict -- the fused path: score, select and compact in one call on one stream (Eq. 3-14).
+ *   scores_out   optional device float [batch, n_kv_heads, n_kv] (NULL: kept in the workspace only)
+ *   indices      device int32 [batch, n_kv_heads, min(budget, n_kv)]
+ *   K_out, V_out device [batch, n_kv_heads, min(budget, n_kv), head_dim]
+ */
+restkv_status restkv_evict(restkv_handle* h, const restkv_shape* shape, const void* Q_obs, const void* K,
+                           const void* V, float ema_decay, const restkv_pool_params* pool, int budget,
+                           float* scores_out, int32_t* indices, void* K_out, void* V_out, void* workspace,
+                           size_t workspace_bytes, restkv_stream stream);
+
+/*
+ * restkv_evict_host -- the fused path for callers whose tensors live in HOST memory: copies Q_obs, K, V
+ * (contiguous, host, ideally pinned) into caller-provided device staging buffers, runs restkv_evict and
+ * copies indices, K_out and V_out back to host memory, all asynchronously on `stream`.  shape strides
+ * must be 0 (contiguous).  The device buffers d_* have the sizes of their host counterparts.
+ */
+restkv_status restkv_evict_host(restkv_handle* h, const restkv_shape* shape, const void* Q_host, const void* K_host,
+                                const void* V_host, float ema_decay, const restkv_pool_params* pool, int budget,
+                                int32_t* indices_host, void* K_out_host, void* V_out_host, void* d_Q, void* d_K,
+                                void* d_V, int32_t* d_indices, void* d_K_out, void* d_V_out, void* workspace,
+                                size_t workspace_bytes, restkv_stream stream);
+
+/*
+ * restkv_decode -- one decode step (Eq. 3) of every query head over a cache of n_rows rows, split along
+ * the rows and merged by log-sum-exp.  Built to time decode over the compacted against the full cache.
+ *   q        device [batch, n_q_heads, head_dim]
+ *   Kc, Vc   device [batch, n_kv_heads, n_rows, head_dim] contiguous
+ *   out      device float [batch, n_q_heads, head_dim]
+ *   lse      optional device float [batch, n_q_heads] (natural-log sum of exp of the scaled logits)
+ * shape->n_kv, w, causal_tail and the strides are ignored.
+ */
+restkv_status restkv_decode(restkv_handle* h, const restkv_shape* shape, const void* q, const void* Kc,
+                            const void* Vc, int n_rows, float* out, float* lse, void* workspace,
+                            size_t workspace_bytes, restkv_stream stream);
+
+/* Synchronises `stream`, then returns and clears the sticky device status (RESTKV_OK if none). */
+restkv_status restkv_poll_status(restkv_handle* h, restkv_stream stream);
+
+/* Number of kernel launches the library has enqueued through this handle since creation. */
+long long restkv_launch_count(const restkv_handle* h);
+
+/* Last CUDA error code seen by this handle (0 = none). */
+int restkv_last_cuda_error(const restkv_handle* h);
+
+const char* restkv_error_string(restkv_status s);
+
+/* Profiling aid: while a pair of events is set for kernel `which` (RESTKV_KERNEL_*, not NONE), every call records
+ * `start` right before and `stop` right after that kernel's launch on the call's stream, so a caller can time
+ * single kernels of the fused path with CUDA events.  start/stop are cudaEvent_t handles created by the caller
+ * with timing enabled; passing NULL for both clears the pair. */
+typedef enum {
+  RESTKV_KERNEL_NONE = 0, RESTKV_KERNEL_PASS1 = 1, RESTKV_KERNEL_COMBINE = 2, RESTKV_KERNEL_PASS2 = 3,
+  RESTKV_KERNEL_POOL = 4, RESTKV_KERNEL_SELECT = 5, RESTKV_KERNEL_COMPACT = 6
+} restkv_kernel_id;
+restkv_status restkv_set_profile_events(restkv_handle* h, int which, void* start, void* stop);
+
+/* Testing aids: 0 = choose automatically, 1 = force the fp32 SIMT kernels, 2 = require tensor-core kernels. */
+restkv_status restkv_set_kernel_path(restkv_handle* h, int path);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RESTKV_H_ */

@@ -1,0 +1,218 @@
+// One decode step of every query head over a cache of n_rows rows (Eq. 3): split along the rows,
+// partial softmax attention per split, log-sum-exp merge.  Memory-bound streaming of K and V; all
+// G query heads of a KV head share each row that is loaded.
+#include "restkv_common.cuh"
+
+namespace restkv {
+
+namespace {
+
+constexpr int kDecThreads = 256;
+
+template <typename T> struct Chunk;   // 16 bytes of a row
+template <> struct Chunk<__nv_bfloat16> {
+  static constexpr int kElems = 8;
+  __device__ static void load(const __nv_bfloat16* p, float* out) {
+    const uint4 u = __ldg(reinterpret_cast<const uint4*>(p));
+    const unsigned int w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      out[2 * i] = __uint_as_float(w[i] << 16);
+      out[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+  }
+};
+template <> struct Chunk<float> {
+  static constexpr int kElems = 4;
+  __device__ static void load(const float* p, float* out) {
+    const float4 u = __ldg(reinterpret_cast<const float4*>(p));
+    out[0] = u.x; out[1] = u.y; out[2] = u.z; out[3] = u.w;
+  }
+};
+
+// grid (splits, batch*Hkv); block 256.  LPR lanes share one row (each owns CPL 16-byte chunks of it);
+// a warp covers 32/LPR rows per step.  Every lane group keeps its own running (m, l, o) per query head
+// and the groups are merged through shared memory at the end.
+template <typename T, int G, int LPR, int CPL>
+__global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(
+    int Hq, int Hkv, int d, int n_rows, float scale, const T* __restrict__ q, const T* __restrict__ Kc,
+    const T* __restrict__ Vc, float* __restrict__ part, int splits) {
+  constexpr int E = Chunk<T>::kElems;
+  constexpr int EPL = E * CPL;                 // elements of a row owned by one lane
+  constexpr int RPW = 32 / LPR;                // rows per warp step
+  constexpr int kGroups = (kDecThreads / 32) * RPW;
+  const int split = blockIdx.x, bh = blockIdx.y;
+  const int b = bh / Hkv, h = bh % Hkv;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const int sub = lane % LPR, grp = wid * RPW + lane / LPR;
+
+  float qf[G][EPL];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    const T* qr = q + ((long long)b * Hq + (long long)h * G + g) * d;
+#pragma unroll
+    for (int c = 0; c < CPL; ++c) Chunk<T>::load(qr + (c * LPR + sub) * E, &qf[g][c * E]);
+  }
+  float m[G], l[G], o[G][EPL];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    m[g] = -INFINITY; l[g] = 0.f;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) o[g][e] = 0.f;
+  }
+
+  const long long per = ((long long)n_rows + splits - 1) / splits;
+  const long long r0 = (long long)split * per;
+  const long long r1 = (r0 + per < n_rows) ? r0 + per : n_rows;
+  const T* Kh = Kc + (long long)bh * n_rows * d;
+  const T* Vh = Vc + (long long)bh * n_rows * d;
+
+  for (long long base = r0; base < r1; base += kGroups) {
+    const long long row = base + grp;
+    const bool in = row < r1;
+    float kf[EPL], vf[EPL];
+    if (in) {
+#pragma unroll
+      for (int c = 0; c < CPL; ++c) {
+        Chunk<T>::load(Kh + row * d + (c * LPR + sub) * E, &kf[c * E]);
+        Chunk<T>::load(Vh + row * d + (c * LPR + sub) * E, &vf[c * E]);
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) { kf[e] = 0.f; vf[e] = 0.f; }
+    }
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      float s = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) s = fmaf(qf[g][e], kf[e], s);
+#pragma unroll
+      for (int off = LPR / 2; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+      s = in ? s * scale : -INFINITY;
+      if (s > m[g]) {                         // new running maximum: rescale what was accumulated
+        const float corr = __expf(m[g] - s);  // m = -inf gives 0
+        l[g] *= corr;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) o[g][e] *= corr;
+        m[g] = s;
+      }
+      const float pexp = in ? __expf(s - m[g]) : 0.f;
+      l[g] += pexp;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) o[g][e] = fmaf(pexp, vf[e], o[g][e]);
+    }
+  }
+
+  // merge the lane groups of this block
+  __shared__ float sm_m[kGroups][G], sm_l[kGroups][G];
+  __shared__ float sm_scale[kGroups][G];
+  __shared__ float sm_o[G][LPR * EPL];
+  if (sub == 0) {
+#pragma unroll
+    for (int g = 0; g < G; ++g) { sm_m[grp][g] = m[g]; sm_l[grp][g] = l[g]; }
+  }
+  for (int e = threadIdx.x; e < G * LPR * EPL; e += kDecThreads) (&sm_o[0][0])[e] = 0.f;
+  __syncthreads();
+  float* my_part = part + ((long long)bh * splits + split) * G * (d + 2);
+  if (threadIdx.x < G) {
+    const int g = threadIdx.x;
+    float mm = -INFINITY;
+    for (int k = 0; k < kGroups; ++k) mm = fmaxf(mm, sm_m[k][g]);
+    float ll = 0.f;
+    for (int k = 0; k < kGroups; ++k) {
+      const float sc = (sm_m[k][g] == -INFINITY) ? 0.f : __expf(sm_m[k][g] - mm);
+      sm_scale[k][g] = sc;
+      ll += sm_l[k][g] * sc;
+    }
+    my_part[g * (d + 2) + 0] = mm;
+    my_part[g * (d + 2) + 1] = ll;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    const float sc = sm_scale[grp][g];
+#pragma unroll
+    for (int c = 0; c < CPL; ++c)
+#pragma unroll
+      for (int e = 0; e < E; ++e) atomicAdd(&sm_o[g][(c * LPR + sub) * E + e], o[g][c * E + e] * sc);
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < G * d; e += kDecThreads) {
+    const int g = e / d, k = e - g * d;
+    my_part[g * (d + 2) + 2 + k] = sm_o[g][k];
+  }
+}
+
+// grid (Hq, batch); block d threads (rounded to a warp).  Merges the splits.
+__global__ void decode_combine_kernel(int Hq, int G, int d, int splits, const float* __restrict__ part,
+                                      float* __restrict__ out, float* __restrict__ lse) {
+  const int hq = blockIdx.x, b = blockIdx.y;
+  const int Hkv = Hq / G, h = hq / G, g = hq % G;
+  const float* base = part + (((long long)b * Hkv + h) * splits) * G * (d + 2) + (long long)g * (d + 2);
+  const long long stride = (long long)G * (d + 2);
+  float mm = -INFINITY;
+  for (int s = 0; s < splits; ++s) mm = fmaxf(mm, base[s * stride]);
+  float ll = 0.f;
+  for (int s = 0; s < splits; ++s) {
+    const float ms = base[s * stride];
+    if (ms != -INFINITY) ll += base[s * stride + 1] * __expf(ms - mm);
+  }
+  for (int k = threadIdx.x; k < d; k += blockDim.x) {
+    float acc = 0.f;
+    for (int s = 0; s < splits; ++s) {
+      const float ms = base[s * stride];
+      if (ms != -INFINITY) acc += base[s * stride + 2 + k] * __expf(ms - mm);
+    }
+    out[((long long)b * Hq + hq) * d + k] = acc / ll;
+  }
+  if (lse && threadIdx.x == 0) lse[(long long)b * Hq + hq] = mm + logf(ll);
+}
+
+template <typename T, int G>
+cudaError_t launch_partial(const Problem& p, const void* q, const void* Kc, const void* Vc, int n_rows, float* part,
+                           int splits, cudaStream_t st) {
+  constexpr int E = Chunk<T>::kElems;
+  dim3 grid(splits, p.BH);
+  const int chunks = p.d / E;   // 16-byte chunks per row
+#define RESTKV_DEC(LPR, CPL)                                                                              \
+  decode_partial_kernel<T, G, LPR, CPL><<<grid, kDecThreads, 0, st>>>(p.Hq, p.Hkv, p.d, n_rows, p.scale, \
+                                                                      (const T*)q, (const T*)Kc, (const T*)Vc, part, splits)
+  if (chunks == 8) RESTKV_DEC(8, 1);
+  else if (chunks == 16) RESTKV_DEC(8, 2);
+  else if (chunks == 32) RESTKV_DEC(16, 2);
+  else if (chunks == 64) RESTKV_DEC(32, 2);
+  else if (chunks == 4) RESTKV_DEC(4, 1);
+  else if (chunks == 2) RESTKV_DEC(2, 1);
+  else return cudaErrorInvalidValue;
+#undef RESTKV_DEC
+  return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t launch_partial_g(const Problem& p, const void* q, const void* Kc, const void* Vc, int n_rows, float* part,
+                             int splits, cudaStream_t st) {
+  switch (p.G) {
+    case 1: return launch_partial<T, 1>(p, q, Kc, Vc, n_rows, part, splits, st);
+    case 2: return launch_partial<T, 2>(p, q, Kc, Vc, n_rows, part, splits, st);
+    case 4: return launch_partial<T, 4>(p, q, Kc, Vc, n_rows, part, splits, st);
+    case 8: return launch_partial<T, 8>(p, q, Kc, Vc, n_rows, part, splits, st);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_decode(const Problem& p, const void* q, const void* Kc, const void* Vc, int n_rows, float* out,
+                          float* lse, float* part, int splits, cudaStream_t st, int* n_launches) {
+  cudaError_t e = (p.dtype == RESTKV_BF16)
+                      ? launch_partial_g<__nv_bfloat16>(p, q, Kc, Vc, n_rows, part, splits, st)
+                      : launch_partial_g<float>(p, q, Kc, Vc, n_rows, part, splits, st);
+  if (e != cudaSuccess) return e;
+  const int threads = ((p.d + 31) / 32) * 32;
+  dim3 grid(p.Hq, p.batch);
+  decode_combine_kernel<<<grid, threads, 0, st>>>(p.Hq, p.G, p.d, splits, part, out, lse);
+  *n_launches = 2;
+  return cudaGetLastError();
+}
+
+}  // namespace restkv

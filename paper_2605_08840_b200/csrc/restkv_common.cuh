@@ -1,0 +1,88 @@
+// Shared declarations of the CUDA library: handle, workspace plan, kernel launch prototypes.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/restkv.h"
+
+namespace restkv {
+
+// Device status block (one per handle).  word[0] is a sticky bit mask written by kernels.
+enum : unsigned int {
+  kDevTimeout = 1u,      // a bounded wait (mbarrier / flag) expired
+  kDevBadIndex = 2u,     // an index outside [0, n_kv) reached the gather
+};
+
+struct Problem {
+  int batch, Hq, Hkv, G, d;
+  int n_kv, n, w, tail;   // n = scored prefix rows, tail = causal_tail
+  int R;                  // w * G query rows per KV head
+  int BH;                 // batch * Hkv
+  float scale;            // softmax scale
+  long long ksb, ksh, ksn, vsb, vsh, vsn;  // element strides
+  restkv_dtype dtype;
+};
+
+// Workspace carve-up (all offsets 256-byte aligned).
+struct Workspace {
+  int splits;             // token splits of pass 1 per (batch, KV head)
+  float* part_m;          // [BH, splits, R]
+  float* part_l;          // [BH, splits, R]
+  float* part_O;          // [BH, splits, R, d]
+  float* fin_m;           // [BH, R]    row max of the scaled logits (natural units)
+  float* fin_l;           // [BH, R]    sum of exp(s - m)
+  float* fin_M2;          // [BH, R]    m*log2(e) + log2(l): A = exp2(s*scale*log2(e) - M2)
+  float* fin_on;          // [BH, R]    squared norm of the bf16-rounded output row
+  float* O_f32;           // [BH, R, d]
+  __nv_bfloat16* O_bf16;  // [BH, R, d]
+  float* I_hat;           // [BH, n]
+  float* scores;          // [BH, n_kv] (used when the caller passes no scores buffer)
+  int* pool;              // [BH, 2] (W, gamma)
+  unsigned int* sel_scratch;  // select scratch: [BH, kSelScratchWords]
+  float* dec_part;        // decode partials
+  float* I_raw;           // adaptive only: [batch, Hq, w, n]
+  int32_t* adaptive_idx;  // adaptive only: [batch*Hq*w, B_p] per-query top-B_p indices
+  unsigned long long* adaptive_sums;  // adaptive only: [BH, 2] index sums (front, rear)
+  size_t bytes;
+};
+
+constexpr int kSelScratchWords = 64;
+constexpr int kDecodeMaxSplits = 64;
+
+int pass1_splits(const Problem& p, int sm_count);
+size_t plan_workspace(const Problem& p, int budget, int sm_count, bool adaptive, void* base, Workspace* ws);
+
+// ---- launches (each returns the cudaError_t of the launch) -------------------------------------
+cudaError_t launch_simt_pass1(const Problem& p, const Workspace& ws, const void* Q, const void* K, const void* V,
+                              cudaStream_t st);
+cudaError_t launch_combine(const Problem& p, const Workspace& ws, cudaStream_t st);
+cudaError_t launch_simt_pass2(const Problem& p, const Workspace& ws, const void* Q, const void* K, const void* V,
+                              float ema_decay, float* I_raw, cudaStream_t st);
+cudaError_t launch_set_pool(const Problem& p, const Workspace& ws, int W, int gamma, cudaStream_t st);
+cudaError_t launch_pool(const Problem& p, const Workspace& ws, float* scores, int32_t* pool_used, cudaStream_t st);
+cudaError_t launch_select(int rows, int n_kv, int budget, const float* scores, int32_t* indices,
+                          unsigned int* scratch, cudaStream_t st);
+cudaError_t launch_compact(const Problem& p, const void* K, const void* V, const int32_t* indices, int n_sel,
+                           void* K_out, void* V_out, unsigned int* dev_status, cudaStream_t st);
+cudaError_t launch_decode(const Problem& p, const void* q, const void* Kc, const void* Vc, int n_rows, float* out,
+                          float* lse, float* part, int splits, cudaStream_t st, int* n_launches);
+cudaError_t launch_adaptive_params(const Problem& p, const Workspace& ws, int budget, float beta, int base_width,
+                                   cudaStream_t st, int* n_launches);
+
+// Tensor-core (tcgen05 / TMEM / TMA) score kernels.  `supported` says whether the shape qualifies.
+bool tc_supported(const Problem& p);
+cudaError_t tc_init(void** state);   // resolves the driver entry point for tensor-map encoding
+cudaError_t launch_tc_pass1(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
+                            const void* V, unsigned int* dev_status, cudaStream_t st);
+cudaError_t launch_tc_pass2(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
+                            const void* V, float ema_decay, unsigned int* dev_status, cudaStream_t st);
+
+// ---- small device helpers ------------------------------------------------------------------------
+template <typename T> __device__ __forceinline__ float to_f32(T x);
+template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+}  // namespace restkv

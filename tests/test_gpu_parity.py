@@ -1,0 +1,385 @@
+"""GPU parity: the CUDA library, called through its C ABI binding, against the CPU oracle on the same
+seeded inputs.  Scores within the stated relative tolerance, selections identical up to rows whose
+oracle score lies inside that tolerance of the budget-th score, compaction bit-exact."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2605_08840_b200 import binding as rk
+from paper_2605_08840_b200.inputs import CONFIGS, Case, make_inputs, make_decode_query, round_to_bf16_bits
+
+from helpers import (TOL, GpuRun, assert_compaction_exact, assert_scores_close, assert_selection_valid, shape_of,
+                     torch_dev)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def handle():
+    h = rk.Handle()
+    yield h
+    h.close()
+
+
+def oracle_scores(inp, **kw):
+    c = inp.case
+    args = dict(causal_tail=c.causal_tail, ema_decay=c.ema_decay, width=c.width, shift=c.shift)
+    args.update(kw)
+    return oracle.score(inp.Q, inp.K, inp.V, **args)
+
+
+def full_check(handle, inp, budget=None, path=rk.PATH_AUTO, **pool_kw):
+    """evict on the GPU vs score+select on the oracle, all three acceptance rules."""
+    c = inp.case
+    handle.set_kernel_path(path)
+    try:
+        run = GpuRun(handle, inp, budget=budget)
+        scores, idx, K_out, V_out = run.evict(pool=run.pool(**pool_kw))
+    finally:
+        handle.set_kernel_path(rk.PATH_AUTO)
+    ref = oracle_scores(inp, **pool_kw)
+    tol = TOL[c.dtype]
+    worst = assert_scores_close(scores, ref.scores, tol)
+    exact = assert_selection_valid(idx, ref.scores, run.budget, tol)
+    _, kbits, vbits = inp.device_arrays()
+    assert_compaction_exact(idx, kbits, K_out)
+    assert_compaction_exact(idx, vbits, V_out)
+    return worst, exact
+
+
+# ------------------------------------------------------------------ config 1 (tiny, fp32 and bf16)
+@pytest.mark.parametrize("name", ["cfg1a", "cfg1b"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("tail", [0, 32])
+def test_config1(handle, name, dtype, tail):
+    case = CONFIGS[name].with_(dtype=dtype, causal_tail=tail)
+    full_check(handle, make_inputs(case))
+
+
+def test_config1_separate_calls_match_fused(handle):
+    inp = make_inputs(CONFIGS["cfg1b"])
+    run = GpuRun(handle, inp)
+    s_f, i_f, k_f, v_f = run.evict()
+    s = run.score()
+    i = run.select()
+    k, v = run.compact()
+    np.testing.assert_array_equal(s, s_f)
+    np.testing.assert_array_equal(i, i_f)
+    np.testing.assert_array_equal(k, k_f)
+    np.testing.assert_array_equal(v, v_f)
+
+
+@pytest.mark.parametrize("tail", [0, 32])
+def test_config1_adaptive_window(handle, tail):
+    case = CONFIGS["cfg1b"].with_(causal_tail=tail)
+    inp = make_inputs(case)
+    B = case.budget
+    probe = oracle_scores(inp, pool_mode=1, beta=1e9, base_width=1, budget=B)
+    delta = abs(probe.D[..., 0] - probe.D[..., 1]).min()
+    assert delta > 0
+    # beta chosen from the oracle's own D so that (D_front - D_rear)/beta sits mid-way between integers
+    for target, base in ((0.5, 1), (1.5, 1), (2.5, 5)):
+        beta = float(delta / target)
+        ref = oracle_scores(inp, pool_mode=1, beta=beta, base_width=base, budget=B)
+        x = (ref.D[..., 0] - ref.D[..., 1]) / beta
+        if np.any(np.abs(x - np.round(x)) < 0.05):
+            continue   # too close to a rounding boundary for an fp32-vs-fp64 ranking comparison
+        run = GpuRun(handle, inp, adaptive_budget=B)
+        scores = run.score(pool=rk.adaptive_pool(beta, base, B))
+        np.testing.assert_array_equal(run.pool_used.cpu().numpy(), ref.pool)
+        assert_scores_close(scores, ref.scores, TOL[case.dtype])
+
+
+# ------------------------------------------------------------------ config 2 (8B-shaped layer)
+@pytest.mark.parametrize("path", [rk.PATH_AUTO, rk.PATH_SIMT])
+def test_config2(handle, path):
+    inp = make_inputs(CONFIGS["cfg2"])
+    worst, exact = full_check(handle, inp, path=path)
+    # the planted heavy rows and sinks should be kept (reported, and checked loosely)
+    run = GpuRun(handle, inp)
+    _, idx, _, _ = run.evict()
+    planted = np.concatenate([inp.heavy_rows, np.broadcast_to(np.arange(4), inp.heavy_rows.shape[:2] + (4,))], -1)
+    recall = np.mean([np.isin(planted[0, h], idx[0, h]).mean() for h in range(8)])
+    assert recall > 0.9
+
+
+def test_config2_causal_tail(handle):
+    full_check(handle, make_inputs(CONFIGS["cfg2"].with_(causal_tail=32)))
+
+
+def test_config2_is_deterministic(handle):
+    run = GpuRun(handle, make_inputs(CONFIGS["cfg2"]))
+    a = run.evict()
+    b = run.evict()
+    for x, y in zip(a, b):
+        np.testing.assert_array_equal(x, y)
+
+
+# ------------------------------------------------------------------ config 3 (32 layers, drifting keys)
+def _subset_heads(inp, heads):
+    """The same workload restricted to some KV heads (and their query heads), for a bounded oracle run."""
+    c = inp.case
+    G = c.group
+    qh = np.concatenate([np.arange(h * G, (h + 1) * G) for h in heads])
+    sub = type(inp)(c.with_(n_q_heads=len(qh), n_kv_heads=len(heads)), inp.Q[:, qh], inp.K[:, heads], inp.V[:, heads])
+    return sub
+
+
+@pytest.mark.parametrize("layer", list(range(32)))
+def test_config3_layer(handle, layer):
+    case = CONFIGS["cfg3"].with_(seed=3000 + layer)
+    inp = make_inputs(case)
+    run = GpuRun(handle, inp)
+    scores, idx, K_out, V_out = run.evict()
+    heads = [layer % 8, (layer + 3) % 8]          # the oracle checks two of the eight heads per layer
+    ref = oracle_scores(_subset_heads(inp, heads))
+    assert_scores_close(scores[:, heads], ref.scores, TOL["bf16"])
+    assert_selection_valid(idx[:, heads], ref.scores, case.budget, TOL["bf16"])
+    _, kbits, vbits = inp.device_arrays()
+    assert_compaction_exact(idx, kbits, K_out)
+    assert_compaction_exact(idx, vbits, V_out)
+
+
+def test_config3_wide_pooling_changes_the_selection(handle):
+    inp = make_inputs(CONFIGS["cfg3"])
+    run = GpuRun(handle, inp)
+    _, idx7, _, _ = run.evict()
+    idx7 = idx7.copy()
+    scores, idx31, _, _ = run.evict(pool=run.pool(width=31))
+    ref = oracle_scores(_subset_heads(inp, [0]), width=31)
+    assert_scores_close(scores[:, [0]], ref.scores, TOL["bf16"])
+    assert_selection_valid(idx31[:, [0]], ref.scores, inp.case.budget, TOL["bf16"])
+    assert not np.array_equal(idx7, idx31)
+
+
+# ------------------------------------------------------------------ config 4 (128k, the timed headline)
+def test_config4_full_size(handle):
+    inp = make_inputs(CONFIGS["cfg4"])
+    worst, exact = full_check(handle, inp)
+    print("cfg4: worst rel err %.2e, heads with identical index sets %.2f" % (worst, exact))
+
+
+# ------------------------------------------------------------------ config 5 (batched sweep)
+@pytest.fixture(scope="module")
+def cfg5_inputs():
+    return make_inputs(CONFIGS["cfg5"])
+
+
+@pytest.mark.parametrize("decay", [0.5, 0.9, 0.99])
+@pytest.mark.parametrize("width", [1, 7, 31])
+def test_config5_sweep(handle, cfg5_inputs, decay, width):
+    inp = cfg5_inputs
+    pairs = [(1, 2), (6, 5)]       # (batch element, KV head) pairs the oracle checks at full length
+    refs = []
+    for b, h in pairs:
+        one = _subset_heads(type(inp)(inp.case.with_(batch=1), inp.Q[b:b + 1], inp.K[b:b + 1], inp.V[b:b + 1]), [h])
+        refs.append(oracle_scores(one, ema_decay=decay, width=width).scores[0, 0])
+    _, kbits, vbits = inp.device_arrays()
+    for budget in (128, 512, 2048):
+        run = GpuRun(handle, inp, budget=budget)
+        scores, idx, K_out, V_out = run.evict(pool=run.pool(width=width), ema_decay=decay)
+        for (b, h), ref in zip(pairs, refs):
+            assert_scores_close(scores[b, h], ref, TOL["bf16"])
+            assert_selection_valid(idx[b:b + 1, h:h + 1], ref[None, None], budget, TOL["bf16"])
+        assert_compaction_exact(idx, kbits, K_out)
+        assert_compaction_exact(idx, vbits, V_out)
+        del run
+
+
+# ------------------------------------------------------------------ edge cases
+EDGE = [
+    # name, Hq, Hkv, d, n, w, budget, width, dtype, tail
+    ("one_row", 4, 1, 128, 1, 32, 1, 1, "bf16", 0),
+    ("five_rows", 4, 1, 128, 5, 32, 3, 3, "bf16", 0),
+    ("tile_minus_one", 4, 1, 128, 127, 32, 17, 7, "bf16", 0),
+    ("tile_exact", 4, 1, 128, 128, 32, 128, 7, "bf16", 0),
+    ("tile_plus_one", 8, 2, 128, 129, 32, 1, 7, "bf16", 0),
+    ("ragged", 8, 2, 128, 1000, 32, 100, 5, "bf16", 0),
+    ("ragged_tail", 8, 2, 128, 4097, 32, 640, 21, "bf16", 32),
+    ("budget_over_n", 4, 1, 128, 300, 32, 1000, 7, "bf16", 0),
+    ("w1", 4, 1, 128, 200, 1, 20, 3, "bf16", 0),
+    ("w7_tail", 4, 2, 64, 333, 7, 40, 5, "bf16", 7),
+    ("mha", 2, 2, 64, 500, 32, 64, 7, "f32", 0),
+    ("g2_d32", 4, 2, 32, 257, 16, 33, 7, "f32", 16),
+    ("d256", 2, 1, 256, 130, 8, 13, 3, "bf16", 0),
+    ("g8", 8, 1, 128, 700, 16, 70, 7, "bf16", 0),
+]
+
+
+@pytest.mark.parametrize("spec", EDGE, ids=[e[0] for e in EDGE])
+def test_edge_cases(handle, spec):
+    name, Hq, Hkv, d, n, w, budget, width, dtype, tail = spec
+    case = Case(name, 2, Hq, Hkv, d, n, w, budget, width, 0, 0.7, dtype, tail, "normal", 77)
+    full_check(handle, make_inputs(case))
+
+
+@pytest.mark.parametrize("decay", [0.0, 1.0])
+def test_ema_extremes(handle, decay):
+    case = Case("ema", 1, 8, 2, 128, 600, 16, 50, 1, 0, decay, "bf16", 0, "normal", 5)
+    full_check(handle, make_inputs(case))
+
+
+def test_pool_shift(handle):
+    case = Case("shift", 1, 8, 2, 64, 400, 32, 50, 5, 0, 0.9, "f32", 0, "normal", 6)
+    inp = make_inputs(case)
+    for shift in (-3, 2, 40):
+        full_check(handle, inp, shift=shift)
+
+
+def test_strided_kv_layout(handle):
+    """K and V stored as [batch, n_kv, Hkv, d] (token-major), addressed through the strides."""
+    import torch
+    case = Case("strided", 2, 8, 2, 128, 900, 32, 90, 7, 0, 0.9, "bf16", 0, "normal", 8)
+    inp = make_inputs(case)
+    q, k, v = inp.device_arrays()
+    Q = torch_dev(q, "bf16")
+    Kt = torch_dev(np.ascontiguousarray(k.transpose(0, 2, 1, 3)), "bf16")   # [b, n, H, d]
+    Vt = torch_dev(np.ascontiguousarray(v.transpose(0, 2, 1, 3)), "bf16")
+    H, n, d = case.n_kv_heads, case.n_kv, case.head_dim
+    strides = (n * H * d, d, H * d)
+    shape = shape_of(case, k_strides=strides, v_strides=strides)
+    ref_run = GpuRun(handle, inp)
+    s_ref, i_ref, k_ref, v_ref = ref_run.evict()
+    run = GpuRun(handle, inp)
+    handle.evict(shape, Q, Kt, Vt, case.ema_decay, run.pool(), case.budget, run.indices, run.K_out, run.V_out, run.ws,
+                 scores_out=run.scores)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(run.scores.cpu().numpy(), s_ref)
+    np.testing.assert_array_equal(run.indices.cpu().numpy(), i_ref)
+    np.testing.assert_array_equal(run.K_out.view(torch.int16).cpu().numpy(), k_ref)
+    np.testing.assert_array_equal(run.V_out.view(torch.int16).cpu().numpy(), v_ref)
+
+
+# ------------------------------------------------------------------ unit: select, compact, decode
+def test_select_matches_stable_sort_with_ties_and_inf(handle):
+    import torch
+    rng = np.random.default_rng(3)
+    n_kv = 5000
+    s = rng.standard_normal((2, 3, n_kv)).astype(np.float32)
+    s[0, 0, ::7] = 0.25                       # many ties
+    s[0, 1] = 1.0                             # all equal
+    s[1, 0, -40:] = np.inf
+    s[1, 1] = np.abs(s[1, 1]) * 1e-30         # tiny positives
+    s[1, 2, 100:200] = -s[1, 2, 100:200] - 5  # negatives
+    case = Case("sel", 2, 3, 3, 64, n_kv, 32)
+    shape = shape_of(case)
+    d_s = torch.from_numpy(s).cuda()
+    for B in (1, 2, 31, 32, 33, 1000, 4999, 5000, 9000):
+        keep = min(B, n_kv)
+        idx = torch.empty((2, 3, keep), dtype=torch.int32, device="cuda")
+        ws = torch.empty(handle.workspace_bytes(shape, B), dtype=torch.uint8, device="cuda")
+        handle.select(shape, d_s, B, idx, ws)
+        torch.cuda.synchronize()
+        got = idx.cpu().numpy()
+        np.testing.assert_array_equal(got, oracle.select(s.astype(np.float64), B))
+
+
+def test_compact_bit_exact_and_bad_index_reported(handle):
+    import torch
+    case = Case("cmp", 2, 4, 2, 64, 300, 8, dtype="f32")
+    shape = shape_of(case)
+    rng = np.random.default_rng(4)
+    K = rng.standard_normal((2, 2, 300, 64)).astype(np.float32)
+    V = rng.standard_normal((2, 2, 300, 64)).astype(np.float32)
+    idx = np.sort(rng.choice(300, size=(2, 2, 37)), axis=-1).astype(np.int32)
+    dK, dV, dI = torch.from_numpy(K).cuda(), torch.from_numpy(V).cuda(), torch.from_numpy(idx).cuda()
+    Ko = torch.zeros((2, 2, 37, 64), device="cuda")
+    Vo = torch.zeros_like(Ko)
+    handle.compact(shape, dK, dV, dI, 37, Ko, Vo)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(Ko.cpu().numpy(), oracle.compact(K, idx))
+    np.testing.assert_array_equal(Vo.cpu().numpy(), oracle.compact(V, idx))
+    assert handle.poll_status() == rk.RESTKV_OK
+    bad = idx.copy()
+    bad[1, 1, 5] = 300                       # out of range: skipped and reported, never dereferenced
+    handle.compact(shape, dK, dV, torch.from_numpy(bad).cuda(), 37, Ko, Vo)
+    assert handle.poll_status() == rk.ERR_INVALID_ARG
+    assert handle.poll_status() == rk.RESTKV_OK     # sticky word is cleared by the poll
+
+
+@pytest.mark.parametrize("spec", [("bf16", 32, 8, 128, 2048), ("bf16", 32, 8, 128, 131072), ("f32", 8, 2, 64, 777),
+                                  ("bf16", 4, 4, 64, 100), ("bf16", 16, 2, 256, 1500)])
+def test_decode_matches_oracle(handle, spec):
+    import torch
+    dtype, Hq, Hkv, d, rows = spec
+    rng = np.random.default_rng(11)
+    b = 1 if rows > 10000 else 2
+
+    def draw(shape):
+        x = rng.standard_normal(shape).astype(np.float32)
+        if dtype == "bf16":
+            bits = round_to_bf16_bits(x)
+            return (bits.astype(np.uint32) << 16).view(np.float32), bits.view(np.int16)
+        return x, x
+
+    q, qd = draw((b, Hq, d))
+    K, Kd = draw((b, Hkv, rows, d))
+    V, Vd = draw((b, Hkv, rows, d))
+    ref, ref_lse = oracle.decode(q, K, V)
+    case = Case("dec", b, Hq, Hkv, d, rows, 1, dtype=dtype)
+    shape = shape_of(case)
+    out = torch.empty((b, Hq, d), dtype=torch.float32, device="cuda")
+    lse = torch.empty((b, Hq), dtype=torch.float32, device="cuda")
+    ws = torch.empty(handle.workspace_bytes(shape, 0), dtype=torch.uint8, device="cuda")
+    handle.decode(shape, torch_dev(qd, dtype), torch_dev(Kd, dtype), torch_dev(Vd, dtype), rows, out, ws, lse=lse)
+    torch.cuda.synchronize()
+    tol = 2e-3 if dtype == "bf16" else 2e-5
+    scale = np.abs(ref).max(axis=-1, keepdims=True)
+    assert np.max(np.abs(out.cpu().numpy() - ref) / scale) < tol
+    np.testing.assert_allclose(lse.cpu().numpy(), ref_lse, rtol=1e-5, atol=1e-5)
+
+
+def test_decode_over_compacted_cache_of_config2(handle):
+    import torch
+    inp = make_inputs(CONFIGS["cfg2"])
+    run = GpuRun(handle, inp)
+    _, idx, K_out, V_out = run.evict()
+    q = make_decode_query(inp)
+    qd = round_to_bf16_bits(q).view(np.int16)
+    c = inp.case
+    out = torch.empty((c.batch, c.n_q_heads, c.head_dim), dtype=torch.float32, device="cuda")
+    handle.decode(run.shape, torch_dev(qd, "bf16"), run.K_out, run.V_out, run.keep, out, run.ws)
+    torch.cuda.synchronize()
+    Kc = np.take_along_axis(inp.K, idx[..., None].astype(np.int64), axis=2)
+    Vc = np.take_along_axis(inp.V, idx[..., None].astype(np.int64), axis=2)
+    ref, _ = oracle.decode(q, Kc, Vc)
+    assert np.max(np.abs(out.cpu().numpy() - ref)) < 2e-3 * np.abs(ref).max()
+
+
+# ------------------------------------------------------------------ API misuse: error codes, never a fault
+def test_api_rejects_bad_arguments(handle):
+    import torch
+    case = CONFIGS["cfg1b"]
+    inp = make_inputs(case)
+    run = GpuRun(handle, inp)
+
+    def status_of(fn):
+        try:
+            fn()
+        except rk.RestKVError as e:
+            return e.status
+        return rk.RESTKV_OK
+
+    pool = run.pool()
+    ev = lambda **kw: handle.evict(kw.get("shape", run.shape), kw.get("Q", run.Q), run.K, run.V, kw.get("decay", 0.9),
+                                   kw.get("pool", pool), kw.get("budget", 128), run.indices, run.K_out, run.V_out,
+                                   kw.get("ws", run.ws))
+    assert status_of(lambda: ev()) == rk.RESTKV_OK
+    assert status_of(lambda: ev(Q=None)) == rk.ERR_INVALID_ARG
+    assert status_of(lambda: ev(budget=0)) == rk.ERR_INVALID_ARG
+    assert status_of(lambda: ev(decay=1.5)) == rk.ERR_INVALID_ARG
+    assert status_of(lambda: ev(pool=rk.fixed_pool(4))) == rk.ERR_INVALID_ARG              # even width
+    assert status_of(lambda: ev(ws=run.ws[:1024])) == rk.ERR_WORKSPACE                     # too small
+    assert status_of(lambda: ev(ws=run.ws[1:])) == rk.ERR_WORKSPACE                        # misaligned
+    assert status_of(lambda: ev(Q=run.Q.view(-1)[1:])) == rk.ERR_INVALID_ARG               # misaligned tensor
+    bad = shape_of(case.with_(causal_tail=5))
+    assert status_of(lambda: ev(shape=bad)) == rk.ERR_INVALID_ARG
+    bad = shape_of(case.with_(n_q_heads=7))
+    assert status_of(lambda: ev(shape=bad)) == rk.ERR_INVALID_ARG
+    bad = shape_of(case.with_(head_dim=20))
+    assert status_of(lambda: ev(shape=bad)) == rk.ERR_UNSUPPORTED
+    bad = shape_of(case, k_strides=(0, 0, 7))
+    assert status_of(lambda: ev(shape=bad)) == rk.ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert handle.poll_status() == rk.RESTKV_OK
+    assert handle.launch_count() > 0
