@@ -22,8 +22,8 @@ namespace restkv {
 static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 int pass1_splits(const Problem& p, int sm_count) {
-  // enough (batch, head, split) blocks to fill the GPU, at least one 128-token tile per split
-  int splits = (sm_count + p.BH - 1) / p.BH;
+  // one wave of (batch, head, split) blocks over the SMs, at least one 128-token tile per split
+  int splits = sm_count / p.BH;
   const int tiles = (p.n_kv + 127) / 128;
   if (splits > tiles) splits = tiles;
   if (splits < 1) splits = 1;

@@ -1,10 +1,564 @@
-// Tensor-core score kernels (placeholder until the tcgen05 kernels land).
+// Tensor-core score kernels for sm_100a: bf16 inputs, head_dim 128, w * group = 128 query rows per KV head.
+//
+// Both kernels work on tiles of 128 tokens.  K and V tiles arrive in shared memory through TMA
+// (128-byte swizzle, two [128 x 64] boxes per tile), the contractions run on tcgen05.mma with fp32
+// accumulators in tensor memory, and warp-specialised CTAs (one TMA warp, one MMA warp, epilogue
+// warpgroups) overlap the three.
+//
+//   pass 1  (Eq. 3)   S = Q K^T per tile (queries in TMEM lanes), online softmax statistics with a lazily
+//                     updated reference maximum, P = exp2(.) written to TMEM as bf16 and used as the A operand
+//                     of O += P V.  One partial (m, l, O) per (batch, head, token split).
+//   pass 2  (Eq. 7-9) S^T = K Q^T and C^T = V O^T per tile (tokens in TMEM lanes, one thread per token):
+//                     A = exp2(s*c - M), ||o - v||^2 = ||o||^2 + ||v||^2 - 2 o.v, I = A/(1-A) * ||o - v||,
+//                     EMA over the window queries as a Horner chain down the accumulator columns,
+//                     mean over the query heads of the group.
+// Every mbarrier wait is bounded; a wait that runs out sets the sticky timeout bit and the CTA unwinds.
+#include <cuda.h>
+
 #include "restkv_common.cuh"
+#include "sm100_ptx.cuh"
+
 namespace restkv {
-bool tc_supported(const Problem&) { return false; }
-cudaError_t tc_init(void** state) { *state = nullptr; return cudaSuccess; }
-cudaError_t launch_tc_pass1(void*, const Problem&, const Workspace&, const void*, const void*, const void*,
-                            unsigned int*, cudaStream_t) { return cudaErrorNotSupported; }
-cudaError_t launch_tc_pass2(void*, const Problem&, const Workspace&, const void*, const void*, const void*, float,
-                            unsigned int*, cudaStream_t) { return cudaErrorNotSupported; }
+
+namespace {
+
+using namespace ptx;
+
+constexpr int kTile = 128;                       // tokens per tile
+constexpr int kHeadDim = 128;
+constexpr int kRows = 128;                       // query rows per KV head (w * G)
+constexpr uint32_t kBoxBytes = 128 * 64 * 2;     // one [128 rows x 64 bf16] TMA box
+constexpr uint32_t kTileBytes = 2 * kBoxBytes;   // a [128 x 128] bf16 operand tile
+constexpr uint32_t kStageBytes = 2 * kTileBytes; // K tile + V tile
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kRescaleThreshold = 8.0f;        // log2 units the running maximum may exceed the reference by
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct TcState {
+  EncodeTiledFn encode;
+};
+
+constexpr uint32_t kIdescKK = make_idesc_bf16(128, 128, false);   // both operands K-major
+constexpr uint32_t kIdescKMN = make_idesc_bf16(128, 128, true);   // B operand MN-major (V in O += P V)
+
+__device__ __forceinline__ uint64_t kmajor_desc(uint32_t addr) { return make_smem_desc(addr, 16, 1024); }
+
+// D[128 x 128] (+)= A[128 x 128] * B[128 x 128]^T, both operands K-major 128B-swizzled [128 x 128] bf16 tiles
+// made of two [128 x 64] boxes.  One thread issues the eight K = 16 steps.
+__device__ __forceinline__ void mma_tile_kk(uint32_t tmem_d, uint32_t a_smem, uint32_t b_smem, bool accumulate) {
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const uint32_t off = (uint32_t)(k >> 2) * kBoxBytes + (uint32_t)(k & 3) * 32u;
+    umma_ss(tmem_d, kmajor_desc(a_smem + off), kmajor_desc(b_smem + off), kIdescKK, accumulate || k > 0);
+  }
+}
+
+// ================================================================================================
+// Pass 1
+// ================================================================================================
+constexpr int kP1Threads = 192;   // warp 0: TMA, warp 1: MMA, warps 2-5: softmax (one thread per query row)
+
+__global__ void __launch_bounds__(kP1Threads, 1)
+tc_pass1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                const __grid_constant__ CUtensorMap tmV, int Hkv, int n, int n_kv, int w, float scale, int splits,
+                float* __restrict__ part_m, float* __restrict__ part_l, float* __restrict__ part_O,
+                unsigned int* __restrict__ dev_status) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bar_q_full, bar_kv_full[2], bar_s_full[2], bar_p_full[2], bar_pv_done[2];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sQ = smem_base;
+  const uint32_t sKV = smem_base + kTileBytes;   // stage s: K at sKV + s*kStageBytes, V right after it
+  uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int split = blockIdx.x, bh = blockIdx.y;
+  const int b = bh / Hkv, h = bh % Hkv;
+
+  const int n_tiles = (n_kv + kTile - 1) / kTile;
+  const int per = (n_tiles + splits - 1) / splits;
+  const int tile0 = split * per;
+  const int T = max(0, min(n_tiles, tile0 + per) - tile0);
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(&bar_q_full, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bar_kv_full[i], 1);
+      mbar_init(&bar_s_full[i], 1);
+      mbar_init(&bar_p_full[i], 128);
+      mbar_init(&bar_pv_done[i], 1);
+    }
+    fence_mbar_init();
+    prefetch_tensormap(&tmQ);
+    prefetch_tensormap(&tmK);
+    prefetch_tensormap(&tmV);
+  }
+  if (warp == 1) {
+    tmem_alloc(&tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_slot;
+  // columns: S0 [0,128) S1 [128,256) O [256,384) P0 [384,448) P1 [448,512)
+  const uint32_t tO = tmem + 256;
+  auto tS = [tmem](int i) { return tmem + (uint32_t)i * 128u; };
+  auto tP = [tmem](int i) { return tmem + 384u + (uint32_t)i * 64u; };
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0 && T > 0) {
+      mbar_arrive_expect_tx(&bar_q_full, kTileBytes);
+      tma_load_3d(gen_base, &tmQ, &bar_q_full, 0, 0, bh);
+      tma_load_3d(gen_base + kBoxBytes, &tmQ, &bar_q_full, 64, 0, bh);
+      for (int it = 0; it < T; ++it) {
+        const int s = it & 1;
+        if (it >= 2 && !mbar_wait(&bar_pv_done[s], ((it >> 1) - 1) & 1, &abort_flag, dev_status, kDevTimeout)) break;
+        uint8_t* dK = gen_base + kTileBytes + (size_t)s * kStageBytes;
+        uint8_t* dV = dK + kTileBytes;
+        const int j0 = (tile0 + it) * kTile;
+        mbar_arrive_expect_tx(&bar_kv_full[s], kStageBytes);
+        tma_load_4d(dK, &tmK, &bar_kv_full[s], 0, j0, h, b);
+        tma_load_4d(dK + kBoxBytes, &tmK, &bar_kv_full[s], 64, j0, h, b);
+        tma_load_4d(dV, &tmV, &bar_kv_full[s], 0, j0, h, b);
+        tma_load_4d(dV + kBoxBytes, &tmV, &bar_kv_full[s], 64, j0, h, b);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0 && T > 0) {
+      bool ok = mbar_wait(&bar_q_full, 0, &abort_flag, dev_status, kDevTimeout) &&
+                mbar_wait(&bar_kv_full[0], 0, &abort_flag, dev_status, kDevTimeout);
+      if (ok) {
+        tc_fence_after();
+        mma_tile_kk(tS(0), sQ, sKV, false);
+        umma_commit(&bar_s_full[0]);
+      }
+      for (int it = 0; ok && it < T; ++it) {
+        const int bsel = it & 1;
+        if (it + 1 < T) {
+          const int nb = (it + 1) & 1;
+          if (!mbar_wait(&bar_kv_full[nb], ((it + 1) >> 1) & 1, &abort_flag, dev_status, kDevTimeout)) break;
+          tc_fence_after();
+          mma_tile_kk(tS(nb), sQ, sKV + (uint32_t)nb * kStageBytes, false);   // S(it+1) = Q K^T
+          umma_commit(&bar_s_full[nb]);
+        }
+        if (!mbar_wait(&bar_p_full[bsel], (it >> 1) & 1, &abort_flag, dev_status, kDevTimeout)) break;
+        tc_fence_after();
+        // O += P(it) V(it): A = P in TMEM (16 tokens = 8 packed columns per step), B = V tile, MN-major
+        const uint32_t sV = sKV + (uint32_t)bsel * kStageBytes + kTileBytes;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const uint64_t bdesc = make_smem_desc(sV + (uint32_t)k * 2048u, kBoxBytes, 1024);
+          umma_ts(tO, tP(bsel) + (uint32_t)k * 8u, bdesc, kIdescKMN, it > 0 || k > 0);
+        }
+        umma_commit(&bar_pv_done[bsel]);
+      }
+    }
+  } else {
+    // ---------------- softmax warps: thread = query row ----------------
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;
+    const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+    const int i_q = row % w;                  // window position of this row (row = g*w + i)
+    const float c2 = scale * kLog2e;
+    float m_ref = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int it = 0; it < T; ++it) {
+      const int bsel = it & 1;
+      if (!mbar_wait(&bar_s_full[bsel], (it >> 1) & 1, &abort_flag, dev_status, kDevTimeout)) { ok = false; break; }
+      tc_fence_after();
+      float s[128];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld32(tS(bsel) + lane_base + c * 32, s + c * 32);
+      tmem_wait_ld();
+      const int j0 = (tile0 + it) * kTile;
+      if (j0 + kTile > n) {   // tile touches rows past the scored prefix: window rows (causal) or padding
+#pragma unroll
+        for (int c = 0; c < 128; ++c) {
+          const int j = j0 + c;
+          const bool vis = (j < n_kv) && (j < n || (j - n) <= i_q);
+          s[c] = vis ? s[c] : -INFINITY;
+        }
+      }
+      float tmax = s[0];
+#pragma unroll
+      for (int c = 1; c < 128; ++c) tmax = fmaxf(tmax, s[c]);
+      const float m_tile = tmax * c2;
+      const bool need = m_tile > m_ref + kRescaleThreshold;   // also true for the first visible entries (m_ref = -inf)
+      float factor = 1.f;
+      if (need) {
+        factor = ex2_approx(m_ref - m_tile);   // 0 when m_ref = -inf
+        l *= factor;
+        m_ref = m_tile;
+      }
+      if (it > 0 && __any_sync(0xffffffffu, need)) {
+        // rescale the running output: needs O += P V of the previous tile to have landed
+        if (!mbar_wait(&bar_pv_done[(it - 1) & 1], ((it - 1) >> 1) & 1, &abort_flag, dev_status, kDevTimeout)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          float o[32];
+          tmem_ld32(tO + lane_base + c * 32, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int u = 0; u < 32; ++u) o[u] *= factor;
+          tmem_st32(tO + lane_base + c * 32, o);
+        }
+      }
+      if (it >= 2 && !mbar_wait(&bar_pv_done[bsel], ((it >> 1) - 1) & 1, &abort_flag, dev_status, kDevTimeout)) {
+        ok = false;
+        break;
+      }
+      const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t packed[16];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) {
+          const float p0 = ex2_approx(fmaf(s[c * 32 + 2 * u], c2, -m_use));
+          const float p1 = ex2_approx(fmaf(s[c * 32 + 2 * u + 1], c2, -m_use));
+          l += p0 + p1;
+          packed[u] = pack_bf16x2(p0, p1);
+        }
+        tmem_st16(tP(bsel) + lane_base + c * 16, packed);
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&bar_p_full[bsel]);
+    }
+    // ---- write the partial (m, l, O) of this split ----
+    const long long o_idx = ((long long)bh * splits + split) * kRows + row;
+    float* Op = part_O + o_idx * kHeadDim;
+    if (T > 0 && ok) ok = mbar_wait(&bar_pv_done[(T - 1) & 1], ((T - 1) >> 1) & 1, &abort_flag, dev_status, kDevTimeout);
+    if (T > 0 && ok) {
+      tc_fence_after();
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        float o[32];
+        tmem_ld32(tO + lane_base + c * 32, o);
+        tmem_wait_ld();
+#pragma unroll
+        for (int u = 0; u < 32; u += 4)
+          *reinterpret_cast<float4*>(Op + c * 32 + u) = make_float4(o[u], o[u + 1], o[u + 2], o[u + 3]);
+      }
+      part_m[o_idx] = (m_ref == -INFINITY) ? -INFINITY : m_ref * kLn2;   // natural-log units
+      part_l[o_idx] = l;
+    } else {
+      for (int u = 0; u < kHeadDim; u += 4) *reinterpret_cast<float4*>(Op + u) = make_float4(0.f, 0.f, 0.f, 0.f);
+      part_m[o_idx] = -INFINITY;
+      part_l[o_idx] = 0.f;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+// ================================================================================================
+// Pass 2
+// ================================================================================================
+constexpr int kP2Threads = 320;   // warp 0: TMA, warp 1: MMA, warps 2-5 and 6-9: two epilogue warpgroups
+
+// Exact ||o - v||^2 for the rare entries whose attention weight is large (the expansion
+// ||o||^2 + ||v||^2 - 2 o.v cancels when o approaches v).
+__device__ __noinline__ float exact_dist2(const float* __restrict__ o_row, const __nv_bfloat16* __restrict__ v_row) {
+  float ss = 0.f;
+  for (int k = 0; k < kHeadDim; k += 2) {
+    const float2 o = *reinterpret_cast<const float2*>(o_row + k);
+    const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(v_row + k);
+    const float d0 = o.x - __low2float(v), d1 = o.y - __high2float(v);
+    ss = fmaf(d0, d0, ss);
+    ss = fmaf(d1, d1, ss);
+  }
+  return ss;
+}
+
+template <int kW>
+__global__ void __launch_bounds__(kP2Threads, 1)
+tc_pass2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmO,
+                const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, int Hkv, int n,
+                float scale, float ema_decay, int splits, const float* __restrict__ fin_M2,
+                const float* __restrict__ fin_on, const float* __restrict__ O_f32,
+                const __nv_bfloat16* __restrict__ V, long long vsb, long long vsh, long long vsn,
+                float* __restrict__ I_hat, unsigned int* __restrict__ dev_status) {
+  constexpr int kG = kRows / kW;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bar_qo_full, bar_kv_full[2], bar_kv_empty[2], bar_acc_full[2], bar_acc_empty[2];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  __shared__ float2 cst[kRows];   // per query row: (M2, ||o||^2)
+
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sQ = smem_base, sO = smem_base + kTileBytes, sKV = smem_base + 2 * kTileBytes;
+  uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int split = blockIdx.x, bh = blockIdx.y;
+  const int b = bh / Hkv, h = bh % Hkv;
+
+  const int n_tiles = (n + kTile - 1) / kTile;   // only the scored prefix rows
+  const int per = (n_tiles + splits - 1) / splits;
+  const int tile0 = split * per;
+  const int T = max(0, min(n_tiles, tile0 + per) - tile0);
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(&bar_qo_full, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bar_kv_full[i], 1);
+      mbar_init(&bar_kv_empty[i], 5);      // MMA commit + one arrival per epilogue warp of the warpgroup
+      mbar_init(&bar_acc_full[i], 1);
+      mbar_init(&bar_acc_empty[i], 128);
+    }
+    fence_mbar_init();
+    prefetch_tensormap(&tmQ);
+    prefetch_tensormap(&tmO);
+    prefetch_tensormap(&tmK);
+    prefetch_tensormap(&tmV);
+  }
+  if (warp == 1) {
+    tmem_alloc(&tmem_slot, 512);
+    tmem_relinquish();
+  }
+  if (threadIdx.x >= 64 && threadIdx.x < 64 + kRows) {
+    const int r = threadIdx.x - 64;
+    cst[r] = make_float2(fin_M2[(long long)bh * kRows + r], fin_on[(long long)bh * kRows + r]);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_slot;   // buffer b: S^T at b*256, C^T at b*256 + 128
+
+  if (warp == 0) {
+    if (lane == 0 && T > 0) {
+      mbar_arrive_expect_tx(&bar_qo_full, 2 * kTileBytes);
+      tma_load_3d(gen_base, &tmQ, &bar_qo_full, 0, 0, bh);
+      tma_load_3d(gen_base + kBoxBytes, &tmQ, &bar_qo_full, 64, 0, bh);
+      tma_load_3d(gen_base + kTileBytes, &tmO, &bar_qo_full, 0, 0, bh);
+      tma_load_3d(gen_base + kTileBytes + kBoxBytes, &tmO, &bar_qo_full, 64, 0, bh);
+      for (int it = 0; it < T; ++it) {
+        const int s = it & 1;
+        if (it >= 2 && !mbar_wait(&bar_kv_empty[s], ((it >> 1) - 1) & 1, &abort_flag, dev_status, kDevTimeout)) break;
+        uint8_t* dK = gen_base + 2 * kTileBytes + (size_t)s * kStageBytes;
+        uint8_t* dV = dK + kTileBytes;
+        const int j0 = (tile0 + it) * kTile;
+        mbar_arrive_expect_tx(&bar_kv_full[s], kStageBytes);
+        tma_load_4d(dK, &tmK, &bar_kv_full[s], 0, j0, h, b);
+        tma_load_4d(dK + kBoxBytes, &tmK, &bar_kv_full[s], 64, j0, h, b);
+        tma_load_4d(dV, &tmV, &bar_kv_full[s], 0, j0, h, b);
+        tma_load_4d(dV + kBoxBytes, &tmV, &bar_kv_full[s], 64, j0, h, b);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && T > 0) {
+      bool ok = mbar_wait(&bar_qo_full, 0, &abort_flag, dev_status, kDevTimeout);
+      for (int it = 0; ok && it < T; ++it) {
+        const int s = it & 1;
+        if (!mbar_wait(&bar_kv_full[s], (it >> 1) & 1, &abort_flag, dev_status, kDevTimeout)) break;
+        if (it >= 2 && !mbar_wait(&bar_acc_empty[s], ((it >> 1) - 1) & 1, &abort_flag, dev_status, kDevTimeout)) break;
+        tc_fence_after();
+        const uint32_t sK = sKV + (uint32_t)s * kStageBytes, sV = sK + kTileBytes;
+        mma_tile_kk(tmem + (uint32_t)s * 256u, sK, sQ, false);          // S^T = K Q^T
+        mma_tile_kk(tmem + (uint32_t)s * 256u + 128u, sV, sO, false);   // C^T = V O^T
+        umma_commit(&bar_acc_full[s]);
+        umma_commit(&bar_kv_empty[s]);
+      }
+    }
+  } else {
+    // ---------------- epilogue: warpgroup wg handles tiles it = wg, wg + 2, ...; thread = token ----------------
+    const int wg = (warp - 2) >> 2;
+    const int quad = warp & 3;
+    const int t_in_tile = quad * 32 + lane;
+    const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+    const float c2 = scale * kLog2e;
+    const float alpha = 1.f - ema_decay;
+    const bool alpha_zero = !(alpha > 0.f);
+    const float k0 = alpha_zero ? 1.f : 1.f / alpha;
+    const float fin_scale = (alpha_zero ? 1.f : alpha) / (float)kG;
+    const float* O_head = O_f32 + (long long)bh * kRows * kHeadDim;
+    const __nv_bfloat16* V_head = V + (long long)b * vsb + (long long)h * vsh;
+
+    for (int it = wg; it < T; it += 2) {
+      const int s = wg;
+      const uint32_t par = (uint32_t)(it >> 1) & 1u;
+      if (!mbar_wait(&bar_kv_full[s], par, &abort_flag, dev_status, kDevTimeout)) break;
+      // ||v||^2 of this thread's token from the swizzled V tile: 16-byte chunk c of row r sits at chunk c ^ (r & 7)
+      float vn = 0.f;
+      {
+        const uint8_t* vt = gen_base + 2 * kTileBytes + (size_t)s * kStageBytes + kTileBytes;
+        const int r = t_in_tile;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const uint8_t* rowp = vt + half * kBoxBytes + (r >> 3) * 1024 + (r & 7) * 128;
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            const uint4 u = *reinterpret_cast<const uint4*>(rowp + ((c ^ (r & 7)) << 4));
+            const unsigned int wv[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const float lo = __uint_as_float(wv[q] << 16), hi = __uint_as_float(wv[q] & 0xFFFF0000u);
+              vn = fmaf(lo, lo, vn);
+              vn = fmaf(hi, hi, vn);
+            }
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bar_kv_empty[s]);
+      if (!mbar_wait(&bar_acc_full[s], par, &abort_flag, dev_status, kDevTimeout)) break;
+      tc_fence_after();
+
+      const int j = (tile0 + it) * kTile + t_in_tile;
+      const uint32_t tSt = tmem + (uint32_t)s * 256u + lane_base, tCt = tSt + 128u;
+      float hacc[kG];
+#pragma unroll
+      for (int g = 0; g < kG; ++g) hacc[g] = 0.f;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        float sv[32], cv[32];
+        __syncwarp();
+        tmem_ld32(tSt + c * 32, sv);
+        tmem_ld32(tCt + c * 32, cv);
+        tmem_wait_ld();
+#pragma unroll
+        for (int u = 0; u < 32; ++u) {
+          const int r = c * 32 + u;          // query row = g * kW + i
+          const int i = r % kW, g = r / kW;
+          const float2 k = cst[r];
+          const float A = ex2_approx(fmaf(sv[u], c2, -k.x));
+          float x = fmaf(-2.f, cv[u], k.y + vn);
+          if (A > 0.125f && j < n) x = exact_dist2(O_head + r * kHeadDim, V_head + (long long)j * vsn);
+          x = fmaxf(x, 0.f);
+          const float y = fmaxf(1.f - A, 5.9604645e-8f);
+          const float I = A * x * rsqrt_approx(fmaxf(x * y * y, 1e-36f));   // A / (1 - A) * sqrt(x)
+          if (i == 0) hacc[g] = I * k0;                                     // EMA seeded with the oldest query
+          else if (!alpha_zero) hacc[g] = fmaf(hacc[g], ema_decay, I);      // Horner form of Eq. 9
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(&bar_acc_empty[s]);
+      float tot = 0.f;
+#pragma unroll
+      for (int g = 0; g < kG; ++g) tot += hacc[g];
+      if (j < n) I_hat[(long long)bh * n + j] = tot * fin_scale;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+CUresult encode_tiles(TcState* st, CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims,
+                      const cuuint64_t* strides_bytes) {
+  cuuint32_t box[4] = {64, 128, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  return st->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), dims,
+                    strides_bytes, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
+bool make_rows_map(TcState* st, CUtensorMap* map, const void* base, int BH) {   // [BH, 128, 128] contiguous
+  cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)kRows, (cuuint64_t)BH};
+  cuuint64_t str[2] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)kRows * kHeadDim * 2};
+  return encode_tiles(st, map, base, 3, dims, str) == CUDA_SUCCESS;
+}
+
+bool make_kv_map(TcState* st, CUtensorMap* map, const void* base, const Problem& p, long long sb, long long sh,
+                 long long sn) {
+  cuuint64_t dims[4] = {(cuuint64_t)p.d, (cuuint64_t)p.n_kv, (cuuint64_t)p.Hkv, (cuuint64_t)p.batch};
+  // a dimension of extent 1 may carry any stride; give it a valid one
+  cuuint64_t str[3] = {(cuuint64_t)sn * 2, (cuuint64_t)(p.Hkv > 1 ? sh : sn) * 2,
+                       (cuuint64_t)(p.batch > 1 ? sb : sn) * 2};
+  return encode_tiles(st, map, base, 4, dims, str) == CUDA_SUCCESS;
+}
+
+constexpr size_t kP1Smem = kTileBytes + 2 * kStageBytes + 1024;        // Q + two K/V stages + alignment slack
+constexpr size_t kP2Smem = 2 * kTileBytes + 2 * kStageBytes + 1024;    // Q + O + two K/V stages + slack
+
+}  // namespace
+
+bool tc_supported(const Problem& p) {
+  if (p.dtype != RESTKV_BF16 || p.d != kHeadDim || p.R != kRows) return false;
+  if (p.w != 16 && p.w != 32 && p.w != 64 && p.w != 128) return false;
+  return true;
+}
+
+cudaError_t tc_init(void** state) {
+  *state = nullptr;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess) return e;
+  if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+  e = cudaFuncSetAttribute(tc_pass1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kP1Smem);
+  if (e != cudaSuccess) return e;
+  cudaFuncSetAttribute(tc_pass2_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kP2Smem);
+  cudaFuncSetAttribute(tc_pass2_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kP2Smem);
+  cudaFuncSetAttribute(tc_pass2_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kP2Smem);
+  e = cudaFuncSetAttribute(tc_pass2_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kP2Smem);
+  if (e != cudaSuccess) return e;
+  static TcState the_state;
+  the_state.encode = (EncodeTiledFn)fn;
+  *state = &the_state;
+  return cudaSuccess;
+}
+
+cudaError_t launch_tc_pass1(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
+                            const void* V, unsigned int* dev_status, cudaStream_t st) {
+  TcState* ts = (TcState*)state;
+  CUtensorMap tmQ, tmK, tmV;
+  if (!make_rows_map(ts, &tmQ, Q, p.BH) || !make_kv_map(ts, &tmK, K, p, p.ksb, p.ksh, p.ksn) ||
+      !make_kv_map(ts, &tmV, V, p, p.vsb, p.vsh, p.vsn))
+    return cudaErrorInvalidValue;
+  dim3 grid(ws.splits, p.BH);
+  tc_pass1_kernel<<<grid, kP1Threads, kP1Smem, st>>>(tmQ, tmK, tmV, p.Hkv, p.n, p.n_kv, p.w, p.scale, ws.splits,
+                                                     ws.part_m, ws.part_l, ws.part_O, dev_status);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_tc_pass2(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
+                            const void* V, float ema_decay, unsigned int* dev_status, cudaStream_t st) {
+  TcState* ts = (TcState*)state;
+  CUtensorMap tmQ, tmO, tmK, tmV;
+  if (!make_rows_map(ts, &tmQ, Q, p.BH) || !make_rows_map(ts, &tmO, ws.O_bf16, p.BH) ||
+      !make_kv_map(ts, &tmK, K, p, p.ksb, p.ksh, p.ksn) || !make_kv_map(ts, &tmV, V, p, p.vsb, p.vsh, p.vsn))
+    return cudaErrorInvalidValue;
+  dim3 grid(ws.splits, p.BH);
+#define RESTKV_P2(W)                                                                                              \
+  tc_pass2_kernel<W><<<grid, kP2Threads, kP2Smem, st>>>(tmQ, tmO, tmK, tmV, p.Hkv, p.n, p.scale, ema_decay,       \
+                                                        ws.splits, ws.fin_M2, ws.fin_on, ws.O_f32,                \
+                                                        (const __nv_bfloat16*)V, p.vsb, p.vsh, p.vsn, ws.I_hat,   \
+                                                        dev_status)
+  switch (p.w) {
+    case 16: RESTKV_P2(16); break;
+    case 32: RESTKV_P2(32); break;
+    case 64: RESTKV_P2(64); break;
+    case 128: RESTKV_P2(128); break;
+    default: return cudaErrorInvalidValue;
+  }
+#undef RESTKV_P2
+  return cudaGetLastError();
+}
+
 }  // namespace restkv
