@@ -93,6 +93,8 @@ size_t restkv_workspace_bytes_adaptive(const restkv_shape* shape, int budget);
  * always the box width).
  *   Q_obs, K, V  device, dtype per shape->dtype
  *   scores       device float [batch, n_kv_heads, n_kv]; rows >= n receive +inf
+ *                When K,V hold a single row (n_kv == 1) every attention weight is 1 and Eq. 7 is 0/0;
+ *                the score of that row is defined as 0.
  *   pool_used    optional device int32 [batch, n_kv_heads, 2] receiving (W, gamma) per head, or NULL
  * RESTKV_BF16 with head_dim 128 and w * (n_q_heads/n_kv_heads) == 128 runs on the tcgen05 tensor-core
  * kernels; every other supported shape (head_dim <= 256 and a multiple of 8, w*group <= 256) runs on

@@ -160,7 +160,14 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
   if (c.h->kernel_path == 1) use_tc = false;
   if (c.h->kernel_path == 2 && !use_tc) return RESTKV_ERR_UNSUPPORTED;
   if (!use_tc && !simt_supported(p)) return RESTKV_ERR_UNSUPPORTED;
-  if (use_tc) {
+  if (p.n_kv == 1) {
+    // A single visible row has A = 1 and nothing to redistribute its weight to: the indicator is
+    // 0/0 there and is defined as 0 (Eq. 7 has no value), so no kernel is needed.
+    cudaError_t e = cudaMemsetAsync(ws.I_hat, 0, (size_t)p.BH * p.n * sizeof(float), c.st);
+    if (e == cudaSuccess && adaptive)
+      e = cudaMemsetAsync(ws.I_raw, 0, (size_t)p.batch * p.Hq * p.w * p.n * sizeof(float), c.st);
+    if (e != cudaSuccess) return c.fail(e);
+  } else if (use_tc) {
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS1, launch_tc_pass1(c.h->tc_state, p, ws, Q, K, V, c.h->dev_status, c.st), 1);
     RESTKV_LAUNCH(c, RESTKV_KERNEL_COMBINE, launch_combine(p, ws, c.st), 1);
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2, launch_tc_pass2(c.h->tc_state, p, ws, Q, K, V, ema_decay, c.h->dev_status, c.st), 1);
