@@ -246,8 +246,9 @@ def main():
     def step():
         handle.evict(shape, Q, K, V, case.ema_decay, pool, case.budget, indices, K_out, V_out, ws)
 
+    # the fused path pools inside the select kernel
     kernel_ids = {"pass1": rk.KERNEL_PASS1, "combine": rk.KERNEL_COMBINE, "pass2": rk.KERNEL_PASS2,
-                  "pool": rk.KERNEL_POOL, "select": rk.KERNEL_SELECT, "compact": rk.KERNEL_COMPACT}
+                  "pool_select": rk.KERNEL_SELECT, "compact": rk.KERNEL_COMPACT}
     prof = {}
     for name, kid in kernel_ids.items():
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

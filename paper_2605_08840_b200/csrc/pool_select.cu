@@ -1,39 +1,37 @@
 // Spatial pooling (Eq. 13), top-B selection and row gather (Eq. 14).
+#include <cooperative_groups.h>
+
 #include "restkv_common.cuh"
 
 namespace restkv {
 
 namespace {
 
+namespace cg = cooperative_groups;
+
 // ------------------------------------------------------------------------------------------------
-__global__ void set_pool_kernel(int* pool, int BH, int W, int gamma) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < BH) { pool[2 * i] = W; pool[2 * i + 1] = gamma; }
+// Box mean of Eq. 13 at row j of one head: (1/W) * sum_{k=-W/2+gamma}^{W/2+gamma} I_hat[j+k], taps outside
+// [0,n) are zero; rows n..n_kv-1 (the window's own tokens) get +inf.
+__device__ __forceinline__ float box_mean(const float* __restrict__ src, int n, int j, int W, int gamma) {
+  if (j >= n) return INFINITY;
+  const int half = W / 2;
+  long long lo = (long long)j - half + gamma, hi = (long long)j + half + gamma;
+  if (lo < 0) lo = 0;
+  if (hi > n - 1) hi = n - 1;
+  float s = 0.f;
+  for (long long t = lo; t <= hi; ++t) s += src[t];
+  return s / (float)W;
 }
 
-// scores[j] = (1/W) * sum_{k=-W/2+gamma}^{W/2+gamma} I_hat[j+k], taps outside [0,n) are zero;
-// rows n..n_kv-1 (the window's own tokens) get +inf.  grid (ceil(n_kv/256), BH).
-__global__ void pool_kernel(int n, int n_kv, const float* __restrict__ I_hat, const int* __restrict__ pool,
-                            float* __restrict__ scores, int32_t* __restrict__ pool_used) {
+// grid (ceil(n_kv/256), BH).  The window (W, gamma) comes from `pool` (per head, device) when it is non-null.
+__global__ void pool_kernel(int n, int n_kv, const float* __restrict__ I_hat, const int* __restrict__ pool, int W,
+                            int gamma, float* __restrict__ scores, int32_t* __restrict__ pool_used) {
   const int bh = blockIdx.y;
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  const int W = pool[2 * bh], gamma = pool[2 * bh + 1];
+  if (pool) { W = pool[2 * bh]; gamma = pool[2 * bh + 1]; }
   if (pool_used && j == 0) { pool_used[2 * bh] = W; pool_used[2 * bh + 1] = gamma; }
   if (j >= n_kv) return;
-  float out;
-  if (j >= n) {
-    out = INFINITY;
-  } else {
-    const float* src = I_hat + (long long)bh * n;
-    const int half = W / 2;
-    long long lo = (long long)j - half + gamma, hi = (long long)j + half + gamma;
-    if (lo < 0) lo = 0;
-    if (hi > n - 1) hi = n - 1;
-    float s = 0.f;
-    for (long long t = lo; t <= hi; ++t) s += src[t];
-    out = s / (float)W;
-  }
-  scores[(long long)bh * n_kv + j] = out;
+  scores[(long long)bh * n_kv + j] = box_mean(I_hat + (long long)bh * n, n, j, W, gamma);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -44,90 +42,174 @@ __device__ __forceinline__ unsigned int float_key(float x) {
 }
 
 constexpr int kSelThreads = 1024;
+constexpr int kSelBins = 2048;
+constexpr int kSelMaxSmemKeys = 48 * 1024;   // keys of one CTA's slice kept in shared memory (192 KB)
 
-// One block per row.  Four 8-bit passes from the most significant digit find the key T of the
-// keep-th largest score and how many scores are strictly larger; a last ordered pass writes, in
-// ascending index order, every index whose key is > T plus the first (keep - #larger) indices
-// whose key equals T (lower index wins ties).
-__global__ void __launch_bounds__(kSelThreads) select_kernel(int n_kv, int keep, const float* __restrict__ scores,
-                                                             int32_t* __restrict__ indices) {
-  __shared__ unsigned int hist[256];
-  __shared__ unsigned int s_prefix, s_remaining;
-  __shared__ unsigned int warp_sel[32], warp_eq[32];
-  __shared__ unsigned int s_base_sel, s_base_eq;
+// Inclusive scan over the 1024 threads of the block, in thread order.
+__device__ __forceinline__ unsigned int block_inclusive_scan(unsigned int v, unsigned int* warp_sums) {
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const unsigned int t = __shfl_up_sync(0xffffffffu, v, off);
+    if (lane >= off) v += t;
+  }
+  if (lane == 31) warp_sums[wid] = v;
+  __syncthreads();
+  if (wid == 0) {
+    unsigned int w = warp_sums[lane];
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const unsigned int t = __shfl_up_sync(0xffffffffu, w, off);
+      if (lane >= off) w += t;
+    }
+    warp_sums[lane] = w;   // inclusive over warps
+  }
+  __syncthreads();
+  if (wid > 0) v += warp_sums[wid - 1];
+  __syncthreads();   // warp_sums may be reused by the caller
+  return v;
+}
 
-  const int row = blockIdx.x;
-  const float* src = scores + (long long)row * n_kv;
-  int32_t* dst = indices + (long long)row * keep;
+// One thread-block cluster per row; CTA `rank` of the cluster owns the contiguous slice [rank*per, (rank+1)*per)
+// of the row.  With I_hat non-null the kernel first applies the box mean of Eq. 13 and writes the pooled scores;
+// otherwise it reads `scores`.  The keys of the slice stay in shared memory (use_smem) or are re-read from
+// `scores`.  Three radix passes (11, 11 and 10 bits from the top; per-CTA histograms summed through distributed
+// shared memory) find the key T of the keep-th largest score and how many scores equal to T are kept; an ordered
+// pass then writes, in ascending index order, every index whose key is > T plus the first kept ones whose key
+// equals T (lower index wins ties).
+__global__ void __launch_bounds__(kSelThreads, 1)
+select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const int* __restrict__ pool, int W,
+              int gamma, float* scores, int32_t* __restrict__ indices, int32_t* __restrict__ pool_used, int per,
+              int use_smem) {
+  cg::cluster_group cluster = cg::this_cluster();
+  const unsigned int CS = cluster.num_blocks(), rank = cluster.block_rank();
+  const int row = blockIdx.x / CS;
+  extern __shared__ unsigned int skeys[];
+  __shared__ unsigned int hist[kSelBins];
+  __shared__ unsigned int warp_a[32], warp_b[32];
+  __shared__ unsigned int s_digit, s_remaining;
+  __shared__ unsigned int cta_counts[2];
+
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const long long j0 = (long long)rank * per;
+  const int cnt = (int)max(0ll, min((long long)n_kv, j0 + per) - j0);
+  float* srow = scores + (long long)row * n_kv;
+  int32_t* dst = indices + (long long)row * keep;
 
-  if (keep >= n_kv) {   // budget covers everything: identity
-    for (int j = tid; j < n_kv; j += kSelThreads) dst[j] = j;
+  // ---- keys of the slice ----
+  if (I_hat) {
+    if (pool) { W = pool[2 * row]; gamma = pool[2 * row + 1]; }
+    if (pool_used && rank == 0 && tid == 0) { pool_used[2 * row] = W; pool_used[2 * row + 1] = gamma; }
+    const float* src = I_hat + (long long)row * n;
+    for (int jj = tid; jj < cnt; jj += kSelThreads) {
+      const float out = box_mean(src, n, (int)(j0 + jj), W, gamma);
+      srow[j0 + jj] = out;
+      if (use_smem) skeys[jj] = float_key(out);
+    }
+  } else if (use_smem) {
+    for (int jj = tid; jj < cnt; jj += kSelThreads) skeys[jj] = float_key(srow[j0 + jj]);
+  }
+  __syncthreads();
+  auto key_at = [&](int jj) -> unsigned int { return use_smem ? skeys[jj] : float_key(srow[j0 + jj]); };
+
+  if (keep >= n_kv) {   // budget covers everything: identity (uniform over the cluster)
+    for (int jj = tid; jj < cnt; jj += kSelThreads) dst[j0 + jj] = (int32_t)(j0 + jj);
     return;
   }
 
-  unsigned int prefix = 0, remaining = keep;   // remaining: rank (1-based) still to find inside the prefix class
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
-    const unsigned int mask_hi = (pass == 0) ? 0u : (0xFFFFFFFFu << (shift + 8));
-    if (tid < 256) hist[tid] = 0;
+  // ---- radix passes ----
+  unsigned int prefix = 0, mask_hi = 0, remaining = (unsigned int)keep;
+#pragma unroll 1
+  for (int pass = 0; pass < 3; ++pass) {
+    const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+    const unsigned int dmask = pass == 2 ? 1023u : 2047u;
+    for (int b = tid; b < kSelBins; b += kSelThreads) hist[b] = 0;
     __syncthreads();
-    for (int j = tid; j < n_kv; j += kSelThreads) {
-      const unsigned int key = float_key(src[j]);
-      if ((key & mask_hi) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
-    }
-    __syncthreads();
-    if (tid == 0) {
-      unsigned int acc = 0;
-      int digit = 255;
-      for (; digit > 0; --digit) {
-        if (acc + hist[digit] >= remaining) break;
-        acc += hist[digit];
+    for (int base = 0; base < cnt; base += kSelThreads) {
+      const int jj = base + tid;
+      unsigned int digit = 0xFFFFFFFFu;
+      if (jj < cnt) {
+        const unsigned int key = key_at(jj);
+        if ((key & mask_hi) == prefix) digit = (key >> shift) & dmask;
       }
-      s_prefix = prefix | ((unsigned int)digit << shift);
-      s_remaining = remaining - acc;
+      const unsigned int peers = __match_any_sync(0xffffffffu, digit);
+      if (digit != 0xFFFFFFFFu && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], (unsigned int)__popc(peers));
     }
     __syncthreads();
-    prefix = s_prefix;
+    cluster.sync();
+    // totals over the cluster of this thread's two bins (bins in descending order along the threads)
+    const int b0 = kSelBins - 1 - 2 * tid;
+    unsigned int t0 = 0, t1 = 0;
+    for (unsigned int r = 0; r < CS; ++r) {
+      const unsigned int* rh = cluster.map_shared_rank(hist, r);
+      t0 += rh[b0];
+      t1 += rh[b0 - 1];
+    }
+    const unsigned int incl = block_inclusive_scan(t0 + t1, warp_a);
+    const unsigned int excl = incl - (t0 + t1);
+    if (excl < remaining && remaining <= incl) {   // exactly one thread
+      if (excl + t0 >= remaining) { s_digit = (unsigned int)b0; s_remaining = remaining - excl; }
+      else { s_digit = (unsigned int)(b0 - 1); s_remaining = remaining - excl - t0; }
+    }
+    __syncthreads();
+    prefix |= s_digit << shift;
+    mask_hi |= dmask << shift;
     remaining = s_remaining;
-    __syncthreads();
+    cluster.sync();   // no CTA clears its histogram while a peer still reads it
   }
-  const unsigned int T = prefix;          // key of the keep-th largest score
-  const unsigned int need_eq = remaining; // how many keys equal to T are kept (>= 1)
+  const unsigned int T = prefix;            // key of the keep-th largest score
+  const unsigned int need_eq = remaining;   // how many keys equal to T are kept (>= 1)
 
-  if (tid == 0) { s_base_sel = 0; s_base_eq = 0; }
-  __syncthreads();
-  for (int j0 = 0; j0 < n_kv; j0 += kSelThreads) {
-    const int j = j0 + tid;
-    unsigned int key = 0;
-    const bool in = j < n_kv;
-    if (in) key = float_key(src[j]);
-    const bool gt = in && key > T;
-    const bool eq = in && key == T;
-    // rank among equal keys, in index order
-    const unsigned int eq_mask = __ballot_sync(0xffffffffu, eq);
-    const unsigned int eq_before_in_warp = __popc(eq_mask & ((1u << lane) - 1u));
-    if (lane == 0) warp_eq[wid] = __popc(eq_mask);
-    __syncthreads();
-    unsigned int eq_before = s_base_eq + eq_before_in_warp;
-    for (int wv = 0; wv < wid; ++wv) eq_before += warp_eq[wv];
-    const bool sel = gt || (eq && eq_before < need_eq);
-    const unsigned int sel_mask = __ballot_sync(0xffffffffu, sel);
-    const unsigned int sel_before_in_warp = __popc(sel_mask & ((1u << lane) - 1u));
-    if (lane == 0) warp_sel[wid] = __popc(sel_mask);
-    __syncthreads();
-    unsigned int pos = s_base_sel + sel_before_in_warp;
-    for (int wv = 0; wv < wid; ++wv) pos += warp_sel[wv];
-    if (sel && pos < (unsigned int)keep) dst[pos] = j;
-    __syncthreads();
-    if (tid == 0) {
-      unsigned int a = 0, c = 0;
-      for (int wv = 0; wv < 32; ++wv) { a += warp_sel[wv]; c += warp_eq[wv]; }
-      s_base_sel += a;
-      s_base_eq += c;
-    }
-    __syncthreads();
+  // ---- ordered emit: warp `wid` owns a contiguous run of the slice ----
+  const int cw = (((cnt + 31) / 32) + 31) & ~31;
+  const int wbeg = min(cnt, wid * cw), wend = min(cnt, wbeg + cw);
+  const unsigned int lt_mask = (1u << lane) - 1u;
+  unsigned int cgt = 0, ceq = 0;
+  for (int base = wbeg; base < wend; base += 32) {
+    const int jj = base + lane;
+    const bool valid = jj < wend;
+    const unsigned int key = valid ? key_at(jj) : 0u;
+    cgt += __popc(__ballot_sync(0xffffffffu, valid && key > T));
+    ceq += __popc(__ballot_sync(0xffffffffu, valid && key == T));
   }
+  if (lane == 0) { warp_a[wid] = cgt; warp_b[wid] = ceq; }
+  __syncthreads();
+  if (wid == 0) {
+    unsigned int a = warp_a[lane], b = warp_b[lane];
+    const unsigned int a_own = a, b_own = b;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const unsigned int ta = __shfl_up_sync(0xffffffffu, a, off), tb = __shfl_up_sync(0xffffffffu, b, off);
+      if (lane >= off) { a += ta; b += tb; }
+    }
+    warp_a[lane] = a - a_own;   // exclusive over the warps
+    warp_b[lane] = b - b_own;
+    if (lane == 31) { cta_counts[0] = a; cta_counts[1] = b; }
+  }
+  __syncthreads();
+  cluster.sync();
+  unsigned int run_gt = warp_a[wid], run_eq = warp_b[wid];
+  for (unsigned int r = 0; r < rank; ++r) {
+    const unsigned int* rc = cluster.map_shared_rank(cta_counts, r);
+    run_gt += rc[0];
+    run_eq += rc[1];
+  }
+  for (int base = wbeg; base < wend; base += 32) {
+    const int jj = base + lane;
+    const bool valid = jj < wend;
+    const unsigned int key = valid ? key_at(jj) : 0u;
+    const bool gt = valid && key > T, eq = valid && key == T;
+    const unsigned int mgt = __ballot_sync(0xffffffffu, gt), meq = __ballot_sync(0xffffffffu, eq);
+    const unsigned int gt_before = run_gt + __popc(mgt & lt_mask);
+    const unsigned int eq_before = run_eq + __popc(meq & lt_mask);
+    if (gt || (eq && eq_before < need_eq)) {
+      const unsigned int pos = gt_before + min(eq_before, need_eq);
+      if (pos < (unsigned int)keep) dst[pos] = (int32_t)(j0 + jj);
+    }
+    run_gt += __popc(mgt);
+    run_eq += __popc(meq);
+  }
+  cluster.sync();   // shared memory stays alive until every peer has read cta_counts
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -160,23 +242,40 @@ __global__ void compact_kernel(int Hkv, int n_kv, int n_sel, int row_chunks, lon
 
 }  // namespace
 
-cudaError_t launch_set_pool(const Problem& p, const Workspace& ws, int W, int gamma, cudaStream_t st) {
-  set_pool_kernel<<<(p.BH + 127) / 128, 128, 0, st>>>(ws.pool, p.BH, W, gamma);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_pool(const Problem& p, const Workspace& ws, float* scores, int32_t* pool_used, cudaStream_t st) {
+cudaError_t launch_pool(const Problem& p, const Workspace& ws, const int* pool_dev, int W, int gamma, float* scores,
+                        int32_t* pool_used, cudaStream_t st) {
   dim3 grid((p.n_kv + 255) / 256, p.BH);
-  pool_kernel<<<grid, 256, 0, st>>>(p.n, p.n_kv, ws.I_hat, ws.pool, scores, pool_used);
+  pool_kernel<<<grid, 256, 0, st>>>(p.n, p.n_kv, ws.I_hat, pool_dev, W, gamma, scores, pool_used);
   return cudaGetLastError();
 }
 
-cudaError_t launch_select(int rows, int n_kv, int budget, const float* scores, int32_t* indices,
-                          unsigned int* scratch, cudaStream_t st) {
-  (void)scratch;
+// rows x n_kv scores -> rows x min(budget, n_kv) indices.  I_hat non-null: pool first (n scored rows per row of
+// I_hat, window from pool_dev or (W, gamma)) and write the pooled scores.
+cudaError_t launch_select(int rows, int n, int n_kv, int budget, const float* I_hat, const int* pool_dev, int W,
+                          int gamma, float* scores, int32_t* indices, int32_t* pool_used, cudaStream_t st) {
   const int keep = budget < n_kv ? budget : n_kv;
-  select_kernel<<<rows, kSelThreads, 0, st>>>(n_kv, keep, scores, indices);
-  return cudaGetLastError();
+  const int CS = n_kv > 4096 ? 8 : 1;
+  int per = (n_kv + CS - 1) / CS;
+  per = (per + 3) & ~3;
+  const int use_smem = per <= kSelMaxSmemKeys ? 1 : 0;
+  const size_t smem = use_smem ? (size_t)per * sizeof(unsigned int) : 0;
+  cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kSelMaxSmemKeys * (int)sizeof(unsigned int));
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned int)(rows * CS));
+  cfg.blockDim = dim3(kSelThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CS;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, select_kernel, n, n_kv, keep, I_hat, pool_dev, W, gamma, scores, indices, pool_used,
+                            per, use_smem);
 }
 
 cudaError_t launch_compact(const Problem& p, const void* K, const void* V, const int32_t* indices, int n_sel,

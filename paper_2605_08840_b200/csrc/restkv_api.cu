@@ -151,7 +151,8 @@ struct Call {
     (call).h->launches += (count);                                                              \
   } while (0)
 
-// score: pass 1, combine, pass 2, window parameters, pooling.  `scores` must be non-null here.
+// score: pass 1, combine, pass 2, window parameters and, when `scores` is non-null, pooling.  With `scores`
+// null the caller pools (the fused path does it inside the select kernel).
 static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, const void* Q, const void* K,
                                const void* V, float ema_decay, const restkv_pool_params* pool, float* scores,
                                int32_t* pool_used) {
@@ -181,10 +182,10 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
     cudaError_t e = launch_adaptive_params(p, ws, pool->budget, pool->beta, pool->base_width, c.st, &nl);
     if (e != cudaSuccess) return c.fail(e);
     c.h->launches += nl;
-  } else {
-    RESTKV_LAUNCH(c, RESTKV_KERNEL_NONE, launch_set_pool(p, ws, pool->width, pool->shift, c.st), 1);
   }
-  RESTKV_LAUNCH(c, RESTKV_KERNEL_POOL, launch_pool(p, ws, scores, pool_used, c.st), 1);
+  if (scores)
+    RESTKV_LAUNCH(c, RESTKV_KERNEL_POOL,
+                  launch_pool(p, ws, adaptive ? ws.pool : nullptr, pool->width, pool->shift, scores, pool_used, c.st), 1);
   return RESTKV_OK;
 }
 
@@ -281,7 +282,9 @@ restkv_status restkv_select(restkv_handle* h, const restkv_shape* shape, const f
   Workspace ws;
   if ((s = check_ws(p, budget, h->sm_count, false, workspace, workspace_bytes, &ws)) != RESTKV_OK) return s;
   Call c{h, (cudaStream_t)stream};
-  RESTKV_LAUNCH(c, RESTKV_KERNEL_SELECT, launch_select(p.BH, p.n_kv, budget, scores, indices, ws.sel_scratch, c.st), 1);
+  RESTKV_LAUNCH(c, RESTKV_KERNEL_SELECT,
+                launch_select(p.BH, p.n, p.n_kv, budget, nullptr, nullptr, 1, 0, const_cast<float*>(scores), indices, nullptr,
+                              c.st), 1);
   return RESTKV_OK;
 }
 
@@ -316,8 +319,11 @@ restkv_status restkv_evict(restkv_handle* h, const restkv_shape* shape, const vo
   if ((s = check_ws(p, ws_budget, h->sm_count, adaptive, workspace, workspace_bytes, &ws)) != RESTKV_OK) return s;
   Call c{h, (cudaStream_t)stream};
   float* scores = scores_out ? scores_out : ws.scores;
-  if ((s = run_score(c, p, ws, Q_obs, K, V, ema_decay, pool, scores, nullptr)) != RESTKV_OK) return s;
-  RESTKV_LAUNCH(c, RESTKV_KERNEL_SELECT, launch_select(p.BH, p.n_kv, budget, scores, indices, ws.sel_scratch, c.st), 1);
+  if ((s = run_score(c, p, ws, Q_obs, K, V, ema_decay, pool, nullptr, nullptr)) != RESTKV_OK) return s;
+  // pooling (Eq. 13) runs inside the select kernel, which also writes the pooled scores
+  RESTKV_LAUNCH(c, RESTKV_KERNEL_SELECT,
+                launch_select(p.BH, p.n, p.n_kv, budget, ws.I_hat, adaptive ? ws.pool : nullptr, pool->width,
+                              pool->shift, scores, indices, nullptr, c.st), 1);
   const int n_sel = budget < p.n_kv ? budget : p.n_kv;
   RESTKV_LAUNCH(c, RESTKV_KERNEL_COMPACT, launch_compact(p, K, V, indices, n_sel, K_out, V_out, h->dev_status, c.st), 1);
   return RESTKV_OK;
