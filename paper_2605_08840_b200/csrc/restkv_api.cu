@@ -54,10 +54,9 @@ size_t plan_workspace(const Problem& p, int budget, int sm_count, bool adaptive,
   w.part_O = (float*)take(BH * w.splits * R * d * sizeof(float));
   w.fin_m = (float*)take(BH * R * sizeof(float));
   w.fin_l = (float*)take(BH * R * sizeof(float));
-  w.fin_M2 = (float*)take(BH * R * sizeof(float));
-  w.fin_on = (float*)take(BH * R * sizeof(float));
   w.O_f32 = (float*)take(BH * R * d * sizeof(float));
-  w.O_bf16 = (__nv_bfloat16*)take(BH * R * d * sizeof(__nv_bfloat16));
+  w.O_m2 = (__nv_bfloat16*)take(BH * R * d * sizeof(__nv_bfloat16));
+  w.aug = (__nv_bfloat16*)take(BH * R * 64 * sizeof(__nv_bfloat16));
   w.I_hat = (float*)take(BH * (size_t)p.n * sizeof(float));
   w.scores = (float*)take(BH * (size_t)p.n_kv * sizeof(float));
   w.pool = (int*)take(BH * 2 * sizeof(int));
@@ -157,7 +156,8 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
                                const void* V, float ema_decay, const restkv_pool_params* pool, float* scores,
                                int32_t* pool_used) {
   const bool adaptive = pool->mode == RESTKV_POOL_ADAPTIVE;
-  bool use_tc = tc_supported(p) && c.h->tc_state != nullptr && !adaptive;
+  // the tensor-core pass 2 seeds its EMA chain with 1/alpha, so ema_decay = 1 (alpha = 0) runs on the SIMT kernels
+  bool use_tc = tc_supported(p) && c.h->tc_state != nullptr && !adaptive && ema_decay < 1.f;
   if (c.h->kernel_path == 1) use_tc = false;
   if (c.h->kernel_path == 2 && !use_tc) return RESTKV_ERR_UNSUPPORTED;
   if (!use_tc && !simt_supported(p)) return RESTKV_ERR_UNSUPPORTED;

@@ -34,10 +34,9 @@ struct Workspace {
   float* part_O;          // [BH, splits, R, d]
   float* fin_m;           // [BH, R]    row max of the scaled logits (natural units)
   float* fin_l;           // [BH, R]    sum of exp(s - m)
-  float* fin_M2;          // [BH, R]    m*log2(e) + log2(l): A = exp2(s*scale*log2(e) - M2)
-  float* fin_on;          // [BH, R]    squared norm of the bf16-rounded output row
   float* O_f32;           // [BH, R, d]
-  __nv_bfloat16* O_bf16;  // [BH, R, d]
+  __nv_bfloat16* O_m2;    // [BH, R, d]   -2 * bf16(O)
+  __nv_bfloat16* aug;     // [BH, R, 64]  per-row constants as bf16 pieces (see combine_kernel)
   float* I_hat;           // [BH, n]
   float* scores;          // [BH, n_kv] (used when the caller passes no scores buffer)
   int* pool;              // [BH, 2] (W, gamma)

@@ -273,7 +273,24 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 // ================================================================================================
 // Pass 2
 // ================================================================================================
-constexpr int kP2Threads = 320;   // warp 0: TMA, warp 1: MMA, warps 2-5 and 6-9: two epilogue warpgroups
+// Warp 0: TMA producer.  Warp 1: MMA issuer.  Warps 2-17: four epilogue warpgroups; all of them work on the same
+// tile, warpgroup c on accumulator columns [32c, 32c + 32) (one thread per token and 32 query rows).
+//
+// The per-query-row constants ride through the tensor core: one extra K = 16 step against a block of ones adds
+//   -(m*log2e + log2 l)/(scale*log2e)  to  S^T = K Q^T      (so that exp2(-scale*log2e * S') = 1/A), and
+//   ||o||^2                            to  C^T = V (-2 O)^T (so that C' + ||v||^2 = ||o - v||^2),
+// which leaves the epilogue without any per-column operand.  With u = 1/A and x = ||o - v||^2 the indicator is
+//   A/(1-A) * sqrt(x) = sqrt(x)/(u - 1) = x * rsqrt(x * (u-1)^2).
+constexpr int kP2EpiWarps = 16;
+constexpr int kP2EpiThreads = kP2EpiWarps * 32;
+constexpr int kP2Threads = 64 + kP2EpiThreads;
+constexpr uint32_t kAugBytes = kBoxBytes;     // [128 rows x 64 bf16], only K steps 0 (S') and 1 (C') are used
+constexpr uint32_t kOnesBytes = 1024;         // one 8-row group of ones, shared by all 16 groups (stride 0)
+constexpr float kHeavyA = 0.125f;             // attention weight above which ||o - v||^2 is recomputed exactly
+
+__device__ __forceinline__ void named_barrier_sync(int id, int count) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
 
 // Exact ||o - v||^2 for the rare entries whose attention weight is large (the expansion
 // ||o||^2 + ||v||^2 - 2 o.v cancels when o approaches v).
@@ -292,21 +309,23 @@ __device__ __noinline__ float exact_dist2(const float* __restrict__ o_row, const
 template <int kW>
 __global__ void __launch_bounds__(kP2Threads, 1)
 tc_pass2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmO,
-                const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, int Hkv, int n,
-                float scale, float ema_decay, int splits, const float* __restrict__ fin_M2,
-                const float* __restrict__ fin_on, const float* __restrict__ O_f32,
-                const __nv_bfloat16* __restrict__ V, long long vsb, long long vsh, long long vsn,
-                float* __restrict__ I_hat, unsigned int* __restrict__ dev_status) {
+                const __grid_constant__ CUtensorMap tmAug, const __grid_constant__ CUtensorMap tmK,
+                const __grid_constant__ CUtensorMap tmV, int Hkv, int n, float scale, float ema_decay, int splits,
+                const float* __restrict__ O_f32, const __nv_bfloat16* __restrict__ V, long long vsb, long long vsh,
+                long long vsn, float* __restrict__ I_hat, unsigned int* __restrict__ dev_status) {
   constexpr int kG = kRows / kW;
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bar_qo_full, bar_kv_full[2], bar_kv_empty[2], bar_acc_full[2], bar_acc_empty[2];
+  __shared__ __align__(8) uint64_t bar_const_full, bar_kv_full[2], bar_kv_empty[2], bar_acc_full[2], bar_acc_empty[2];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
-  __shared__ float2 cst[kRows];   // per query row: (M2, ||o||^2)
+  __shared__ float vn_part[2][4][kTile];   // ||v||^2 of each token, one quarter of the row per warpgroup
+  __shared__ float red[2][4][kTile];       // per-warpgroup share of the token's score
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t sQ = smem_base, sO = smem_base + kTileBytes, sKV = smem_base + 2 * kTileBytes;
+  const uint32_t sQ = smem_base, sO = sQ + kTileBytes, sAug = sO + kTileBytes, sOnes = sAug + kAugBytes;
+  const uint32_t sKV = sOnes + kOnesBytes;
   uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
+  uint8_t* gen_kv = gen_base + (sKV - smem_base);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, bh = blockIdx.y;
@@ -319,16 +338,17 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
-    mbar_init(&bar_qo_full, 1);
+    mbar_init(&bar_const_full, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&bar_kv_full[i], 1);
-      mbar_init(&bar_kv_empty[i], 5);      // MMA commit + one arrival per epilogue warp of the warpgroup
+      mbar_init(&bar_kv_empty[i], 1 + kP2EpiWarps);   // MMA commit + one arrival per epilogue warp
       mbar_init(&bar_acc_full[i], 1);
-      mbar_init(&bar_acc_empty[i], 128);
+      mbar_init(&bar_acc_empty[i], kP2EpiWarps);
     }
     fence_mbar_init();
     prefetch_tensormap(&tmQ);
     prefetch_tensormap(&tmO);
+    prefetch_tensormap(&tmAug);
     prefetch_tensormap(&tmK);
     prefetch_tensormap(&tmV);
   }
@@ -336,26 +356,26 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     tmem_alloc(&tmem_slot, 512);
     tmem_relinquish();
   }
-  if (threadIdx.x >= 64 && threadIdx.x < 64 + kRows) {
-    const int r = threadIdx.x - 64;
-    cst[r] = make_float2(fin_M2[(long long)bh * kRows + r], fin_on[(long long)bh * kRows + r]);
-  }
+  if (threadIdx.x >= 64 && threadIdx.x < 64 + (int)(kOnesBytes / 4))   // the block of ones (bf16 1.0 = 0x3F80)
+    reinterpret_cast<uint32_t*>(gen_base + (sOnes - smem_base))[threadIdx.x - 64] = 0x3F803F80u;
+  fence_proxy_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = tmem_slot;   // buffer b: S^T at b*256, C^T at b*256 + 128
+  const uint32_t tmem = tmem_slot;   // buffer b: S' at b*256, C' at b*256 + 128
 
   if (warp == 0) {
     if (lane == 0 && T > 0) {
-      mbar_arrive_expect_tx(&bar_qo_full, 2 * kTileBytes);
-      tma_load_3d(gen_base, &tmQ, &bar_qo_full, 0, 0, bh);
-      tma_load_3d(gen_base + kBoxBytes, &tmQ, &bar_qo_full, 64, 0, bh);
-      tma_load_3d(gen_base + kTileBytes, &tmO, &bar_qo_full, 0, 0, bh);
-      tma_load_3d(gen_base + kTileBytes + kBoxBytes, &tmO, &bar_qo_full, 64, 0, bh);
+      mbar_arrive_expect_tx(&bar_const_full, 2 * kTileBytes + kAugBytes);
+      tma_load_3d(gen_base, &tmQ, &bar_const_full, 0, 0, bh);
+      tma_load_3d(gen_base + kBoxBytes, &tmQ, &bar_const_full, 64, 0, bh);
+      tma_load_3d(gen_base + kTileBytes, &tmO, &bar_const_full, 0, 0, bh);
+      tma_load_3d(gen_base + kTileBytes + kBoxBytes, &tmO, &bar_const_full, 64, 0, bh);
+      tma_load_3d(gen_base + 2 * kTileBytes, &tmAug, &bar_const_full, 0, 0, bh);
       for (int it = 0; it < T; ++it) {
         const int s = it & 1;
         if (it >= 2 && !mbar_wait(&bar_kv_empty[s], ((it >> 1) - 1) & 1, &abort_flag, dev_status, kDevTimeout)) break;
-        uint8_t* dK = gen_base + 2 * kTileBytes + (size_t)s * kStageBytes;
+        uint8_t* dK = gen_kv + (size_t)s * kStageBytes;
         uint8_t* dV = dK + kTileBytes;
         const int j0 = (tile0 + it) * kTile;
         mbar_arrive_expect_tx(&bar_kv_full[s], kStageBytes);
@@ -367,96 +387,142 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
   } else if (warp == 1) {
     if (lane == 0 && T > 0) {
-      bool ok = mbar_wait(&bar_qo_full, 0, &abort_flag, dev_status, kDevTimeout);
+      bool ok = mbar_wait(&bar_const_full, 0, &abort_flag, dev_status, kDevTimeout);
+      const uint64_t ones_desc = make_smem_desc(sOnes, 16, 0);   // every 8-row group reads the same block
+      const uint64_t aug_s = kmajor_desc(sAug), aug_c = kmajor_desc(sAug + 32u);
       for (int it = 0; ok && it < T; ++it) {
         const int s = it & 1;
         if (!mbar_wait(&bar_kv_full[s], (it >> 1) & 1, &abort_flag, dev_status, kDevTimeout)) break;
         if (it >= 2 && !mbar_wait(&bar_acc_empty[s], ((it >> 1) - 1) & 1, &abort_flag, dev_status, kDevTimeout)) break;
         tc_fence_after();
         const uint32_t sK = sKV + (uint32_t)s * kStageBytes, sV = sK + kTileBytes;
-        mma_tile_kk(tmem + (uint32_t)s * 256u, sK, sQ, false);          // S^T = K Q^T
-        mma_tile_kk(tmem + (uint32_t)s * 256u + 128u, sV, sO, false);   // C^T = V O^T
+        const uint32_t tS = tmem + (uint32_t)s * 256u, tC = tS + 128u;
+        mma_tile_kk(tS, sK, sQ, false);                       // S^T = K Q^T
+        umma_ss(tS, ones_desc, aug_s, kIdescKK, true);        //   + row constant
+        mma_tile_kk(tC, sV, sO, false);                       // C^T = V (-2 O)^T
+        umma_ss(tC, ones_desc, aug_c, kIdescKK, true);        //   + ||o||^2
         umma_commit(&bar_acc_full[s]);
         umma_commit(&bar_kv_empty[s]);
       }
     }
   } else {
-    // ---------------- epilogue: warpgroup wg handles tiles it = wg, wg + 2, ...; thread = token ----------------
-    const int wg = (warp - 2) >> 2;
-    const int quad = warp & 3;
-    const int t_in_tile = quad * 32 + lane;
+    // ---------------- epilogue: thread = token, warpgroup = 32 query rows ----------------
+    const int cgp = (warp - 2) >> 2;                 // column group 0..3
+    const int quad = warp & 3;                       // TMEM lane quarter this warp may touch
+    const int t = quad * 32 + lane;
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-    const float c2 = scale * kLog2e;
-    const float alpha = 1.f - ema_decay;
-    const bool alpha_zero = !(alpha > 0.f);
-    const float k0 = alpha_zero ? 1.f : 1.f / alpha;
-    const float fin_scale = (alpha_zero ? 1.f : alpha) / (float)kG;
+    const float neg_c2 = -scale * kLog2e;
+    const float heavy_thr = log2f(1.f / kHeavyA) / neg_c2;   // S' above this <=> A > kHeavyA
+    const float alpha = 1.f - ema_decay;                     // > 0 on this path
+    // Eq. 9 over a run of consecutive window positions i_a..i_b as a Horner chain H = sum c_i I_i decay^(i_b - i),
+    // c_0 = 1/alpha (the seed), c_i = 1: the run contributes alpha * decay^(w-1-i_b) * H.
+    constexpr int kRun = kW < 32 ? kW : 32;                  // columns of one run inside this warpgroup
+    const int i_first = (cgp * 32) % kW;
+    const float seed_coef = (i_first == 0) ? 1.f / alpha : 1.f;
+    const float fin_scale = alpha * powf(ema_decay, (float)(kW - 1 - (i_first + kRun - 1))) / (float)kG;
     const float* O_head = O_f32 + (long long)bh * kRows * kHeadDim;
     const __nv_bfloat16* V_head = V + (long long)b * vsb + (long long)h * vsh;
+    float* I_head = I_hat + (long long)bh * n;
+    bool ok = true;
 
-    for (int it = wg; it < T; it += 2) {
-      const int s = wg;
+    for (int it = 0; it < T; ++it) {
+      const int s = it & 1;
       const uint32_t par = (uint32_t)(it >> 1) & 1u;
-      if (!mbar_wait(&bar_kv_full[s], par, &abort_flag, dev_status, kDevTimeout)) break;
-      // ||v||^2 of this thread's token from the swizzled V tile: 16-byte chunk c of row r sits at chunk c ^ (r & 7)
-      float vn = 0.f;
-      {
-        const uint8_t* vt = gen_base + 2 * kTileBytes + (size_t)s * kStageBytes + kTileBytes;
-        const int r = t_in_tile;
+      ok = ok && mbar_wait(&bar_kv_full[s], par, &abort_flag, dev_status, kDevTimeout);
+      // ---- quarter of ||v||^2 of this thread's token from the swizzled V tile:
+      //      16-byte chunk c of row r sits at chunk c ^ (r & 7) of the row's 128 bytes ----
+      if (ok) {
+        const uint8_t* rowp = gen_kv + (size_t)s * kStageBytes + kTileBytes + (cgp >> 1) * kBoxBytes +
+                              (t >> 3) * 1024 + (t & 7) * 128;
+        float vp = 0.f;
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const uint8_t* rowp = vt + half * kBoxBytes + (r >> 3) * 1024 + (r & 7) * 128;
+        for (int c = 0; c < 4; ++c) {
+          const uint4 u = *reinterpret_cast<const uint4*>(rowp + ((((cgp & 1) * 4 + c) ^ (t & 7)) << 4));
+          const unsigned int wv[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            const uint4 u = *reinterpret_cast<const uint4*>(rowp + ((c ^ (r & 7)) << 4));
-            const unsigned int wv[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const float lo = __uint_as_float(wv[q] << 16), hi = __uint_as_float(wv[q] & 0xFFFF0000u);
-              vn = fmaf(lo, lo, vn);
-              vn = fmaf(hi, hi, vn);
-            }
+          for (int q = 0; q < 4; ++q) {
+            const float lo = __uint_as_float(wv[q] << 16), hi = __uint_as_float(wv[q] & 0xFFFF0000u);
+            vp = fmaf(lo, lo, vp);
+            vp = fmaf(hi, hi, vp);
           }
         }
+        vn_part[s][cgp][t] = vp;
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&bar_kv_empty[s]);
-      if (!mbar_wait(&bar_acc_full[s], par, &abort_flag, dev_status, kDevTimeout)) break;
-      tc_fence_after();
-
-      const int j = (tile0 + it) * kTile + t_in_tile;
-      const uint32_t tSt = tmem + (uint32_t)s * 256u + lane_base, tCt = tSt + 128u;
-      float hacc[kG];
-#pragma unroll
-      for (int g = 0; g < kG; ++g) hacc[g] = 0.f;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        float sv[32], cv[32];
-        __syncwarp();
-        tmem_ld32(tSt + c * 32, sv);
-        tmem_ld32(tCt + c * 32, cv);
-        tmem_wait_ld();
-#pragma unroll
-        for (int u = 0; u < 32; ++u) {
-          const int r = c * 32 + u;          // query row = g * kW + i
-          const int i = r % kW, g = r / kW;
-          const float2 k = cst[r];
-          const float A = ex2_approx(fmaf(sv[u], c2, -k.x));
-          float x = fmaf(-2.f, cv[u], k.y + vn);
-          if (A > 0.125f && j < n) x = exact_dist2(O_head + r * kHeadDim, V_head + (long long)j * vsn);
-          x = fmaxf(x, 0.f);
-          const float y = fmaxf(1.f - A, 5.9604645e-8f);
-          const float I = A * x * rsqrt_approx(fmaxf(x * y * y, 1e-36f));   // A / (1 - A) * sqrt(x)
-          if (i == 0) hacc[g] = I * k0;                                     // EMA seeded with the oldest query
-          else if (!alpha_zero) hacc[g] = fmaf(hacc[g], ema_decay, I);      // Horner form of Eq. 9
-        }
+      named_barrier_sync(1, kP2EpiThreads);
+      const float vn = (vn_part[s][0][t] + vn_part[s][1][t]) + (vn_part[s][2][t] + vn_part[s][3][t]);
+      if (it > 0 && cgp == 0) {   // the previous tile's shares are complete: sum them in a fixed order
+        const int jp = (tile0 + it - 1) * kTile + t;
+        if (jp < n) I_head[jp] = (red[s ^ 1][0][t] + red[s ^ 1][1][t]) + (red[s ^ 1][2][t] + red[s ^ 1][3][t]);
       }
-      tc_fence_before();
-      mbar_arrive(&bar_acc_empty[s]);
+      ok = ok && mbar_wait(&bar_acc_full[s], par, &abort_flag, dev_status, kDevTimeout);
       float tot = 0.f;
+      if (ok) {
+        tc_fence_after();
+        const int j = (tile0 + it) * kTile + t;
+        const uint32_t tS = tmem + (uint32_t)s * 256u + lane_base + (uint32_t)cgp * 32u, tC = tS + 128u;
+        float hacc = 0.f;
 #pragma unroll
-      for (int g = 0; g < kG; ++g) tot += hacc[g];
-      if (j < n) I_hat[(long long)bh * n + j] = tot * fin_scale;
+        for (int c = 0; c < 2; ++c) {
+          float sv[16], cv[16];
+          tmem_ld16(tS + c * 16, sv);
+          tmem_ld16(tC + c * 16, cv);
+          tmem_wait_ld();
+          const float hacc_in = hacc, tot_in = tot;
+          float smax = sv[0];
+#pragma unroll
+          for (int u = 1; u < 16; ++u) smax = fmaxf(smax, sv[u]);
+#pragma unroll
+          for (int u = 0; u < 16; ++u) {
+            const float uinv = ex2_approx(sv[u] * neg_c2);          // 1 / A
+            const float um = uinv - 1.f;
+            const float x = fmaxf(cv[u] + vn, 1e-30f);              // ||o - v||^2
+            const float bq = fmaxf(x * um * um, 1e-36f);
+            const float I = x * rsqrt_approx(bq);
+            const int col = c * 16 + u;
+            if (col % kRun == 0) {
+              if (col > 0) tot += hacc;
+              hacc = I * seed_coef;
+            } else {
+              hacc = fmaf(hacc, ema_decay, I);
+            }
+          }
+          if (smax > heavy_thr && j < n) {   // rare: redo the chunk with the exact distance where A is large
+            hacc = hacc_in;
+            tot = tot_in;
+#pragma unroll
+            for (int u = 0; u < 16; ++u) {
+              const int col = c * 16 + u;
+              const float uinv = ex2_approx(sv[u] * neg_c2);
+              const float um = uinv - 1.f;
+              float x = cv[u] + vn;
+              if (sv[u] > heavy_thr)
+                x = exact_dist2(O_head + (cgp * 32 + col) * kHeadDim, V_head + (long long)j * vsn);
+              x = fmaxf(x, 1e-30f);
+              const float bq = fmaxf(x * um * um, 1e-36f);
+              const float I = x * rsqrt_approx(bq);
+              if (col % kRun == 0) {
+                if (col > 0) tot += hacc;
+                hacc = I * seed_coef;
+              } else {
+                hacc = fmaf(hacc, ema_decay, I);
+              }
+            }
+          }
+        }
+        tot += hacc;
+        tc_fence_before();
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bar_acc_empty[s]);
+      red[s][cgp][t] = tot * fin_scale;
+    }
+    named_barrier_sync(1, kP2EpiThreads);
+    if (T > 0 && cgp == 0) {
+      const int sl = (T - 1) & 1;
+      const int jl = (tile0 + T - 1) * kTile + t;
+      if (jl < n) I_head[jl] = (red[sl][0][t] + red[sl][1][t]) + (red[sl][2][t] + red[sl][3][t]);
     }
   }
 
@@ -484,6 +550,12 @@ bool make_rows_map(TcState* st, CUtensorMap* map, const void* base, int BH) {   
   return encode_tiles(st, map, base, 3, dims, str) == CUDA_SUCCESS;
 }
 
+bool make_aug_map(TcState* st, CUtensorMap* map, const void* base, int BH) {   // [BH, 128, 64] contiguous
+  cuuint64_t dims[3] = {64, (cuuint64_t)kRows, (cuuint64_t)BH};
+  cuuint64_t str[2] = {64 * 2, (cuuint64_t)kRows * 64 * 2};
+  return encode_tiles(st, map, base, 3, dims, str) == CUDA_SUCCESS;
+}
+
 bool make_kv_map(TcState* st, CUtensorMap* map, const void* base, const Problem& p, long long sb, long long sh,
                  long long sn) {
   cuuint64_t dims[4] = {(cuuint64_t)p.d, (cuuint64_t)p.n_kv, (cuuint64_t)p.Hkv, (cuuint64_t)p.batch};
@@ -494,7 +566,7 @@ bool make_kv_map(TcState* st, CUtensorMap* map, const void* base, const Problem&
 }
 
 constexpr size_t kP1Smem = kTileBytes + 2 * kStageBytes + 1024;        // Q + two K/V stages + alignment slack
-constexpr size_t kP2Smem = 2 * kTileBytes + 2 * kStageBytes + 1024;    // Q + O + two K/V stages + slack
+constexpr size_t kP2Smem = 2 * kTileBytes + kAugBytes + kOnesBytes + 2 * kStageBytes + 1024;   // + alignment slack
 
 }  // namespace
 
@@ -540,16 +612,16 @@ cudaError_t launch_tc_pass1(void* state, const Problem& p, const Workspace& ws, 
 cudaError_t launch_tc_pass2(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
                             const void* V, float ema_decay, unsigned int* dev_status, cudaStream_t st) {
   TcState* ts = (TcState*)state;
-  CUtensorMap tmQ, tmO, tmK, tmV;
-  if (!make_rows_map(ts, &tmQ, Q, p.BH) || !make_rows_map(ts, &tmO, ws.O_bf16, p.BH) ||
-      !make_kv_map(ts, &tmK, K, p, p.ksb, p.ksh, p.ksn) || !make_kv_map(ts, &tmV, V, p, p.vsb, p.vsh, p.vsn))
+  CUtensorMap tmQ, tmO, tmAug, tmK, tmV;
+  if (!make_rows_map(ts, &tmQ, Q, p.BH) || !make_rows_map(ts, &tmO, ws.O_m2, p.BH) ||
+      !make_aug_map(ts, &tmAug, ws.aug, p.BH) || !make_kv_map(ts, &tmK, K, p, p.ksb, p.ksh, p.ksn) ||
+      !make_kv_map(ts, &tmV, V, p, p.vsb, p.vsh, p.vsn))
     return cudaErrorInvalidValue;
   dim3 grid(ws.splits, p.BH);
 #define RESTKV_P2(W)                                                                                              \
-  tc_pass2_kernel<W><<<grid, kP2Threads, kP2Smem, st>>>(tmQ, tmO, tmK, tmV, p.Hkv, p.n, p.scale, ema_decay,       \
-                                                        ws.splits, ws.fin_M2, ws.fin_on, ws.O_f32,                \
-                                                        (const __nv_bfloat16*)V, p.vsb, p.vsh, p.vsn, ws.I_hat,   \
-                                                        dev_status)
+  tc_pass2_kernel<W><<<grid, kP2Threads, kP2Smem, st>>>(tmQ, tmO, tmAug, tmK, tmV, p.Hkv, p.n, p.scale, ema_decay, \
+                                                        ws.splits, ws.O_f32, (const __nv_bfloat16*)V, p.vsb,      \
+                                                        p.vsh, p.vsn, ws.I_hat, dev_status)
   switch (p.w) {
     case 16: RESTKV_P2(16); break;
     case 32: RESTKV_P2(32); break;
