@@ -49,9 +49,11 @@ size_t plan_workspace(const Problem& p, int budget, int sm_count, bool adaptive,
   Workspace w{};
   w.splits = pass1_splits(p, sm_count);
   const size_t BH = (size_t)p.BH, R = (size_t)p.R, d = (size_t)p.d;
-  w.part_m = (float*)take(BH * w.splits * R * sizeof(float));
-  w.part_l = (float*)take(BH * w.splits * R * sizeof(float));
-  w.part_O = (float*)take(BH * w.splits * R * d * sizeof(float));
+  w.parts = w.splits;
+  w.part_m = (float*)take(BH * 2 * w.splits * R * sizeof(float));
+  w.part_l = (float*)take(BH * 2 * w.splits * R * sizeof(float));
+  w.part_O = (float*)take(BH * 2 * w.splits * R * d * sizeof(float));
+  w.vnorm = (float*)take(BH * (size_t)p.n_kv * sizeof(float));
   w.fin_m = (float*)take(BH * R * sizeof(float));
   w.fin_l = (float*)take(BH * R * sizeof(float));
   w.O_f32 = (float*)take(BH * R * d * sizeof(float));
@@ -170,11 +172,11 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
     if (e != cudaSuccess) return c.fail(e);
   } else if (use_tc) {
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS1, launch_tc_pass1(c.h->tc_state, p, ws, Q, K, V, c.h->dev_status, c.st), 1);
-    RESTKV_LAUNCH(c, RESTKV_KERNEL_COMBINE, launch_combine(p, ws, c.st), 1);
+    RESTKV_LAUNCH(c, RESTKV_KERNEL_COMBINE, launch_combine(p, ws, 2 * ws.splits, c.st), 1);   // two warpgroups per CTA
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2, launch_tc_pass2(c.h->tc_state, p, ws, Q, K, V, ema_decay, c.h->dev_status, c.st), 1);
   } else {
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS1, launch_simt_pass1(p, ws, Q, K, V, c.st), 1);
-    RESTKV_LAUNCH(c, RESTKV_KERNEL_COMBINE, launch_combine(p, ws, c.st), 1);
+    RESTKV_LAUNCH(c, RESTKV_KERNEL_COMBINE, launch_combine(p, ws, ws.splits, c.st), 1);
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2, launch_simt_pass2(p, ws, Q, K, V, ema_decay, adaptive ? ws.I_raw : nullptr, c.st), 1);
   }
   if (adaptive) {

@@ -28,10 +28,12 @@ struct Problem {
 
 // Workspace carve-up (all offsets 256-byte aligned).
 struct Workspace {
-  int splits;             // token splits of pass 1 per (batch, KV head)
-  float* part_m;          // [BH, splits, R]
-  float* part_l;          // [BH, splits, R]
-  float* part_O;          // [BH, splits, R, d]
+  int splits;             // token splits (CTAs) of the score passes per (batch, KV head)
+  int parts;              // partials per (batch, KV head) that pass 1 writes and combine merges
+  float* part_m;          // [BH, parts, R]   (room for 2 * splits)
+  float* part_l;          // [BH, parts, R]
+  float* part_O;          // [BH, parts, R, d]
+  float* vnorm;           // [BH, n_kv]  ||v_j||^2 (tensor-core path)
   float* fin_m;           // [BH, R]    row max of the scaled logits (natural units)
   float* fin_l;           // [BH, R]    sum of exp(s - m)
   float* O_f32;           // [BH, R, d]
@@ -57,7 +59,7 @@ size_t plan_workspace(const Problem& p, int budget, int sm_count, bool adaptive,
 // ---- launches (each returns the cudaError_t of the launch) -------------------------------------
 cudaError_t launch_simt_pass1(const Problem& p, const Workspace& ws, const void* Q, const void* K, const void* V,
                               cudaStream_t st);
-cudaError_t launch_combine(const Problem& p, const Workspace& ws, cudaStream_t st);
+cudaError_t launch_combine(const Problem& p, const Workspace& ws, int parts, cudaStream_t st);
 cudaError_t launch_simt_pass2(const Problem& p, const Workspace& ws, const void* Q, const void* K, const void* V,
                               float ema_decay, float* I_raw, cudaStream_t st);
 cudaError_t launch_pool(const Problem& p, const Workspace& ws, const int* pool_dev, int W, int gamma, float* scores,

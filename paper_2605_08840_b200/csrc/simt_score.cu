@@ -273,9 +273,9 @@ cudaError_t launch_simt_pass1(const Problem& p, const Workspace& ws, const void*
   return cudaGetLastError();
 }
 
-cudaError_t launch_combine(const Problem& p, const Workspace& ws, cudaStream_t st) {
+cudaError_t launch_combine(const Problem& p, const Workspace& ws, int parts, cudaStream_t st) {
   dim3 grid(p.R, p.BH);
-  combine_kernel<<<grid, 128, 0, st>>>(p.R, p.d, ws.splits, p.scale, ws.part_m, ws.part_l, ws.part_O, ws.fin_m,
+  combine_kernel<<<grid, 128, 0, st>>>(p.R, p.d, parts, p.scale, ws.part_m, ws.part_l, ws.part_O, ws.fin_m,
                                        ws.fin_l, ws.O_f32, ws.O_m2, ws.aug);
   return cudaGetLastError();
 }

@@ -60,21 +60,32 @@ __device__ __forceinline__ void mma_tile_kk(uint32_t tmem_d, uint32_t a_smem, ui
 // ================================================================================================
 // Pass 1
 // ================================================================================================
-constexpr int kP1Threads = 192;   // warp 0: TMA, warp 1: MMA, warps 2-5: softmax (one thread per query row)
+// Warp 0: TMA producer.  Warp 1: MMA issuer.  Warps 2-5 and 6-9: two softmax warpgroups (thread = query row);
+// warpgroup g owns the tiles it = g, g + 2, ... of the CTA with its own running (m, l) and its own output
+// accumulator, so the CTA writes two partials.  Tensor memory: S_g at g*128 (the bf16 P_g overwrites its first
+// 64 columns once the logits are in registers), O_g at 256 + g*128.  K and V travel in separate rings (2 and 3
+// slots of 32 KB): a K slot is free as soon as S = Q K^T has run, a V slot after O += P V.
+// The warpgroup that owns a tile also computes ||v_j||^2 of its 128 tokens from the V tile in shared memory
+// and stores them for pass 2.
+constexpr int kP1SoftWarps = 8;
+constexpr int kP1Threads = 64 + kP1SoftWarps * 32;
+constexpr int kP1KSlots = 2, kP1VSlots = 3;
 
 __global__ void __launch_bounds__(kP1Threads, 1)
 tc_pass1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, int Hkv, int n, int n_kv, int w, float scale, int splits,
                 float* __restrict__ part_m, float* __restrict__ part_l, float* __restrict__ part_O,
-                unsigned int* __restrict__ dev_status) {
+                float* __restrict__ vnorm, unsigned int* __restrict__ dev_status) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bar_q_full, bar_kv_full[2], bar_s_full[2], bar_p_full[2], bar_pv_done[2];
+  __shared__ __align__(8) uint64_t bar_q_full, bar_k_full[kP1KSlots], bar_k_empty[kP1KSlots], bar_v_full[kP1VSlots],
+      bar_v_empty[kP1VSlots], bar_s_full[2], bar_p_full[2], bar_pv_done[2];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sQ = smem_base;
-  const uint32_t sKV = smem_base + kTileBytes;   // stage s: K at sKV + s*kStageBytes, V right after it
+  const uint32_t sK = sQ + kTileBytes;                       // K slot i at sK + i*kTileBytes
+  const uint32_t sV = sK + kP1KSlots * kTileBytes;           // V slot i at sV + i*kTileBytes
   uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -89,8 +100,9 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   if (threadIdx.x == 0) {
     abort_flag = 0;
     mbar_init(&bar_q_full, 1);
+    for (int i = 0; i < kP1KSlots; ++i) { mbar_init(&bar_k_full[i], 1); mbar_init(&bar_k_empty[i], 1); }
+    for (int i = 0; i < kP1VSlots; ++i) { mbar_init(&bar_v_full[i], 1); mbar_init(&bar_v_empty[i], 1 + 4); }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&bar_kv_full[i], 1);
       mbar_init(&bar_s_full[i], 1);
       mbar_init(&bar_p_full[i], 128);
       mbar_init(&bar_pv_done[i], 1);
@@ -108,10 +120,6 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = tmem_slot;
-  // columns: S0 [0,128) S1 [128,256) O [256,384) P0 [384,448) P1 [448,512)
-  const uint32_t tO = tmem + 256;
-  auto tS = [tmem](int i) { return tmem + (uint32_t)i * 128u; };
-  auto tP = [tmem](int i) { return tmem + 384u + (uint32_t)i * 64u; };
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -120,141 +128,190 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       tma_load_3d(gen_base, &tmQ, &bar_q_full, 0, 0, bh);
       tma_load_3d(gen_base + kBoxBytes, &tmQ, &bar_q_full, 64, 0, bh);
       for (int it = 0; it < T; ++it) {
-        const int s = it & 1;
-        if (it >= 2 && !mbar_wait(&bar_pv_done[s], ((it >> 1) - 1) & 1, &abort_flag, dev_status, kDevTimeout)) break;
-        uint8_t* dK = gen_base + kTileBytes + (size_t)s * kStageBytes;
-        uint8_t* dV = dK + kTileBytes;
+        const int ks = it % kP1KSlots, vs = it % kP1VSlots;
         const int j0 = (tile0 + it) * kTile;
-        mbar_arrive_expect_tx(&bar_kv_full[s], kStageBytes);
-        tma_load_4d(dK, &tmK, &bar_kv_full[s], 0, j0, h, b);
-        tma_load_4d(dK + kBoxBytes, &tmK, &bar_kv_full[s], 64, j0, h, b);
-        tma_load_4d(dV, &tmV, &bar_kv_full[s], 0, j0, h, b);
-        tma_load_4d(dV + kBoxBytes, &tmV, &bar_kv_full[s], 64, j0, h, b);
+        if (it >= kP1KSlots &&
+            !mbar_wait(&bar_k_empty[ks], (it / kP1KSlots - 1) & 1, &abort_flag, dev_status, kDevTimeout))
+          break;
+        uint8_t* dK = gen_base + kTileBytes + (size_t)ks * kTileBytes;
+        mbar_arrive_expect_tx(&bar_k_full[ks], kTileBytes);
+        tma_load_4d(dK, &tmK, &bar_k_full[ks], 0, j0, h, b);
+        tma_load_4d(dK + kBoxBytes, &tmK, &bar_k_full[ks], 64, j0, h, b);
+        if (it >= kP1VSlots &&
+            !mbar_wait(&bar_v_empty[vs], (it / kP1VSlots - 1) & 1, &abort_flag, dev_status, kDevTimeout))
+          break;
+        uint8_t* dV = gen_base + (1 + kP1KSlots) * kTileBytes + (size_t)vs * kTileBytes;
+        mbar_arrive_expect_tx(&bar_v_full[vs], kTileBytes);
+        tma_load_4d(dV, &tmV, &bar_v_full[vs], 0, j0, h, b);
+        tma_load_4d(dV + kBoxBytes, &tmV, &bar_v_full[vs], 64, j0, h, b);
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
+    // ---------------- MMA issuer: S(it), then O += P V of tile it - 1 ----------------
     if (lane == 0 && T > 0) {
-      bool ok = mbar_wait(&bar_q_full, 0, &abort_flag, dev_status, kDevTimeout) &&
-                mbar_wait(&bar_kv_full[0], 0, &abort_flag, dev_status, kDevTimeout);
-      if (ok) {
-        tc_fence_after();
-        mma_tile_kk(tS(0), sQ, sKV, false);
-        umma_commit(&bar_s_full[0]);
-      }
-      for (int it = 0; ok && it < T; ++it) {
-        const int bsel = it & 1;
-        if (it + 1 < T) {
-          const int nb = (it + 1) & 1;
-          if (!mbar_wait(&bar_kv_full[nb], ((it + 1) >> 1) & 1, &abort_flag, dev_status, kDevTimeout)) break;
+      bool ok = mbar_wait(&bar_q_full, 0, &abort_flag, dev_status, kDevTimeout);
+      for (int it = 0; ok && it <= T; ++it) {
+        if (it < T) {
+          const int ks = it % kP1KSlots, g = it & 1;
+          if (!mbar_wait(&bar_k_full[ks], (it / kP1KSlots) & 1, &abort_flag, dev_status, kDevTimeout)) break;
           tc_fence_after();
-          mma_tile_kk(tS(nb), sQ, sKV + (uint32_t)nb * kStageBytes, false);   // S(it+1) = Q K^T
-          umma_commit(&bar_s_full[nb]);
+          // S_g may be overwritten: O += P V of tile it - 2 (which read P_g) was issued earlier and MMAs run in order
+          mma_tile_kk(tmem + (uint32_t)g * 128u, sQ, sK + (uint32_t)ks * kTileBytes, false);
+          umma_commit(&bar_s_full[g]);
+          umma_commit(&bar_k_empty[ks]);
         }
-        if (!mbar_wait(&bar_p_full[bsel], (it >> 1) & 1, &abort_flag, dev_status, kDevTimeout)) break;
-        tc_fence_after();
-        // O += P(it) V(it): A = P in TMEM (16 tokens = 8 packed columns per step), B = V tile, MN-major
-        const uint32_t sV = sKV + (uint32_t)bsel * kStageBytes + kTileBytes;
+        if (it >= 1) {
+          const int pt = it - 1, g = pt & 1, vs = pt % kP1VSlots;
+          if (!mbar_wait(&bar_p_full[g], (pt >> 1) & 1, &abort_flag, dev_status, kDevTimeout)) break;
+          if (!mbar_wait(&bar_v_full[vs], (pt / kP1VSlots) & 1, &abort_flag, dev_status, kDevTimeout)) break;
+          tc_fence_after();
+          // A = P_g in TMEM (16 tokens = 8 packed columns per K step), B = V tile, MN-major
+          const uint32_t vaddr = sV + (uint32_t)vs * kTileBytes;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const uint64_t bdesc = make_smem_desc(sV + (uint32_t)k * 2048u, kBoxBytes, 1024);
-          umma_ts(tO, tP(bsel) + (uint32_t)k * 8u, bdesc, kIdescKMN, it > 0 || k > 0);
+          for (int k = 0; k < 8; ++k) {
+            const uint64_t bdesc = make_smem_desc(vaddr + (uint32_t)k * 2048u, kBoxBytes, 1024);
+            umma_ts(tmem + 256u + (uint32_t)g * 128u, tmem + (uint32_t)g * 128u + (uint32_t)k * 8u, bdesc, kIdescKMN,
+                    pt >= 2 || k > 0);
+          }
+          umma_commit(&bar_pv_done[g]);
+          umma_commit(&bar_v_empty[vs]);
         }
-        umma_commit(&bar_pv_done[bsel]);
       }
     }
   } else {
-    // ---------------- softmax warps: thread = query row ----------------
+    // ---------------- softmax warpgroups: thread = query row ----------------
+    const int g = (warp - 2) >> 2;
     const int quad = warp & 3;
     const int row = quad * 32 + lane;
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-    const int i_q = row % w;                  // window position of this row (row = g*w + i)
+    const uint32_t tS = tmem + (uint32_t)g * 128u + lane_base, tO = tmem + 256u + (uint32_t)g * 128u + lane_base;
+    const int i_q = row % w;                  // window position of this row (row = group * w + i)
     const float c2 = scale * kLog2e;
-    float m_ref = -INFINITY, l = 0.f;
+    float m_ref = -INFINITY;
+    float2 l2 = make_float2(0.f, 0.f);
     bool ok = true;
-    for (int it = 0; it < T; ++it) {
-      const int bsel = it & 1;
-      if (!mbar_wait(&bar_s_full[bsel], (it >> 1) & 1, &abort_flag, dev_status, kDevTimeout)) { ok = false; break; }
+    int uses = 0;                             // tiles this warpgroup has processed
+    for (int it = g; it < T; it += 2, ++uses) {
+      const uint32_t par = (uint32_t)uses & 1u;
+      ok = ok && mbar_wait(&bar_s_full[g], par, &abort_flag, dev_status, kDevTimeout);
+      if (!ok) break;
       tc_fence_after();
-      float s[128];
-#pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld32(tS(bsel) + lane_base + c * 32, s + c * 32);
-      tmem_wait_ld();
       const int j0 = (tile0 + it) * kTile;
-      if (j0 + kTile > n) {   // tile touches rows past the scored prefix: window rows (causal) or padding
+      const bool ragged = j0 + kTile > n;   // rows past the scored prefix: window rows (causal) or padding
+      // ---- sweep 1: row maximum of the tile ----
+      float tmax = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < 128; ++c) {
-          const int j = j0 + c;
-          const bool vis = (j < n_kv) && (j < n || (j - n) <= i_q);
-          s[c] = vis ? s[c] : -INFINITY;
+      for (int c = 0; c < 4; ++c) {
+        float s[32];
+        tmem_ld32(tS + c * 32, s);
+        tmem_wait_ld();
+        if (ragged) {
+#pragma unroll
+          for (int u = 0; u < 32; ++u) {
+            const int j = j0 + c * 32 + u;
+            const bool vis = (j < n_kv) && (j < n || (j - n) <= i_q);
+            s[u] = vis ? s[u] : -INFINITY;
+          }
         }
-      }
-      float tmax = s[0];
 #pragma unroll
-      for (int c = 1; c < 128; ++c) tmax = fmaxf(tmax, s[c]);
+        for (int u = 0; u < 32; ++u) tmax = fmaxf(tmax, s[u]);
+      }
       const float m_tile = tmax * c2;
       const bool need = m_tile > m_ref + kRescaleThreshold;   // also true for the first visible entries (m_ref = -inf)
       float factor = 1.f;
       if (need) {
         factor = ex2_approx(m_ref - m_tile);   // 0 when m_ref = -inf
-        l *= factor;
+        l2.x *= factor;
+        l2.y *= factor;
         m_ref = m_tile;
       }
-      if (it > 0 && __any_sync(0xffffffffu, need)) {
-        // rescale the running output: needs O += P V of the previous tile to have landed
-        if (!mbar_wait(&bar_pv_done[(it - 1) & 1], ((it - 1) >> 1) & 1, &abort_flag, dev_status, kDevTimeout)) {
-          ok = false;
-          break;
-        }
-        tc_fence_after();
+      // S(it) has landed, so O += P V of this warpgroup's previous tile (issued before it) is complete
+      if (uses > 0 && __any_sync(0xffffffffu, need)) {
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           float o[32];
-          tmem_ld32(tO + lane_base + c * 32, o);
+          tmem_ld32(tO + c * 32, o);
           tmem_wait_ld();
 #pragma unroll
           for (int u = 0; u < 32; ++u) o[u] *= factor;
-          tmem_st32(tO + lane_base + c * 32, o);
+          tmem_st32(tO + c * 32, o);
         }
       }
-      if (it >= 2 && !mbar_wait(&bar_pv_done[bsel], ((it >> 1) - 1) & 1, &abort_flag, dev_status, kDevTimeout)) {
-        ok = false;
-        break;
-      }
+      // ---- sweep 2: P = exp2(s*c2 - m_ref) as bf16 over the first 64 columns of S_g.  Chunk c of P lands on
+      //      columns [16c, 16c + 16), which belong to a chunk of S that is already in registers. ----
       const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+      const float2 c22 = make_float2(c2, c2), nm2 = make_float2(-m_use, -m_use);
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
+        float s[32];
+        tmem_ld32(tS + c * 32, s);
+        tmem_wait_ld();
+        if (ragged) {
+#pragma unroll
+          for (int u = 0; u < 32; ++u) {
+            const int j = j0 + c * 32 + u;
+            const bool vis = (j < n_kv) && (j < n || (j - n) <= i_q);
+            s[u] = vis ? s[u] : -INFINITY;
+          }
+        }
         uint32_t packed[16];
 #pragma unroll
         for (int u = 0; u < 16; ++u) {
-          const float p0 = ex2_approx(fmaf(s[c * 32 + 2 * u], c2, -m_use));
-          const float p1 = ex2_approx(fmaf(s[c * 32 + 2 * u + 1], c2, -m_use));
-          l += p0 + p1;
-          packed[u] = pack_bf16x2(p0, p1);
+          const float2 a = ffma2(make_float2(s[2 * u], s[2 * u + 1]), c22, nm2);
+          const float2 pp = make_float2(ex2_approx(a.x), ex2_approx(a.y));
+          l2 = fadd2(l2, pp);
+          packed[u] = pack_bf16x2(pp.x, pp.y);
         }
-        tmem_st16(tP(bsel) + lane_base + c * 16, packed);
+        tmem_st16(tS + c * 16, packed);
       }
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(&bar_p_full[bsel]);
+      mbar_arrive(&bar_p_full[g]);
+
+      // ---- ||v||^2 of token j0 + row from the swizzled V tile (chunk c of row r sits at chunk c ^ (r & 7)) ----
+      const int vs = it % kP1VSlots;
+      ok = ok && mbar_wait(&bar_v_full[vs], (it / kP1VSlots) & 1, &abort_flag, dev_status, kDevTimeout);
+      if (!ok) break;
+      {
+        const uint8_t* vt = gen_base + (1 + kP1KSlots) * kTileBytes + (size_t)vs * kTileBytes;
+        float2 acc = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const uint8_t* rowp = vt + half * kBoxBytes + (row >> 3) * 1024 + (row & 7) * 128;
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            const uint4 u = *reinterpret_cast<const uint4*>(rowp + ((c ^ (row & 7)) << 4));
+            const unsigned int wv[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const float2 e = make_float2(__uint_as_float(wv[q] << 16), __uint_as_float(wv[q] & 0xFFFF0000u));
+              acc = ffma2(e, e, acc);
+            }
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bar_v_empty[vs]);
+        const int j = j0 + row;
+        if (j < n_kv) vnorm[(long long)bh * n_kv + j] = acc.x + acc.y;
+      }
     }
-    // ---- write the partial (m, l, O) of this split ----
-    const long long o_idx = ((long long)bh * splits + split) * kRows + row;
+    // ---- write this warpgroup's partial (m, l, O) ----
+    const long long o_idx = (((long long)bh * splits + split) * 2 + g) * kRows + row;
     float* Op = part_O + o_idx * kHeadDim;
-    if (T > 0 && ok) ok = mbar_wait(&bar_pv_done[(T - 1) & 1], ((T - 1) >> 1) & 1, &abort_flag, dev_status, kDevTimeout);
-    if (T > 0 && ok) {
+    if (uses > 0 && ok) ok = mbar_wait(&bar_pv_done[g], (uint32_t)(uses - 1) & 1u, &abort_flag, dev_status, kDevTimeout);
+    if (uses > 0 && ok) {
       tc_fence_after();
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         float o[32];
-        tmem_ld32(tO + lane_base + c * 32, o);
+        tmem_ld32(tO + c * 32, o);
         tmem_wait_ld();
 #pragma unroll
         for (int u = 0; u < 32; u += 4)
           *reinterpret_cast<float4*>(Op + c * 32 + u) = make_float4(o[u], o[u + 1], o[u + 2], o[u + 3]);
       }
       part_m[o_idx] = (m_ref == -INFINITY) ? -INFINITY : m_ref * kLn2;   // natural-log units
-      part_l[o_idx] = l;
+      part_l[o_idx] = l2.x + l2.y;
     } else {
       for (int u = 0; u < kHeadDim; u += 4) *reinterpret_cast<float4*>(Op + u) = make_float4(0.f, 0.f, 0.f, 0.f);
       part_m[o_idx] = -INFINITY;
@@ -312,13 +369,13 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 const __grid_constant__ CUtensorMap tmAug, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, int Hkv, int n, float scale, float ema_decay, int splits,
                 const float* __restrict__ O_f32, const __nv_bfloat16* __restrict__ V, long long vsb, long long vsh,
-                long long vsn, float* __restrict__ I_hat, unsigned int* __restrict__ dev_status) {
+                long long vsn, const float* __restrict__ vnorm, int n_kv, float* __restrict__ I_hat,
+                unsigned int* __restrict__ dev_status) {
   constexpr int kG = kRows / kW;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_const_full, bar_kv_full[2], bar_kv_empty[2], bar_acc_full[2], bar_acc_empty[2];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
-  __shared__ float vn_part[2][4][kTile];   // ||v||^2 of each token, one quarter of the row per warpgroup
   __shared__ float red[2][4][kTile];       // per-warpgroup share of the token's score
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -341,7 +398,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     mbar_init(&bar_const_full, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&bar_kv_full[i], 1);
-      mbar_init(&bar_kv_empty[i], 1 + kP2EpiWarps);   // MMA commit + one arrival per epilogue warp
+      mbar_init(&bar_kv_empty[i], 1);                 // MMA commit
       mbar_init(&bar_acc_full[i], 1);
       mbar_init(&bar_acc_empty[i], kP2EpiWarps);
     }
@@ -415,44 +472,35 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const float heavy_thr = log2f(1.f / kHeavyA) / neg_c2;   // S' above this <=> A > kHeavyA
     const float alpha = 1.f - ema_decay;                     // > 0 on this path
     // Eq. 9 over a run of consecutive window positions i_a..i_b as a Horner chain H = sum c_i I_i decay^(i_b - i),
-    // c_0 = 1/alpha (the seed), c_i = 1: the run contributes alpha * decay^(w-1-i_b) * H.
+    // c_0 = 1/alpha (the seed), c_i = 1: the run contributes alpha * decay^(w-1-i_b) * H.  Even and odd columns
+    // of a run are chained separately in decay^2 (one packed FMA per column pair): H = decay * H_even + H_odd.
     constexpr int kRun = kW < 32 ? kW : 32;                  // columns of one run inside this warpgroup
     const int i_first = (cgp * 32) % kW;
     const float seed_coef = (i_first == 0) ? 1.f / alpha : 1.f;
     const float fin_scale = alpha * powf(ema_decay, (float)(kW - 1 - (i_first + kRun - 1))) / (float)kG;
+    const float2 d2 = make_float2(ema_decay * ema_decay, ema_decay * ema_decay);
+    const float2 nc2 = make_float2(neg_c2, neg_c2), m1 = make_float2(-1.f, -1.f);
     const float* O_head = O_f32 + (long long)bh * kRows * kHeadDim;
     const __nv_bfloat16* V_head = V + (long long)b * vsb + (long long)h * vsh;
+    const float* vn_head = vnorm + (long long)bh * n_kv;
     float* I_head = I_hat + (long long)bh * n;
     bool ok = true;
+    float vn_next = 0.f;
+    if (T > 0) {
+      const int j = tile0 * kTile + t;
+      vn_next = (j < n) ? vn_head[j] : 1.f;
+    }
 
     for (int it = 0; it < T; ++it) {
       const int s = it & 1;
       const uint32_t par = (uint32_t)(it >> 1) & 1u;
-      ok = ok && mbar_wait(&bar_kv_full[s], par, &abort_flag, dev_status, kDevTimeout);
-      // ---- quarter of ||v||^2 of this thread's token from the swizzled V tile:
-      //      16-byte chunk c of row r sits at chunk c ^ (r & 7) of the row's 128 bytes ----
-      if (ok) {
-        const uint8_t* rowp = gen_kv + (size_t)s * kStageBytes + kTileBytes + (cgp >> 1) * kBoxBytes +
-                              (t >> 3) * 1024 + (t & 7) * 128;
-        float vp = 0.f;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const uint4 u = *reinterpret_cast<const uint4*>(rowp + ((((cgp & 1) * 4 + c) ^ (t & 7)) << 4));
-          const unsigned int wv[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const float lo = __uint_as_float(wv[q] << 16), hi = __uint_as_float(wv[q] & 0xFFFF0000u);
-            vp = fmaf(lo, lo, vp);
-            vp = fmaf(hi, hi, vp);
-          }
-        }
-        vn_part[s][cgp][t] = vp;
+      const float vn = vn_next;
+      if (it + 1 < T) {   // next tile's ||v||^2, well ahead of its use
+        const int jn = (tile0 + it + 1) * kTile + t;
+        vn_next = (jn < n) ? vn_head[jn] : 1.f;
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&bar_kv_empty[s]);
-      named_barrier_sync(1, kP2EpiThreads);
-      const float vn = (vn_part[s][0][t] + vn_part[s][1][t]) + (vn_part[s][2][t] + vn_part[s][3][t]);
-      if (it > 0 && cgp == 0) {   // the previous tile's shares are complete: sum them in a fixed order
+      if (it > 0) named_barrier_sync(1, kP2EpiThreads);   // every warpgroup has stored its share of the previous tile
+      if (it > 0 && cgp == 0) {                           // sum the shares in a fixed order
         const int jp = (tile0 + it - 1) * kTile + t;
         if (jp < n) I_head[jp] = (red[s ^ 1][0][t] + red[s ^ 1][1][t]) + (red[s ^ 1][2][t] + red[s ^ 1][3][t]);
       }
@@ -462,56 +510,49 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         tc_fence_after();
         const int j = (tile0 + it) * kTile + t;
         const uint32_t tS = tmem + (uint32_t)s * 256u + lane_base + (uint32_t)cgp * 32u, tC = tS + 128u;
-        float hacc = 0.f;
+        const float2 vn2 = make_float2(vn, vn);
+        float2 h2 = make_float2(0.f, 0.f);
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
-          float sv[16], cv[16];
+          float sv[16], cv[16], I[16];
           tmem_ld16(tS + c * 16, sv);
           tmem_ld16(tC + c * 16, cv);
           tmem_wait_ld();
-          const float hacc_in = hacc, tot_in = tot;
           float smax = sv[0];
 #pragma unroll
           for (int u = 1; u < 16; ++u) smax = fmaxf(smax, sv[u]);
 #pragma unroll
-          for (int u = 0; u < 16; ++u) {
-            const float uinv = ex2_approx(sv[u] * neg_c2);          // 1 / A
-            const float um = uinv - 1.f;
-            const float x = fmaxf(cv[u] + vn, 1e-30f);              // ||o - v||^2
-            const float bq = fmaxf(x * um * um, 1e-36f);
-            const float I = x * rsqrt_approx(bq);
-            const int col = c * 16 + u;
-            if (col % kRun == 0) {
-              if (col > 0) tot += hacc;
-              hacc = I * seed_coef;
-            } else {
-              hacc = fmaf(hacc, ema_decay, I);
-            }
+          for (int u = 0; u < 16; u += 2) {
+            const float2 nt = fmul2(make_float2(sv[u], sv[u + 1]), nc2);
+            const float2 um = fadd2(make_float2(ex2_approx(nt.x), ex2_approx(nt.y)), m1);   // 1/A - 1
+            float2 x = fadd2(make_float2(cv[u], cv[u + 1]), vn2);                          // ||o - v||^2
+            x.x = fmaxf(x.x, 1e-30f);
+            x.y = fmaxf(x.y, 1e-30f);
+            const float2 bq = fmul2(fmul2(x, um), um);
+            const float2 r = make_float2(rsqrt_approx(fmaxf(bq.x, 1e-36f)), rsqrt_approx(fmaxf(bq.y, 1e-36f)));
+            const float2 Iu = fmul2(x, r);
+            I[u] = Iu.x;
+            I[u + 1] = Iu.y;
           }
-          if (smax > heavy_thr && j < n) {   // rare: redo the chunk with the exact distance where A is large
-            hacc = hacc_in;
-            tot = tot_in;
+          if (smax > heavy_thr && j < n) {   // rare: exact distance where the attention weight is large
 #pragma unroll
             for (int u = 0; u < 16; ++u) {
-              const int col = c * 16 + u;
-              const float uinv = ex2_approx(sv[u] * neg_c2);
-              const float um = uinv - 1.f;
-              float x = cv[u] + vn;
-              if (sv[u] > heavy_thr)
-                x = exact_dist2(O_head + (cgp * 32 + col) * kHeadDim, V_head + (long long)j * vsn);
-              x = fmaxf(x, 1e-30f);
-              const float bq = fmaxf(x * um * um, 1e-36f);
-              const float I = x * rsqrt_approx(bq);
-              if (col % kRun == 0) {
-                if (col > 0) tot += hacc;
-                hacc = I * seed_coef;
-              } else {
-                hacc = fmaf(hacc, ema_decay, I);
+              if (sv[u] > heavy_thr) {
+                const float um = ex2_approx(sv[u] * neg_c2) - 1.f;
+                const float x = fmaxf(
+                    exact_dist2(O_head + (cgp * 32 + c * 16 + u) * kHeadDim, V_head + (long long)j * vsn), 1e-30f);
+                I[u] = x * rsqrt_approx(fmaxf(x * um * um, 1e-36f));
               }
             }
           }
+          if ((c * 16) % kRun == 0) I[0] *= seed_coef;
+#pragma unroll
+          for (int u = 0; u < 16; u += 2) h2 = ffma2(h2, d2, make_float2(I[u], I[u + 1]));
+          if ((c * 16 + 16) % kRun == 0) {   // end of a run
+            tot += fmaf(h2.x, ema_decay, h2.y);
+            h2 = make_float2(0.f, 0.f);
+          }
         }
-        tot += hacc;
         tc_fence_before();
       }
       __syncwarp();
@@ -565,7 +606,7 @@ bool make_kv_map(TcState* st, CUtensorMap* map, const void* base, const Problem&
   return encode_tiles(st, map, base, 4, dims, str) == CUDA_SUCCESS;
 }
 
-constexpr size_t kP1Smem = kTileBytes + 2 * kStageBytes + 1024;        // Q + two K/V stages + alignment slack
+constexpr size_t kP1Smem = (1 + kP1KSlots + kP1VSlots) * kTileBytes + 1024;   // Q + K ring + V ring + slack
 constexpr size_t kP2Smem = 2 * kTileBytes + kAugBytes + kOnesBytes + 2 * kStageBytes + 1024;   // + alignment slack
 
 }  // namespace
@@ -605,7 +646,7 @@ cudaError_t launch_tc_pass1(void* state, const Problem& p, const Workspace& ws, 
     return cudaErrorInvalidValue;
   dim3 grid(ws.splits, p.BH);
   tc_pass1_kernel<<<grid, kP1Threads, kP1Smem, st>>>(tmQ, tmK, tmV, p.Hkv, p.n, p.n_kv, p.w, p.scale, ws.splits,
-                                                     ws.part_m, ws.part_l, ws.part_O, dev_status);
+                                                     ws.part_m, ws.part_l, ws.part_O, ws.vnorm, dev_status);
   return cudaGetLastError();
 }
 
@@ -621,7 +662,7 @@ cudaError_t launch_tc_pass2(void* state, const Problem& p, const Workspace& ws, 
 #define RESTKV_P2(W)                                                                                              \
   tc_pass2_kernel<W><<<grid, kP2Threads, kP2Smem, st>>>(tmQ, tmO, tmAug, tmK, tmV, p.Hkv, p.n, p.scale, ema_decay, \
                                                         ws.splits, ws.O_f32, (const __nv_bfloat16*)V, p.vsb,      \
-                                                        p.vsh, p.vsn, ws.I_hat, dev_status)
+                                                        p.vsh, p.vsn, ws.vnorm, p.n_kv, ws.I_hat, dev_status)
   switch (p.w) {
     case 16: RESTKV_P2(16); break;
     case 32: RESTKV_P2(32); break;
