@@ -63,13 +63,13 @@ __device__ __forceinline__ void mma_tile_kk(uint32_t tmem_d, uint32_t a_smem, ui
 // Warp 0: TMA producer.  Warp 1: MMA issuer.  Warps 2-5 and 6-9: two softmax warpgroups (thread = query row);
 // warpgroup g owns the tiles it = g, g + 2, ... of the CTA with its own running (m, l) and its own output
 // accumulator, so the CTA writes two partials.  Tensor memory: S_g at g*128 (the bf16 P_g overwrites its first
-// 64 columns once the logits are in registers), O_g at 256 + g*128.  K and V travel in separate rings (2 and 3
-// slots of 32 KB): a K slot is free as soon as S = Q K^T has run, a V slot after O += P V.
+// 64 columns once the logits are in registers), O_g at 256 + g*128.  K and V travel in separate rings (3 slots
+// of 32 KB each): a K slot is free as soon as S = Q K^T has run, a V slot after O += P V.
 // The warpgroup that owns a tile also computes ||v_j||^2 of its 128 tokens from the V tile in shared memory
 // and stores them for pass 2.
 constexpr int kP1SoftWarps = 8;
 constexpr int kP1Threads = 64 + kP1SoftWarps * 32;
-constexpr int kP1KSlots = 2, kP1VSlots = 3;
+constexpr int kP1KSlots = 3, kP1VSlots = 3;
 
 __global__ void __launch_bounds__(kP1Threads, 1)
 tc_pass1_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -345,10 +345,6 @@ constexpr uint32_t kAugBytes = kBoxBytes;     // [128 rows x 64 bf16], only K st
 constexpr uint32_t kOnesBytes = 1024;         // one 8-row group of ones, shared by all 16 groups (stride 0)
 constexpr float kHeavyA = 0.125f;             // attention weight above which ||o - v||^2 is recomputed exactly
 
-__device__ __forceinline__ void named_barrier_sync(int id, int count) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
-}
-
 // Exact ||o - v||^2 for the rare entries whose attention weight is large (the expansion
 // ||o||^2 + ||v||^2 - 2 o.v cancels when o approaches v).
 __device__ __noinline__ float exact_dist2(const float* __restrict__ o_row, const __nv_bfloat16* __restrict__ v_row) {
@@ -373,10 +369,11 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 unsigned int* __restrict__ dev_status) {
   constexpr int kG = kRows / kW;
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bar_const_full, bar_kv_full[2], bar_kv_empty[2], bar_acc_full[2], bar_acc_empty[2];
+  __shared__ __align__(8) uint64_t bar_const_full, bar_kv_full[2], bar_kv_empty[2], bar_acc_full[2], bar_acc_empty[2],
+      bar_red_full[4];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
-  __shared__ float red[2][4][kTile];       // per-warpgroup share of the token's score
+  __shared__ float red[4][4][kTile];       // [tile & 3][warpgroup][token]: each warpgroup's share of the score
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sQ = smem_base, sO = sQ + kTileBytes, sAug = sO + kTileBytes, sOnes = sAug + kAugBytes;
@@ -402,6 +399,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       mbar_init(&bar_acc_full[i], 1);
       mbar_init(&bar_acc_empty[i], kP2EpiWarps);
     }
+    for (int i = 0; i < 4; ++i) mbar_init(&bar_red_full[i], kP2EpiWarps);
     fence_mbar_init();
     prefetch_tensormap(&tmQ);
     prefetch_tensormap(&tmO);
@@ -478,8 +476,8 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const int i_first = (cgp * 32) % kW;
     const float seed_coef = (i_first == 0) ? 1.f / alpha : 1.f;
     const float fin_scale = alpha * powf(ema_decay, (float)(kW - 1 - (i_first + kRun - 1))) / (float)kG;
-    const float2 d2 = make_float2(ema_decay * ema_decay, ema_decay * ema_decay);
-    const float2 nc2 = make_float2(neg_c2, neg_c2), m1 = make_float2(-1.f, -1.f);
+    const f32x2 d2 = f2_make(ema_decay * ema_decay, ema_decay * ema_decay);
+    const f32x2 nc2 = f2_make(neg_c2, neg_c2), m1 = f2_make(-1.f, -1.f), tiny2 = f2_make(1e-36f, 1e-36f);
     const float* O_head = O_f32 + (long long)bh * kRows * kHeadDim;
     const __nv_bfloat16* V_head = V + (long long)b * vsb + (long long)h * vsh;
     const float* vn_head = vnorm + (long long)bh * n_kv;
@@ -499,10 +497,14 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const int jn = (tile0 + it + 1) * kTile + t;
         vn_next = (jn < n) ? vn_head[jn] : 1.f;
       }
-      if (it > 0) named_barrier_sync(1, kP2EpiThreads);   // every warpgroup has stored its share of the previous tile
-      if (it > 0 && cgp == 0) {                           // sum the shares in a fixed order
+      // The shares of the previous tile are summed in a fixed order by warpgroup 0 once all sixteen warps have
+      // stored theirs.  A slot of `red` is rewritten four tiles later, which the two accumulator buffers only
+      // allow after every warp has moved past this point.
+      if (it > 0 && cgp == 0) {
+        const int rs = (it - 1) & 3;
+        ok = ok && mbar_wait(&bar_red_full[rs], (uint32_t)((it - 1) >> 2) & 1u, &abort_flag, dev_status, kDevTimeout);
         const int jp = (tile0 + it - 1) * kTile + t;
-        if (jp < n) I_head[jp] = (red[s ^ 1][0][t] + red[s ^ 1][1][t]) + (red[s ^ 1][2][t] + red[s ^ 1][3][t]);
+        if (ok && jp < n) I_head[jp] = (red[rs][0][t] + red[rs][1][t]) + (red[rs][2][t] + red[rs][3][t]);
       }
       ok = ok && mbar_wait(&bar_acc_full[s], par, &abort_flag, dev_status, kDevTimeout);
       float tot = 0.f;
@@ -510,11 +512,15 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         tc_fence_after();
         const int j = (tile0 + it) * kTile + t;
         const uint32_t tS = tmem + (uint32_t)s * 256u + lane_base + (uint32_t)cgp * 32u, tC = tS + 128u;
-        const float2 vn2 = make_float2(vn, vn);
-        float2 h2 = make_float2(0.f, 0.f);
+        // ||o - v||^2 = C' + ||v||^2 is formed with ||v||^2 raised by 2^-16 of itself: a bias of ~1e-5 that keeps
+        // the sum positive when the expansion cancels, so that no clamp is needed.
+        const float vnb = vn * 1.0000152587890625f;
+        const f32x2 vn2 = f2_make(vnb, vnb);
+        f32x2 h2 = f2_make(0.f, 0.f);
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
-          float sv[16], cv[16], I[16];
+          float sv[16], cv[16];
+          float I[16];
           tmem_ld16(tS + c * 16, sv);
           tmem_ld16(tC + c * 16, cv);
           tmem_wait_ld();
@@ -522,48 +528,47 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
           for (int u = 1; u < 16; ++u) smax = fmaxf(smax, sv[u]);
 #pragma unroll
-          for (int u = 0; u < 16; u += 2) {
-            const float2 nt = fmul2(make_float2(sv[u], sv[u + 1]), nc2);
-            const float2 um = fadd2(make_float2(ex2_approx(nt.x), ex2_approx(nt.y)), m1);   // 1/A - 1
-            float2 x = fadd2(make_float2(cv[u], cv[u + 1]), vn2);                          // ||o - v||^2
-            x.x = fmaxf(x.x, 1e-30f);
-            x.y = fmaxf(x.y, 1e-30f);
-            const float2 bq = fmul2(fmul2(x, um), um);
-            const float2 r = make_float2(rsqrt_approx(fmaxf(bq.x, 1e-36f)), rsqrt_approx(fmaxf(bq.y, 1e-36f)));
-            const float2 Iu = fmul2(x, r);
-            I[u] = Iu.x;
-            I[u + 1] = Iu.y;
+          for (int q = 0; q < 8; ++q) {
+            const f32x2 nt = f2_mul(f2_make(sv[2 * q], sv[2 * q + 1]), nc2);
+            const f32x2 um = f2_add(f2_make(ex2_approx(f2_lo(nt)), ex2_approx(f2_hi(nt))), m1);   // 1/A - 1
+            const f32x2 x = f2_add(f2_make(cv[2 * q], cv[2 * q + 1]), vn2);                       // ||o - v||^2
+            const f32x2 bq = f2_fma(f2_mul(x, um), um, tiny2);                                    // x (1/A - 1)^2
+            const f32x2 Iq = f2_mul(x, f2_make(rsqrt_approx(f2_lo(bq)), rsqrt_approx(f2_hi(bq))));
+            I[2 * q] = f2_lo(Iq);
+            I[2 * q + 1] = f2_hi(Iq);
           }
           if (smax > heavy_thr && j < n) {   // rare: exact distance where the attention weight is large
 #pragma unroll
             for (int u = 0; u < 16; ++u) {
               if (sv[u] > heavy_thr) {
                 const float um = ex2_approx(sv[u] * neg_c2) - 1.f;
-                const float x = fmaxf(
-                    exact_dist2(O_head + (cgp * 32 + c * 16 + u) * kHeadDim, V_head + (long long)j * vsn), 1e-30f);
-                I[u] = x * rsqrt_approx(fmaxf(x * um * um, 1e-36f));
+                const float x = exact_dist2(O_head + (cgp * 32 + c * 16 + u) * kHeadDim, V_head + (long long)j * vsn);
+                I[u] = x * rsqrt_approx(fmaf(x * um, um, 1e-36f));
               }
             }
           }
           if ((c * 16) % kRun == 0) I[0] *= seed_coef;
 #pragma unroll
-          for (int u = 0; u < 16; u += 2) h2 = ffma2(h2, d2, make_float2(I[u], I[u + 1]));
+          for (int q = 0; q < 8; ++q) h2 = f2_fma(h2, d2, f2_make(I[2 * q], I[2 * q + 1]));
           if ((c * 16 + 16) % kRun == 0) {   // end of a run
-            tot += fmaf(h2.x, ema_decay, h2.y);
-            h2 = make_float2(0.f, 0.f);
+            tot += fmaf(f2_lo(h2), ema_decay, f2_hi(h2));
+            h2 = f2_make(0.f, 0.f);
           }
         }
         tc_fence_before();
       }
+      red[it & 3][cgp][t] = tot * fin_scale;
       __syncwarp();
-      if (lane == 0) mbar_arrive(&bar_acc_empty[s]);
-      red[s][cgp][t] = tot * fin_scale;
+      if (lane == 0) {
+        mbar_arrive(&bar_acc_empty[s]);
+        mbar_arrive(&bar_red_full[it & 3]);
+      }
     }
-    named_barrier_sync(1, kP2EpiThreads);
     if (T > 0 && cgp == 0) {
-      const int sl = (T - 1) & 1;
+      const int rs = (T - 1) & 3;
+      ok = ok && mbar_wait(&bar_red_full[rs], (uint32_t)((T - 1) >> 2) & 1u, &abort_flag, dev_status, kDevTimeout);
       const int jl = (tile0 + T - 1) * kTile + t;
-      if (jl < n) I_head[jl] = (red[sl][0][t] + red[sl][1][t]) + (red[sl][2][t] + red[sl][3][t]);
+      if (ok && jl < n) I_head[jl] = (red[rs][0][t] + red[rs][1][t]) + (red[rs][2][t] + red[rs][3][t]);
     }
   }
 
