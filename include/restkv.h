@@ -158,6 +158,34 @@ restkv_status restkv_decode(restkv_handle* h, const restkv_shape* shape, const v
                             const void* Vc, int n_rows, float* out, float* lse, void* workspace,
                             size_t workspace_bytes, restkv_stream stream);
 
+/*
+ * restkv_decode_static -- restkv_decode for callers that cannot give it a workspace.  (The paper has no
+ * counterpart: this is a packaging variant of the decode step above, not another operation.)
+ *
+ * Some hosts of this library cannot allocate device memory when they reach the decode step: an inference
+ * server that handed the whole GPU to its own memory pool at start-up (a later cudaMalloc fails or eats into
+ * the pool's headroom), or a latency-bound token loop that cannot afford the device-wide synchronisation a
+ * cudaMalloc / cudaFree pair brings.  For them the split partials live in a 2 MiB array that is part of the
+ * library image itself, so this call needs neither a handle (restkv_create allocates a status block) nor a
+ * workspace, and it calls no allocating routine of CUDA or of any other library.
+ *
+ *   shape, q, Kc, Vc, n_rows, out, lse   exactly as for restkv_decode (device pointers, caller-owned)
+ *
+ * Limits and rules
+ *  - Capacity: batch * n_q_heads * (head_dim + 2) floats per split must fit in 524288 floats (2 MiB); larger
+ *    shapes return RESTKV_ERR_WORKSPACE and enqueue nothing.  Within the capacity the call uses as many row
+ *    splits as fit (at most 64), so very wide batches run with fewer splits than restkv_decode would use.
+ *  - Every GPU that loads the library carries the 2 MiB until the process exits.
+ *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that
+ *    device current) and remembers it; make that first call outside any stream capture.
+ *  - All calls on a device share the one array.  A call overwrites every slot it later reads, so nothing from
+ *    an earlier call leaks into a result; but two calls whose kernels overlap on the GPU (different streams,
+ *    no ordering between them) race on it.  Order them on one stream or with events.
+ *  - There is no device status word on this path and no launch counter; errors are the return code only.
+ */
+restkv_status restkv_decode_static(const restkv_shape* shape, const void* q, const void* Kc, const void* Vc,
+                                   int n_rows, float* out, float* lse, restkv_stream stream);
+
 /* Synchronises `stream`, then returns and clears the sticky device status (RESTKV_OK if none). */
 restkv_status restkv_poll_status(restkv_handle* h, restkv_stream stream);
 

@@ -21,7 +21,7 @@ PATH_AUTO, PATH_SIMT, PATH_TENSOR_CORE = 0, 1, 2
 
 EXPORTS = [
     "restkv_create", "restkv_destroy", "restkv_workspace_bytes", "restkv_workspace_bytes_adaptive",
-    "restkv_score", "restkv_select", "restkv_compact", "restkv_evict", "restkv_evict_host", "restkv_decode",
+    "restkv_score", "restkv_select", "restkv_compact", "restkv_evict", "restkv_evict_host", "restkv_decode", "restkv_decode_static",
     "restkv_poll_status", "restkv_launch_count", "restkv_last_cuda_error", "restkv_error_string",
     "restkv_set_kernel_path", "restkv_set_profile_events",
 ]
@@ -77,6 +77,7 @@ def load_library() -> ctypes.CDLL:
     lib.restkv_evict.argtypes = [vp, shp, vp, vp, vp, cf, pool, ci, vp, vp, vp, vp, vp, sz, vp]
     lib.restkv_evict_host.argtypes = [vp, shp, vp, vp, vp, cf, pool, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.restkv_decode.argtypes = [vp, shp, vp, vp, vp, ci, vp, vp, vp, sz, vp]
+    lib.restkv_decode_static.argtypes = [shp, vp, vp, vp, ci, vp, vp, vp]
     lib.restkv_poll_status.argtypes = [vp, vp]
     lib.restkv_launch_count.argtypes = [vp]
     lib.restkv_launch_count.restype = ctypes.c_longlong
@@ -119,6 +120,18 @@ def _stream_ptr(stream) -> Optional[int]:
         import torch
         stream = torch.cuda.current_stream()
     return stream.cuda_stream or None
+
+
+def decode_static(shape, q, Kc, Vc, n_rows, out, lse=None, stream=None) -> None:
+    """restkv_decode_static: decode without a handle or a workspace (partials in the library's own 2 MiB array).
+
+    For callers that cannot allocate device memory at this point; see include/restkv.h for the capacity limit
+    and the rule that calls sharing a device must not overlap on the GPU."""
+    lib = load_library()
+    st = lib.restkv_decode_static(ctypes.byref(shape), _ptr(q), _ptr(Kc), _ptr(Vc), int(n_rows), _ptr(out), _ptr(lse),
+                                  _stream_ptr(stream))
+    if st != RESTKV_OK:
+        raise RestKVError(st, "restkv_decode_static")
 
 
 class Handle:

@@ -1,6 +1,10 @@
 // One decode step of every query head over a cache of n_rows rows (Eq. 3): split along the rows,
 // partial softmax attention per split, log-sum-exp merge.  Memory-bound streaming of K and V; all
 // G query heads of a KV head share each row that is loaded.
+#include <math.h>
+
+#include <mutex>
+
 #include "restkv_common.cuh"
 
 namespace restkv {
@@ -216,3 +220,84 @@ cudaError_t launch_decode(const Problem& p, const void* q, const void* Kc, const
 }
 
 }  // namespace restkv
+
+// ================================================================================================
+// restkv_decode_static: the decode step with its split partials in memory that ships with the library.
+// ================================================================================================
+namespace restkv {
+namespace {
+
+// Room for the per-split partial results (m, l, o[head_dim]) of one call.  The array is part of the loaded module:
+// every GPU that loads the library holds these 2 MiB until the process exits, whether the entry point is used or not.
+constexpr size_t kStaticScratchFloats = 512 * 1024;
+static __device__ __align__(256) float g_static_decode_scratch[kStaticScratchFloats];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+float* g_static_scratch_addr[kMaxDevices];   // device address of the array, per device ordinal (null: not looked up yet)
+int g_static_sm_count[kMaxDevices];
+
+// In host code `g_static_decode_scratch` only names the symbol; the address a kernel can use comes from the
+// runtime, for the device that is current.
+cudaError_t static_scratch_for_current_device(float** ptr, int* sm_count) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (!g_static_scratch_addr[dev]) {
+    void* addr = nullptr;
+    e = cudaGetSymbolAddress(&addr, g_static_decode_scratch);
+    if (e != cudaSuccess) return e;
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    g_static_sm_count[dev] = sms > 0 ? sms : 1;
+    g_static_scratch_addr[dev] = (float*)addr;
+  }
+  *ptr = g_static_scratch_addr[dev];
+  *sm_count = g_static_sm_count[dev];
+  return cudaSuccess;
+}
+
+}  // namespace
+}  // namespace restkv
+
+extern "C" restkv_status restkv_decode_static(const restkv_shape* shape, const void* q, const void* Kc, const void* Vc,
+                                              int n_rows, float* out, float* lse, restkv_stream stream) {
+  using namespace restkv;
+  if (!shape || !q || !Kc || !Vc || !out || n_rows < 1) return RESTKV_ERR_INVALID_ARG;
+  if ((((uintptr_t)q) | ((uintptr_t)Kc) | ((uintptr_t)Vc)) & 15u) return RESTKV_ERR_INVALID_ARG;
+  if (shape->batch < 1 || shape->n_q_heads < 1 || shape->n_kv_heads < 1 || shape->head_dim < 1)
+    return RESTKV_ERR_INVALID_ARG;
+  if (shape->n_q_heads % shape->n_kv_heads != 0) return RESTKV_ERR_INVALID_ARG;
+  if (shape->dtype != RESTKV_BF16 && shape->dtype != RESTKV_F32) return RESTKV_ERR_INVALID_ARG;
+  Problem p{};
+  p.batch = shape->batch; p.Hq = shape->n_q_heads; p.Hkv = shape->n_kv_heads; p.G = p.Hq / p.Hkv;
+  p.d = shape->head_dim; p.dtype = shape->dtype; p.BH = p.batch * p.Hkv;
+  p.scale = shape->softmax_scale != 0.f ? shape->softmax_scale : 1.0f / sqrtf((float)p.d);
+  if (!(p.scale > 0.f) || !isfinite(p.scale)) return RESTKV_ERR_INVALID_ARG;
+  if (p.d % 8 != 0 || p.d > 256) return RESTKV_ERR_UNSUPPORTED;
+  if (p.G != 1 && p.G != 2 && p.G != 4 && p.G != 8) return RESTKV_ERR_UNSUPPORTED;
+  const int chunks = p.d * (p.dtype == RESTKV_BF16 ? 2 : 4) / 16;
+  if (chunks != 2 && chunks != 4 && chunks != 8 && chunks != 16 && chunks != 32 && chunks != 64)
+    return RESTKV_ERR_UNSUPPORTED;
+  // one split's partials for every query head must fit; more splits are used only while they fit
+  const size_t per_split = (size_t)p.BH * p.G * (p.d + 2);
+  if (per_split > kStaticScratchFloats) return RESTKV_ERR_WORKSPACE;
+  float* scratch = nullptr;
+  int sm_count = 0;
+  if (static_scratch_for_current_device(&scratch, &sm_count) != cudaSuccess) return RESTKV_ERR_CUDA;
+  int splits = (2 * sm_count + p.BH - 1) / p.BH;
+  const int by_rows = (n_rows + 255) / 256;
+  if (splits > by_rows) splits = by_rows;
+  if (splits > kDecodeMaxSplits) splits = kDecodeMaxSplits;
+  if ((size_t)splits > kStaticScratchFloats / per_split) splits = (int)(kStaticScratchFloats / per_split);
+  if (splits < 1) splits = 1;
+  int n_launches = 0;
+  // Every (head, split) slot that the merge kernel reads is written by the partial kernel of the same call, so
+  // nothing left in the array by an earlier call is ever read and nothing has to be cleared first.
+  const cudaError_t e = launch_decode(p, q, Kc, Vc, n_rows, out, lse, scratch, splits, (cudaStream_t)stream,
+                                      &n_launches);
+  return e == cudaSuccess ? RESTKV_OK : RESTKV_ERR_CUDA;
+}
