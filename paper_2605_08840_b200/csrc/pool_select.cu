@@ -15,11 +15,10 @@ namespace cg = cooperative_groups;
 __device__ __forceinline__ float box_mean(const float* __restrict__ src, int n, int j, int W, int gamma) {
   if (j >= n) return INFINITY;
   const int half = W / 2;
-  long long lo = (long long)j - half + gamma, hi = (long long)j + half + gamma;
-  if (lo < 0) lo = 0;
-  if (hi > n - 1) hi = n - 1;
+  const long long lo64 = (long long)j - half + gamma, hi64 = (long long)j + half + gamma;
+  const int lo = lo64 < 0 ? 0 : (int)(lo64 < n ? lo64 : n), hi = hi64 > n - 1 ? n - 1 : (int)(hi64 > -1 ? hi64 : -1);
   float s = 0.f;
-  for (long long t = lo; t <= hi; ++t) s += src[t];
+  for (int t = lo; t <= hi; ++t) s += src[t];
   return s / (float)W;
 }
 
@@ -42,8 +41,8 @@ __device__ __forceinline__ unsigned int float_key(float x) {
 }
 
 constexpr int kSelThreads = 1024;
-constexpr int kSelBins = 2048;
-constexpr int kSelMaxSmemKeys = 48 * 1024;   // keys of one CTA's slice kept in shared memory (192 KB)
+constexpr int kSelBins = 256;                // 8-bit digits
+constexpr int kSelMaxSmemKeys = 44 * 1024;   // keys of one CTA's slice kept in shared memory (176 KB)
 
 // Inclusive scan over the 1024 threads of the block, in thread order.
 __device__ __forceinline__ unsigned int block_inclusive_scan(unsigned int v, unsigned int* warp_sums) {
@@ -73,10 +72,13 @@ __device__ __forceinline__ unsigned int block_inclusive_scan(unsigned int v, uns
 // One thread-block cluster per row; CTA `rank` of the cluster owns the contiguous slice [rank*per, (rank+1)*per)
 // of the row.  With I_hat non-null the kernel first applies the box mean of Eq. 13 and writes the pooled scores;
 // otherwise it reads `scores`.  The keys of the slice stay in shared memory (use_smem) or are re-read from
-// `scores`.  Three radix passes (11, 11 and 10 bits from the top; per-CTA histograms summed through distributed
-// shared memory) find the key T of the keep-th largest score and how many scores equal to T are kept; an ordered
-// pass then writes, in ascending index order, every index whose key is > T plus the first kept ones whose key
-// equals T (lower index wins ties).
+// `scores`.  The cluster first agrees on the smallest and largest key: the bits they share are common to every
+// key and are skipped.  The remaining bits are resolved 8 at a time from the top: every warp counts into its own
+// 256-bin histogram (no contention between warps), the CTA sums them, the cluster sums the CTAs' histograms
+// through distributed shared memory, and one warp finds the bin that holds the keep-th largest key.  That yields
+// the key T of the keep-th largest score and how many scores equal to T are kept; an ordered pass then writes,
+// in ascending index order, every index whose key is > T plus the first kept ones whose key equals T (lower
+// index wins ties).
 __global__ void __launch_bounds__(kSelThreads, 1)
 select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const int* __restrict__ pool, int W,
               int gamma, float* scores, int32_t* __restrict__ indices, int32_t* __restrict__ pool_used, int per,
@@ -85,10 +87,13 @@ select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const 
   const unsigned int CS = cluster.num_blocks(), rank = cluster.block_rank();
   const int row = blockIdx.x / CS;
   extern __shared__ unsigned int skeys[];
-  __shared__ unsigned int hist[kSelBins];
+  __shared__ unsigned int wh[32][kSelBins];    // per-warp histograms
+  __shared__ unsigned int hist[2][kSelBins];   // the CTA's histogram of the current pass (double-buffered)
+  __shared__ unsigned int tot[kSelBins];       // the cluster's histogram
   __shared__ unsigned int warp_a[32], warp_b[32];
   __shared__ unsigned int s_digit, s_remaining;
   __shared__ unsigned int cta_counts[2];
+  __shared__ unsigned int cta_minmax[2];
 
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const long long j0 = (long long)rank * per;
@@ -117,45 +122,91 @@ select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const 
     return;
   }
 
-  // ---- radix passes ----
-  unsigned int prefix = 0, mask_hi = 0, remaining = (unsigned int)keep;
+  // ---- smallest and largest key of the row ----
+  unsigned int kmin = 0xFFFFFFFFu, kmax = 0u;
+  for (int jj = tid; jj < cnt; jj += kSelThreads) {
+    const unsigned int key = key_at(jj);
+    kmin = min(kmin, key);
+    kmax = max(kmax, key);
+  }
+  kmin = __reduce_min_sync(0xffffffffu, kmin);
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+  if (lane == 0) { warp_a[wid] = kmin; warp_b[wid] = kmax; }
+  __syncthreads();
+  if (wid == 0) {
+    kmin = __reduce_min_sync(0xffffffffu, warp_a[lane]);
+    kmax = __reduce_max_sync(0xffffffffu, warp_b[lane]);
+    if (lane == 0) { cta_minmax[0] = kmin; cta_minmax[1] = kmax; }
+  }
+  cluster.sync();
+  kmin = 0xFFFFFFFFu;
+  kmax = 0u;
+  for (unsigned int r = 0; r < CS; ++r) {
+    const unsigned int* mm = cluster.map_shared_rank(cta_minmax, r);
+    kmin = min(kmin, mm[0]);
+    kmax = max(kmax, mm[1]);
+  }
+
+  // ---- radix passes over the bits in which the keys differ ----
+  const unsigned int diff = kmin ^ kmax;
+  int hi = diff ? 32 - __clz(diff) : 0;                                  // bits [hi-1 .. 0] vary
+  unsigned int prefix = hi >= 32 ? 0u : (kmax >> hi) << hi;              // the bits every key shares
+  unsigned int remaining = (unsigned int)keep;
+  int pb = 0;
 #pragma unroll 1
-  for (int pass = 0; pass < 3; ++pass) {
-    const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
-    const unsigned int dmask = pass == 2 ? 1023u : 2047u;
-    for (int b = tid; b < kSelBins; b += kSelThreads) hist[b] = 0;
+  while (hi > 0) {
+    const int lo = hi > 8 ? hi - 8 : 0;
+    const unsigned int dmask = (1u << (hi - lo)) - 1u;
+    for (int b = tid; b < 32 * kSelBins; b += kSelThreads) (&wh[0][0])[b] = 0;
     __syncthreads();
-    for (int base = 0; base < cnt; base += kSelThreads) {
-      const int jj = base + tid;
-      unsigned int digit = 0xFFFFFFFFu;
-      if (jj < cnt) {
-        const unsigned int key = key_at(jj);
-        if ((key & mask_hi) == prefix) digit = (key >> shift) & dmask;
-      }
-      const unsigned int peers = __match_any_sync(0xffffffffu, digit);
-      if (digit != 0xFFFFFFFFu && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], (unsigned int)__popc(peers));
+    for (int jj = tid; jj < cnt; jj += kSelThreads) {
+      const unsigned int key = key_at(jj);
+      if (hi >= 32 || ((key ^ prefix) >> hi) == 0) atomicAdd(&wh[wid][(key >> lo) & dmask], 1u);
     }
     __syncthreads();
+    if (tid < kSelBins) {
+      unsigned int h = 0;
+#pragma unroll 8
+      for (int wv = 0; wv < 32; ++wv) h += wh[wv][tid];
+      hist[pb][tid] = h;
+    }
     cluster.sync();
-    // totals over the cluster of this thread's two bins (bins in descending order along the threads)
-    const int b0 = kSelBins - 1 - 2 * tid;
-    unsigned int t0 = 0, t1 = 0;
-    for (unsigned int r = 0; r < CS; ++r) {
-      const unsigned int* rh = cluster.map_shared_rank(hist, r);
-      t0 += rh[b0];
-      t1 += rh[b0 - 1];
-    }
-    const unsigned int incl = block_inclusive_scan(t0 + t1, warp_a);
-    const unsigned int excl = incl - (t0 + t1);
-    if (excl < remaining && remaining <= incl) {   // exactly one thread
-      if (excl + t0 >= remaining) { s_digit = (unsigned int)b0; s_remaining = remaining - excl; }
-      else { s_digit = (unsigned int)(b0 - 1); s_remaining = remaining - excl - t0; }
+    if (tid < kSelBins) {
+      unsigned int h = 0;
+      for (unsigned int r = 0; r < CS; ++r) h += cluster.map_shared_rank(&hist[pb][0], r)[tid];
+      tot[tid] = h;
     }
     __syncthreads();
-    prefix |= s_digit << shift;
-    mask_hi |= dmask << shift;
+    if (wid == 0) {
+      // lane L owns bins 255-8L .. 248-8L, so that the lanes walk the bins from the top
+      unsigned int mine[8], sum = 0;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) { mine[k] = tot[kSelBins - 1 - 8 * lane - k]; sum += mine[k]; }
+      unsigned int incl = sum;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const unsigned int t = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += t;
+      }
+      unsigned int acc = incl - sum;
+      if (acc < remaining && remaining <= incl) {   // exactly one lane
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          if (acc < remaining && remaining <= acc + mine[k]) {
+            s_digit = (unsigned int)(kSelBins - 1 - 8 * lane - k);
+            s_remaining = remaining - acc;
+          }
+          acc += mine[k];
+        }
+      }
+    }
+    __syncthreads();
+    prefix |= s_digit << lo;
     remaining = s_remaining;
-    cluster.sync();   // no CTA clears its histogram while a peer still reads it
+    hi = lo;
+    pb ^= 1;
+    // hist[pb] is rewritten two passes later, after another cluster.sync that every peer reaches only once it
+    // has finished reading this pass's histograms
   }
   const unsigned int T = prefix;            // key of the keep-th largest score
   const unsigned int need_eq = remaining;   // how many keys equal to T are kept (>= 1)
@@ -254,18 +305,17 @@ cudaError_t launch_pool(const Problem& p, const Workspace& ws, const int* pool_d
 cudaError_t launch_select(int rows, int n, int n_kv, int budget, const float* I_hat, const int* pool_dev, int W,
                           int gamma, float* scores, int32_t* indices, int32_t* pool_used, cudaStream_t st) {
   const int keep = budget < n_kv ? budget : n_kv;
-  const int CS = n_kv > 4096 ? 8 : 1;
-  int per = (n_kv + CS - 1) / CS;
-  per = (per + 3) & ~3;
-  const int use_smem = per <= kSelMaxSmemKeys ? 1 : 0;
-  const size_t smem = use_smem ? (size_t)per * sizeof(unsigned int) : 0;
+  int CS = n_kv > 4096 ? 8 : 1;
   cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        kSelMaxSmemKeys * (int)sizeof(unsigned int));
   if (e != cudaSuccess) return e;
+  int per = (n_kv + CS - 1) / CS;
+  per = (per + 3) & ~3;
+  const int use_smem = per <= kSelMaxSmemKeys ? 1 : 0;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned int)(rows * CS));
   cfg.blockDim = dim3(kSelThreads);
-  cfg.dynamicSmemBytes = smem;
+  cfg.dynamicSmemBytes = use_smem ? (size_t)per * sizeof(unsigned int) : 0;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;

@@ -50,9 +50,14 @@ size_t plan_workspace(const Problem& p, int budget, int sm_count, bool adaptive,
   w.splits = pass1_splits(p, sm_count);
   const size_t BH = (size_t)p.BH, R = (size_t)p.R, d = (size_t)p.d;
   w.parts = w.splits;
-  w.part_m = (float*)take(BH * 2 * w.splits * R * sizeof(float));
-  w.part_l = (float*)take(BH * 2 * w.splits * R * sizeof(float));
-  w.part_O = (float*)take(BH * 2 * w.splits * R * d * sizeof(float));
+  // partial slots: two per (head, split) for the two-kernel paths, one per CTA for the head-sequential kernel
+  size_t slots = BH * 2 * w.splits;
+  if (slots < (size_t)sm_count) slots = (size_t)sm_count;
+  w.part_m = (float*)take(slots * R * sizeof(float));
+  w.part_l = (float*)take(slots * R * sizeof(float));
+  w.part_O = (float*)take(slots * R * d * sizeof(float));
+  w.counters = (unsigned int*)take(1024);
+  w.heavy = (unsigned int*)take(BH * (size_t)((p.n_kv + 127) / 128) * 4 * sizeof(unsigned int));
   w.vnorm = (float*)take(BH * (size_t)p.n_kv * sizeof(float));
   w.fin_m = (float*)take(BH * R * sizeof(float));
   w.fin_l = (float*)take(BH * R * sizeof(float));
@@ -161,7 +166,7 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
   // the tensor-core pass 2 seeds its EMA chain with 1/alpha, so ema_decay = 1 (alpha = 0) runs on the SIMT kernels
   bool use_tc = tc_supported(p) && c.h->tc_state != nullptr && !adaptive && ema_decay < 1.f;
   if (c.h->kernel_path == 1) use_tc = false;
-  if (c.h->kernel_path == 2 && !use_tc) return RESTKV_ERR_UNSUPPORTED;
+  if (c.h->kernel_path >= 2 && !use_tc) return RESTKV_ERR_UNSUPPORTED;
   if (!use_tc && !simt_supported(p)) return RESTKV_ERR_UNSUPPORTED;
   if (p.n_kv == 1) {
     // A single visible row has A = 1 and nothing to redistribute its weight to: the indicator is
@@ -170,6 +175,10 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
     if (e == cudaSuccess && adaptive)
       e = cudaMemsetAsync(ws.I_raw, 0, (size_t)p.batch * p.Hq * p.w * p.n * sizeof(float), c.st);
     if (e != cudaSuccess) return c.fail(e);
+  } else if (use_tc && c.h->kernel_path == 4) {
+    // pass 1, merge and pass 2 of every head in one head-sequential launch (timed as "pass 2")
+    RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2,
+                  launch_tc_fused(c.h->tc_state, p, ws, Q, K, V, ema_decay, c.h->sm_count, c.h->dev_status, c.st), 1);
   } else if (use_tc) {
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS1, launch_tc_pass1(c.h->tc_state, p, ws, Q, K, V, c.h->dev_status, c.st), 1);
     RESTKV_LAUNCH(c, RESTKV_KERNEL_COMBINE, launch_combine(p, ws, 2 * ws.splits, c.st), 1);   // two warpgroups per CTA
@@ -219,7 +228,7 @@ restkv_status restkv_create(restkv_handle** out) {
   if (e == cudaSuccess) e = cudaMemset(h->dev_status, 0, 256);
   if (e != cudaSuccess) { delete h; return RESTKV_ERR_CUDA; }
   h->tc_state = nullptr;
-  if (tc_init(&h->tc_state) != cudaSuccess) h->tc_state = nullptr;
+  if (tc_init(&h->tc_state) != cudaSuccess || tc_fused_init() != cudaSuccess) h->tc_state = nullptr;
   h->launches = 0;
   h->last_cuda_error = 0;
   h->kernel_path = 0;
@@ -426,7 +435,7 @@ restkv_status restkv_set_profile_events(restkv_handle* h, int which, void* start
 }
 
 restkv_status restkv_set_kernel_path(restkv_handle* h, int path) {
-  if (!h || path < 0 || path > 2) return RESTKV_ERR_INVALID_ARG;
+  if (!h || path < 0 || path > 4) return RESTKV_ERR_INVALID_ARG;
   h->kernel_path = path;
   return RESTKV_OK;
 }

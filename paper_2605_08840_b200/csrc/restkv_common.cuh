@@ -34,6 +34,8 @@ struct Workspace {
   float* part_l;          // [BH, parts, R]
   float* part_O;          // [BH, parts, R, d]
   float* vnorm;           // [BH, n_kv]  ||v_j||^2 (tensor-core path)
+  unsigned int* counters; // [256] group barrier counters of the head-sequential kernel
+  unsigned int* heavy;    // [BH, tiles, 4] per-tile flags of the head-sequential kernel
   float* fin_m;           // [BH, R]    row max of the scaled logits (natural units)
   float* fin_l;           // [BH, R]    sum of exp(s - m)
   float* O_f32;           // [BH, R, d]
@@ -78,6 +80,9 @@ bool tc_supported(const Problem& p);
 cudaError_t tc_init(void** state);   // resolves the driver entry point for tensor-map encoding
 cudaError_t launch_tc_pass1(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
                             const void* V, unsigned int* dev_status, cudaStream_t st);
+cudaError_t tc_fused_init();
+cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
+                            const void* V, float ema_decay, int sm_count, unsigned int* dev_status, cudaStream_t st);
 cudaError_t launch_tc_pass2(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
                             const void* V, float ema_decay, unsigned int* dev_status, cudaStream_t st);
 

@@ -1,0 +1,98 @@
+// Shared pieces of the tensor-core score kernels: tile geometry, UMMA descriptors, tensor-map builders.
+#pragma once
+
+#include <cuda.h>
+
+#include "restkv_common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace restkv {
+namespace {
+
+using namespace ptx;
+
+constexpr int kTile = 128;                       // tokens per tile
+constexpr int kHeadDim = 128;
+constexpr int kRows = 128;                       // query rows per KV head (w * G)
+constexpr uint32_t kBoxBytes = 128 * 64 * 2;     // one [128 rows x 64 bf16] TMA box
+constexpr uint32_t kTileBytes = 2 * kBoxBytes;   // a [128 x 128] bf16 operand tile
+constexpr uint32_t kStageBytes = 2 * kTileBytes; // K tile + V tile
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kRescaleThreshold = 8.0f;        // log2 units the running maximum may exceed the reference by
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct TcState {
+  EncodeTiledFn encode;
+};
+
+constexpr uint32_t kIdescKK = make_idesc_bf16(128, 128, false);   // both operands K-major
+constexpr uint32_t kIdescKMN = make_idesc_bf16(128, 128, true);   // B operand MN-major (V in O += P V)
+
+__device__ __forceinline__ uint64_t kmajor_desc(uint32_t addr) { return make_smem_desc(addr, 16, 1024); }
+
+// D[128 x 128] (+)= A[128 x 128] * B[128 x 128]^T, both operands K-major 128B-swizzled [128 x 128] bf16 tiles
+// made of two [128 x 64] boxes.  One thread issues the eight K = 16 steps.
+__device__ __forceinline__ void mma_tile_kk(uint32_t tmem_d, uint32_t a_smem, uint32_t b_smem, bool accumulate) {
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const uint32_t off = (uint32_t)(k >> 2) * kBoxBytes + (uint32_t)(k & 3) * 32u;
+    umma_ss(tmem_d, kmajor_desc(a_smem + off), kmajor_desc(b_smem + off), kIdescKK, accumulate || k > 0);
+  }
+}
+
+constexpr uint32_t kAugBytes = kBoxBytes;     // [128 rows x 64 bf16], only K steps 0 (S') and 1 (C') are used
+constexpr uint32_t kOnesBytes = 1024;         // one 8-row group of ones, shared by all 16 groups (stride 0)
+constexpr float kHeavyA = 0.125f;             // attention weight above which ||o - v||^2 is recomputed exactly
+
+// Exact ||o - v||^2 for the rare entries whose attention weight is large (the expansion
+// ||o||^2 + ||v||^2 - 2 o.v cancels when o approaches v).
+__device__ __noinline__ float exact_dist2(const float* __restrict__ o_row, const __nv_bfloat16* __restrict__ v_row) {
+  float ss = 0.f;
+  for (int k = 0; k < kHeadDim; k += 2) {
+    const float2 o = *reinterpret_cast<const float2*>(o_row + k);
+    const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(v_row + k);
+    const float d0 = o.x - __low2float(v), d1 = o.y - __high2float(v);
+    ss = fmaf(d0, d0, ss);
+    ss = fmaf(d1, d1, ss);
+  }
+  return ss;
+}
+
+// ------------------------------------------------------------------------------------------------
+inline CUresult encode_tiles(TcState* st, CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims,
+                      const cuuint64_t* strides_bytes) {
+  cuuint32_t box[4] = {64, 128, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  return st->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), dims,
+                    strides_bytes, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
+inline bool make_rows_map(TcState* st, CUtensorMap* map, const void* base, int BH) {   // [BH, 128, 128] contiguous
+  cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)kRows, (cuuint64_t)BH};
+  cuuint64_t str[2] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)kRows * kHeadDim * 2};
+  return encode_tiles(st, map, base, 3, dims, str) == CUDA_SUCCESS;
+}
+
+inline bool make_aug_map(TcState* st, CUtensorMap* map, const void* base, int BH) {   // [BH, 128, 64] contiguous
+  cuuint64_t dims[3] = {64, (cuuint64_t)kRows, (cuuint64_t)BH};
+  cuuint64_t str[2] = {64 * 2, (cuuint64_t)kRows * 64 * 2};
+  return encode_tiles(st, map, base, 3, dims, str) == CUDA_SUCCESS;
+}
+
+inline bool make_kv_map(TcState* st, CUtensorMap* map, const void* base, const Problem& p, long long sb, long long sh,
+                 long long sn) {
+  cuuint64_t dims[4] = {(cuuint64_t)p.d, (cuuint64_t)p.n_kv, (cuuint64_t)p.Hkv, (cuuint64_t)p.batch};
+  // a dimension of extent 1 may carry any stride; give it a valid one
+  cuuint64_t str[3] = {(cuuint64_t)sn * 2, (cuuint64_t)(p.Hkv > 1 ? sh : sn) * 2,
+                       (cuuint64_t)(p.batch > 1 ? sb : sn) * 2};
+  return encode_tiles(st, map, base, 4, dims, str) == CUDA_SUCCESS;
+}
+
+
+}  // namespace
+}  // namespace restkv

@@ -1,0 +1,855 @@
+// Head-sequential tensor-core score kernel for sm_100a (bf16, head_dim 128, w * group = 128 query rows).
+//
+// One persistent CTA per SM.  The CTAs are divided into groups; a group takes one (batch, KV head) at a time and
+// runs, back to back,
+//   phase A  (Eq. 3)    every CTA of the group: S = Q K^T, online softmax, O += P V over its share of the tiles
+//   phase B             the group's partial (m, l, O) are merged row by row (one warp per query row)
+//   phase C  (Eq. 7-9)  every CTA: S^T = K Q^T, C^T = V (-2 O)^T over its share of the tiles, indicator, EMA,
+//                       group mean
+// so that phase C finds the head's K and V in L2 (a head is 64 MiB at 128k tokens; L2 holds 126 MB) and HBM sees
+// each row once.  The CTAs of a group meet at two counter barriers per head (after A and after B); different
+// groups never wait for one another.  Every wait is bounded: a wait that runs out sets the sticky timeout bit,
+// and the CTA skips the rest of its work and still releases its tensor memory.
+#include "tc_common.cuh"
+
+namespace restkv {
+
+namespace {
+
+constexpr int kFFirstWorker = 2;                  // warp 0: TMA producer, warp 1: MMA issuer
+constexpr int kFWorkerWarps = 16;                 // warps 2..17
+constexpr int kFThreads = (kFFirstWorker + kFWorkerWarps) * 32;
+constexpr int kFRing = 4;                         // 32 KB tile slots after Q | O' | aug | ones
+constexpr size_t kFSmem = 2 * kTileBytes + kAugBytes + kOnesBytes + kFRing * kTileBytes + 1024;
+constexpr int kFVSlots = 3;                       // phase A: V slots = ring 2, ring 3 and the (then unused) O' tile
+
+struct FusedArgs {
+  int Hkv, BH, n, n_kv, w;
+  float scale, ema_decay;
+  int groups, cpg;                   // CTA groups and CTAs per group
+  float* part_m;                     // [CTA, 128]       running maximum, log2 units (one slot per CTA, reused
+  float* part_l;                     // [CTA, 128]        from head to head: a group is past phase B of a head
+  float* part_O;                     // [CTA, 128, 128]   before any of its CTAs writes the next head's partial)
+  float* O_f32;                      // [BH, 128, 128]
+  __nv_bfloat16* O_m2;               // [BH, 128, 128]  -2 * bf16(O)
+  __nv_bfloat16* aug;                // [BH, 128, 64]
+  float* vnorm;                      // [BH, n_kv]
+  unsigned int* heavy;               // [BH, tiles]: bit per softmax warp, set if the tile may hold a weight > kHeavyA
+  float* I_hat;                      // [BH, n]
+  const __nv_bfloat16* V;
+  long long vsb, vsh, vsn;
+  unsigned int* counters;            // [groups] (at most 256), zero at launch
+  unsigned int* dev_status;
+};
+
+struct FusedBars {
+  // phase A
+  uint64_t q_full, k_full[2], k_empty[2], v_full[kFVSlots], v_empty[kFVSlots], s_full[2], p_full[2], pv_done[2];
+  // phase C
+  uint64_t const_full, kv_full[2], kv_empty[2], acc_full[2], acc_empty[2], red_full[4];
+};
+
+__device__ __forceinline__ void mbar_inval(uint64_t* bar) {
+  asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ void named_barrier_sync(int id, int count) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p) {
+  unsigned int v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// (Re)initialises every mbarrier of the CTA for one phase.  Called by one thread between two __syncthreads.
+__device__ void init_bars(FusedBars* B, bool first) {
+  uint64_t* all = reinterpret_cast<uint64_t*>(B);
+  constexpr int kCount = sizeof(FusedBars) / sizeof(uint64_t);
+  if (!first)
+    for (int i = 0; i < kCount; ++i) mbar_inval(all + i);
+  mbar_init(&B->q_full, 1);
+  for (int i = 0; i < 2; ++i) {
+    mbar_init(&B->k_full[i], 1);
+    mbar_init(&B->k_empty[i], 1);
+    mbar_init(&B->s_full[i], 1);
+    mbar_init(&B->p_full[i], 128);
+    mbar_init(&B->pv_done[i], 1);
+    mbar_init(&B->kv_full[i], 1);
+    mbar_init(&B->kv_empty[i], 1);
+    mbar_init(&B->acc_full[i], 1);
+    mbar_init(&B->acc_empty[i], kFWorkerWarps);
+  }
+  for (int i = 0; i < kFVSlots; ++i) {
+    mbar_init(&B->v_full[i], 1);
+    mbar_init(&B->v_empty[i], 1 + 4);   // MMA commit + the four warps that reduce ||v||^2
+  }
+  mbar_init(&B->const_full, 1);
+  for (int i = 0; i < 4; ++i) mbar_init(&B->red_full[i], kFWorkerWarps);
+  fence_mbar_init();
+}
+
+// All CTAs of a group arrive and wait until `target` arrivals have been counted.  Bounded.
+__device__ bool group_barrier(unsigned int* counter, unsigned int target, volatile int* abort_flag,
+                              unsigned int* dev_status) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    // release: everything the CTA wrote before the __syncthreads is visible to whoever acquires the count
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(counter), "r"(1u) : "memory");
+    const long long t0 = clock64();
+    while (ld_acquire_gpu(counter) < target) {
+      if (*abort_flag) break;
+      if (clock64() - t0 > 2000000000ll) {
+        *abort_flag = 1;
+        atomicOr(dev_status, kDevTimeout);
+        break;
+      }
+    }
+  }
+  __syncthreads();
+  return *abort_flag == 0;
+}
+
+struct Ctx {
+  uint32_t smem_base;      // shared-window address of the 1024-aligned dynamic region
+  uint8_t* gen_base;       // the same location as a generic pointer
+  uint32_t tmem;
+  FusedBars* B;
+  int* abort_flag;
+  float* sm_stats;         // [2][128] floats: (m, l) of warpgroup 1 for the in-CTA merge
+  int warp, lane;
+};
+
+constexpr uint32_t kOffQ = 0, kOffO = kTileBytes, kOffAug = 2 * kTileBytes, kOffOnes = kOffAug + kAugBytes,
+                   kOffRing = kOffOnes + kOnesBytes;
+__device__ __forceinline__ uint32_t k_slot_off(int i) { return kOffRing + (uint32_t)i * kTileBytes; }
+__device__ __forceinline__ uint32_t v_slot_off(int i) { return i < 2 ? kOffRing + (uint32_t)(2 + i) * kTileBytes : kOffO; }
+
+// ------------------------------------------------------------------------------------------------
+// Phase A: this CTA's share [tile0, tile0 + T) of one head.  Warp 0 loads, warp 1 issues the MMAs, worker warps
+// 0-7 are two softmax warpgroups (thread = query row; warpgroup g owns tiles g, g+2, ... with its own running
+// maximum and its own O accumulator), worker warps 8-15 reduce ||v_j||^2 of the tokens from the V tiles.
+// Tensor memory: S_g at g*128 (bf16 P_g overwrites its first 64 columns), O_g at 256 + g*128.
+// At the end the two warpgroups' (m, l, O) are merged and written as the CTA's partial.
+__device__ void phase_a(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tmQ, const CUtensorMap* tmK,
+                        const CUtensorMap* tmV, int bh, int rank, int tile0, int T) {
+  FusedBars* B = cx.B;
+  int* abort_flag = cx.abort_flag;
+  unsigned int* dev_status = a.dev_status;
+  const int b = bh / a.Hkv, h = bh % a.Hkv;
+  const int warp = cx.warp, lane = cx.lane;
+  const uint32_t tmem = cx.tmem;
+
+  if (warp == 0) {
+    if (lane == 0 && T > 0) {
+      mbar_arrive_expect_tx(&B->q_full, kTileBytes);
+      tma_load_3d(cx.gen_base + kOffQ, tmQ, &B->q_full, 0, 0, bh);
+      tma_load_3d(cx.gen_base + kOffQ + kBoxBytes, tmQ, &B->q_full, 64, 0, bh);
+      for (int it = 0; it < T; ++it) {
+        const int ks = it & 1, vs = it % kFVSlots;
+        const int j0 = (tile0 + it) * kTile;
+        if (it >= 2 && !mbar_wait(&B->k_empty[ks], ((it >> 1) - 1) & 1, abort_flag, dev_status, kDevTimeout)) break;
+        uint8_t* dK = cx.gen_base + k_slot_off(ks);
+        mbar_arrive_expect_tx(&B->k_full[ks], kTileBytes);
+        tma_load_4d(dK, tmK, &B->k_full[ks], 0, j0, h, b);
+        tma_load_4d(dK + kBoxBytes, tmK, &B->k_full[ks], 64, j0, h, b);
+        if (it >= kFVSlots &&
+            !mbar_wait(&B->v_empty[vs], (it / kFVSlots - 1) & 1, abort_flag, dev_status, kDevTimeout))
+          break;
+        uint8_t* dV = cx.gen_base + v_slot_off(vs);
+        mbar_arrive_expect_tx(&B->v_full[vs], kTileBytes);
+        tma_load_4d(dV, tmV, &B->v_full[vs], 0, j0, h, b);
+        tma_load_4d(dV + kBoxBytes, tmV, &B->v_full[vs], 64, j0, h, b);
+      }
+    }
+  } else if (warp == 1) {
+    // S(it), then O += P V of tile it - 1
+    if (lane == 0 && T > 0) {
+      bool ok = mbar_wait(&B->q_full, 0, abort_flag, dev_status, kDevTimeout);
+      for (int it = 0; ok && it <= T; ++it) {
+        if (it < T) {
+          const int ks = it & 1, g = it & 1;
+          if (!mbar_wait(&B->k_full[ks], (it >> 1) & 1, abort_flag, dev_status, kDevTimeout)) break;
+          tc_fence_after();
+          // S_g may be overwritten: O += P V of tile it - 2 (which read P_g) was issued earlier and MMAs run in order
+          mma_tile_kk(tmem + (uint32_t)g * 128u, cx.smem_base + kOffQ, cx.smem_base + k_slot_off(ks), false);
+          umma_commit(&B->s_full[g]);
+          umma_commit(&B->k_empty[ks]);
+        }
+        if (it >= 1) {
+          const int pt = it - 1, g = pt & 1, vs = pt % kFVSlots;
+          if (!mbar_wait(&B->p_full[g], (pt >> 1) & 1, abort_flag, dev_status, kDevTimeout)) break;
+          if (!mbar_wait(&B->v_full[vs], (pt / kFVSlots) & 1, abort_flag, dev_status, kDevTimeout)) break;
+          tc_fence_after();
+          // A = P_g in TMEM (16 tokens = 8 packed columns per K step), B = V tile, MN-major
+          const uint32_t vaddr = cx.smem_base + v_slot_off(vs);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const uint64_t bdesc = make_smem_desc(vaddr + (uint32_t)k * 2048u, kBoxBytes, 1024);
+            umma_ts(tmem + 256u + (uint32_t)g * 128u, tmem + (uint32_t)g * 128u + (uint32_t)k * 8u, bdesc, kIdescKMN,
+                    pt >= 2 || k > 0);
+          }
+          umma_commit(&B->pv_done[g]);
+          umma_commit(&B->v_empty[vs]);
+        }
+      }
+    }
+  } else if (warp >= kFFirstWorker + 8) {
+    // ---------------- ||v||^2: worker warpgroup 2 takes the even tiles, 3 the odd ones ----------------
+    const int vg = (warp - kFFirstWorker - 8) >> 2;
+    const int row = ((warp - kFFirstWorker - 8) & 3) * 32 + lane;
+    bool ok = true;
+    for (int it = 0; it < T && ok; ++it) {
+      const int vs = it % kFVSlots;
+      // both warpgroups wait for every tile so that neither falls a whole phase behind a slot's barrier
+      ok = mbar_wait(&B->v_full[vs], (it / kFVSlots) & 1, abort_flag, dev_status, kDevTimeout);
+      if (!ok || (it & 1) != vg) continue;
+      // 16-byte chunk c of row r of a 128-byte-swizzled box sits at chunk c ^ (r & 7)
+      const uint8_t* vt = cx.gen_base + v_slot_off(vs);
+      float2 acc = make_float2(0.f, 0.f);
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const uint8_t* rowp = vt + half * kBoxBytes + (row >> 3) * 1024 + (row & 7) * 128;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const uint4 u = *reinterpret_cast<const uint4*>(rowp + ((c ^ (row & 7)) << 4));
+          const unsigned int wv[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const float2 e = make_float2(__uint_as_float(wv[q] << 16), __uint_as_float(wv[q] & 0xFFFF0000u));
+            acc = ffma2(e, e, acc);
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&B->v_empty[vs]);
+      const int j = (tile0 + it) * kTile + row;
+      if (j < a.n_kv) a.vnorm[(long long)bh * a.n_kv + j] = acc.x + acc.y;
+    }
+  } else {
+    // ---------------- softmax warpgroups: thread = query row ----------------
+    const int g = (warp - kFFirstWorker) >> 2;
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;
+    const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+    const uint32_t tS = tmem + (uint32_t)g * 128u + lane_base, tO = tmem + 256u + (uint32_t)g * 128u + lane_base;
+    const int i_q = row % a.w;                // window position of this row (row = group * w + i)
+    const float c2 = a.scale * kLog2e;
+    const int n = a.n, n_kv = a.n_kv;
+    const int nt_all = (n_kv + kTile - 1) / kTile;
+    float m_ref = -INFINITY;
+    float2 l2 = make_float2(0.f, 0.f);
+    bool ok = true;
+    int uses = 0;                             // tiles this warpgroup has processed
+    for (int it = g; it < T; it += 2, ++uses) {
+      ok = ok && mbar_wait(&B->s_full[g], (uint32_t)uses & 1u, abort_flag, dev_status, kDevTimeout);
+      if (!ok) break;
+      tc_fence_after();
+      const int j0 = (tile0 + it) * kTile;
+      const bool ragged = j0 + kTile > n;   // rows past the scored prefix: window rows (causal) or padding
+      // Both sweeps keep the next 16 columns in flight from tensor memory while the current ones are worked on.
+      auto mask = [&](float* s, int c) {
+#pragma unroll
+        for (int u = 0; u < 16; ++u) {
+          const int j = j0 + c * 16 + u;
+          const bool vis = (j < n_kv) && (j < n || (j - n) <= i_q);
+          s[u] = vis ? s[u] : -INFINITY;
+        }
+      };
+      float sa[16], sb[16];
+      // ---- sweep 1: row maximum of the tile ----
+      float tmax = -INFINITY;
+      tmem_ld16(tS, sa);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        float* cur = (c & 1) ? sb : sa;
+        float* nxt = (c & 1) ? sa : sb;
+        tmem_wait_ld();
+        tmem_ld16(tS + ((c + 1) & 7) * 16, nxt);   // after the last chunk: chunk 0 again, for sweep 2
+        if (ragged) mask(cur, c);
+#pragma unroll
+        for (int u = 0; u < 16; ++u) tmax = fmaxf(tmax, cur[u]);
+      }
+      const float m_tile = tmax * c2;
+      const bool need = m_tile > m_ref + kRescaleThreshold;   // also true for the first visible entries (m_ref = -inf)
+      float factor = 1.f;
+      if (need) {
+        factor = ex2_approx(m_ref - m_tile);   // 0 when m_ref = -inf
+        l2.x *= factor;
+        l2.y *= factor;
+        m_ref = m_tile;
+      }
+      // S(it) has landed, so O += P V of this warpgroup's previous tile (issued before it) is complete
+      if (uses > 0 && __any_sync(0xffffffffu, need)) {
+        tmem_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          float o[16];
+          tmem_ld16(tO + c * 16, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int u = 0; u < 16; ++u) o[u] *= factor;
+          tmem_st16(tO + c * 16, reinterpret_cast<const uint32_t*>(o));
+        }
+      }
+      // ---- sweep 2: P = exp2(s*c2 - m_ref) as bf16 over the first 64 columns of S_g.  Chunk c of P lands on
+      //      columns [8c, 8c + 8), which belong to a chunk of S that is already in registers. ----
+      const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+      const float2 c22 = make_float2(c2, c2), nm2 = make_float2(-m_use, -m_use);
+      __nv_bfloat162 pmax2 = __float2bfloat162_rn(0.f);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        float* cur = (c & 1) ? sb : sa;     // chunk 0 sits in sa (loaded at the end of sweep 1)
+        float* nxt = (c & 1) ? sa : sb;
+        tmem_wait_ld();
+        if (c < 7) tmem_ld16(tS + (c + 1) * 16, nxt);
+        if (ragged) mask(cur, c);
+        uint32_t packed[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const float2 e = ffma2(make_float2(cur[2 * u], cur[2 * u + 1]), c22, nm2);
+          const float2 pp = make_float2(ex2_approx(e.x), ex2_approx(e.y));
+          l2 = fadd2(l2, pp);
+          packed[u] = pack_bf16x2(pp.x, pp.y);
+          pmax2 = __hmax2(pmax2, *reinterpret_cast<const __nv_bfloat162*>(&packed[u]));
+        }
+        tmem_st8(tS + c * 8, packed);
+      }
+      // The final attention weight of an entry is p / l_final with both taken against the same reference, and
+      // l_final is at least the sum this warpgroup has so far: a tile without p > kHeavyA * l needs no exact
+      // distances in phase C.
+      {
+        const bool hv = fmaxf(__low2float(pmax2), __high2float(pmax2)) > kHeavyA * (l2.x + l2.y);
+        const unsigned int any = __any_sync(0xffffffffu, hv) ? 1u : 0u;
+        if (lane == 0) a.heavy[((long long)bh * nt_all + tile0 + it) * 4 + quad] = any;
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&B->p_full[g]);
+    }
+    if (uses > 0 && ok) ok = mbar_wait(&B->pv_done[g], (uint32_t)(uses - 1) & 1u, abort_flag, dev_status, kDevTimeout);
+    if (ok && uses > 0) tc_fence_after();
+    const bool have = ok && uses > 0;
+    const float m_mine = have ? m_ref : -INFINITY, l_mine = have ? l2.x + l2.y : 0.f;
+
+    // ---- merge the two warpgroups: 1 hands (m, l, O) over through shared memory (the K slots are idle: every
+    //      MMA of this phase has completed once both warpgroups have seen their last O += P V) ----
+    float* xO = reinterpret_cast<float*>(cx.gen_base + k_slot_off(0));   // [128 cols][128 rows] floats, 64 KB
+    named_barrier_sync(1, 256);
+    if (g == 1) {
+      cx.sm_stats[row] = m_mine;
+      cx.sm_stats[128 + row] = l_mine;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        float o[32];
+        if (have) {
+          tmem_ld32(tO + c * 32, o);
+          tmem_wait_ld();
+        } else {
+#pragma unroll
+          for (int u = 0; u < 32; ++u) o[u] = 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < 32; ++u) xO[(c * 32 + u) * 128 + row] = o[u];
+      }
+    }
+    named_barrier_sync(1, 256);
+    if (g == 0) {
+      const float m1 = cx.sm_stats[row], l1 = cx.sm_stats[128 + row];
+      const float m = fmaxf(m_mine, m1);
+      const float a0 = (m_mine == -INFINITY) ? 0.f : ex2_approx(m_mine - m);
+      const float a1 = (m1 == -INFINITY) ? 0.f : ex2_approx(m1 - m);
+      const long long o_idx = (long long)blockIdx.x * kRows + row;
+      float* Op = a.part_O + o_idx * kHeadDim;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        float o[32];
+        if (have) {
+          tmem_ld32(tO + c * 32, o);
+          tmem_wait_ld();
+        } else {
+#pragma unroll
+          for (int u = 0; u < 32; ++u) o[u] = 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < 32; ++u) o[u] = o[u] * a0 + xO[(c * 32 + u) * 128 + row] * a1;
+#pragma unroll
+        for (int u = 0; u < 32; u += 4)
+          *reinterpret_cast<float4*>(Op + c * 32 + u) = make_float4(o[u], o[u + 1], o[u + 2], o[u + 3]);
+      }
+      a.part_m[o_idx] = m;
+      a.part_l[o_idx] = l_mine * a0 + l1 * a1;
+    }
+    fence_proxy_async_smem();   // the hand-over buffer lies in the tile ring, which TMA loads refill next
+    tc_fence_before();
+  }
+}
+
+// x = hi + mid + lo with three bf16 pieces (24 significant bits).
+__device__ __forceinline__ void split3(float x, __nv_bfloat16* out) {
+  const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+  const float r1 = x - __bfloat162float(hi);
+  const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+  out[0] = hi;
+  out[1] = mid;
+  out[2] = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+}
+
+// ------------------------------------------------------------------------------------------------
+// Phase B: the group's `cpg` partials of one query row are merged by `wpr` warps (lane = four output dims; warp
+// `sub` of the row takes partials sub, sub + wpr, ...), whose sums meet in shared memory and are added in a fixed
+// order: the result does not depend on timing.  Written for phase C: O (fp32), -2 bf16(O), and the row's strip
+// of bf16 constant pieces.  Called by all sixteen worker warps; r < 0 means this warp has no row.
+__device__ void combine_rows(const FusedArgs& a, int bh, int group, int r, int sub, int wpr, int wq, int lane,
+                             float (*xch)[kHeadDim + 4]) {
+  float m = -INFINITY, l = 0.f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (r >= 0) {
+    const long long base = (long long)group * a.cpg * kRows + r;   // + p * kRows
+    // running merge of this warp's partials (all loads of a batch are issued before any is used)
+#pragma unroll 1
+    for (int p0 = sub; p0 < a.cpg; p0 += 4 * wpr) {
+      float mp[4], lp[4];
+      float4 v[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int p = p0 + k * wpr;
+        const bool in = p < a.cpg;
+        const long long pi = base + (long long)(in ? p : p0) * kRows;
+        mp[k] = in ? a.part_m[pi] : -INFINITY;
+        lp[k] = a.part_l[pi];
+        v[k] = *reinterpret_cast<const float4*>(a.part_O + pi * kHeadDim + lane * 4);
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float m_new = fmaxf(m, mp[k]);
+        const float s_old = (m == -INFINITY) ? 0.f : ex2_approx(m - m_new);
+        const float s_p = (mp[k] == -INFINITY) ? 0.f : ex2_approx(mp[k] - m_new);   // an empty partial weighs 0
+        l = l * s_old + lp[k] * s_p;
+        acc.x = acc.x * s_old + v[k].x * s_p;
+        acc.y = acc.y * s_old + v[k].y * s_p;
+        acc.z = acc.z * s_old + v[k].z * s_p;
+        acc.w = acc.w * s_old + v[k].w * s_p;
+        m = m_new;
+      }
+    }
+    *reinterpret_cast<float4*>(&xch[wq][lane * 4]) = acc;
+    if (lane == 0) { xch[wq][kHeadDim] = l; xch[wq][kHeadDim + 1] = m; }
+  }
+  named_barrier_sync(2, kFWorkerWarps * 32);
+  if (r < 0 || sub != 0) return;
+  {
+    // the row's wpr warp results, merged in a fixed order
+    float mm = m;
+    for (int k = 1; k < wpr; ++k) mm = fmaxf(mm, xch[wq + k][kHeadDim + 1]);
+    const float s0 = (m == -INFINITY) ? 0.f : ex2_approx(m - mm);
+    acc.x *= s0; acc.y *= s0; acc.z *= s0; acc.w *= s0;
+    l *= s0;
+    for (int k = 1; k < wpr; ++k) {
+      const float mk = xch[wq + k][kHeadDim + 1];
+      const float sk = (mk == -INFINITY) ? 0.f : ex2_approx(mk - mm);
+      const float4 v = *reinterpret_cast<const float4*>(&xch[wq + k][lane * 4]);
+      acc.x = fmaf(v.x, sk, acc.x); acc.y = fmaf(v.y, sk, acc.y); acc.z = fmaf(v.z, sk, acc.z); acc.w = fmaf(v.w, sk, acc.w);
+      l = fmaf(xch[wq + k][kHeadDim], sk, l);
+    }
+    m = mm;
+  }
+  const float inv_l = 1.f / l;
+  const float4 o = make_float4(acc.x * inv_l, acc.y * inv_l, acc.z * inv_l, acc.w * inv_l);
+  const long long ri = (long long)bh * kRows + r;
+  *reinterpret_cast<float4*>(a.O_f32 + ri * kHeadDim + lane * 4) = o;
+  const __nv_bfloat16 b0 = __float2bfloat16_rn(o.x), b1 = __float2bfloat16_rn(o.y), b2 = __float2bfloat16_rn(o.z),
+                      b3 = __float2bfloat16_rn(o.w);
+  const float f0 = __bfloat162float(b0), f1 = __bfloat162float(b1), f2 = __bfloat162float(b2),
+              f3 = __bfloat162float(b3);
+  __nv_bfloat16* om = a.O_m2 + ri * kHeadDim + lane * 4;   // -2 x is exact for a bf16 x
+  om[0] = __float2bfloat16_rn(-2.f * f0);
+  om[1] = __float2bfloat16_rn(-2.f * f1);
+  om[2] = __float2bfloat16_rn(-2.f * f2);
+  om[3] = __float2bfloat16_rn(-2.f * f3);
+  float on = (f0 * f0 + f1 * f1) + (f2 * f2 + f3 * f3);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) on += __shfl_xor_sync(0xffffffffu, on, off);
+  __nv_bfloat16* arow = a.aug + ri * 64;
+  arow[2 * lane] = __float2bfloat16_rn(0.f);
+  arow[2 * lane + 1] = __float2bfloat16_rn(0.f);
+  __syncwarp();
+  if (lane == 0) {
+    const float c2 = a.scale * kLog2e;
+    const float M2 = m + log2f(l);        // A = exp2(s * c2 - M2)
+    split3(-M2 / c2, arow);
+    split3(on, arow + 16);
+  }
+}
+
+// One K tile and one V tile of phase C into stage s (ring slots 2s and 2s + 1).
+__device__ __forceinline__ void load_stage_c(const Ctx& cx, const CUtensorMap* tmK, const CUtensorMap* tmV, int b, int h,
+                                             int j0, int s) {
+  uint8_t* dK = cx.gen_base + k_slot_off(2 * s);
+  uint8_t* dV = dK + kTileBytes;
+  uint64_t* bar = &cx.B->kv_full[s];
+  mbar_arrive_expect_tx(bar, kStageBytes);
+  tma_load_4d(dK, tmK, bar, 0, j0, h, b);
+  tma_load_4d(dK + kBoxBytes, tmK, bar, 64, j0, h, b);
+  tma_load_4d(dV, tmV, bar, 0, j0, h, b);
+  tma_load_4d(dV + kBoxBytes, tmV, bar, 64, j0, h, b);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Phase C: this CTA's share [tile0, tile0 + T) of the scored rows of one head.  Warp 0 loads, warp 1 issues the
+// MMAs, the sixteen worker warps are four epilogue warpgroups (thread = token, warpgroup c = accumulator columns
+// [32c, 32c + 32)).  Q is still in shared memory from phase A.  The per-query-row constants ride through the
+// tensor core (one extra K = 16 step against a block of ones), so with u = exp2(-scale*log2e * S') = 1/A and
+// x = C' + ||v||^2 = ||o - v||^2 the indicator is x * rsqrt(x * (u - 1)^2).
+template <int kW>
+__device__ void phase_c(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tmO, const CUtensorMap* tmAug,
+                        const CUtensorMap* tmK, const CUtensorMap* tmV, int bh, int tile0, int T, int pre,
+                        float (*red)[4][kTile]) {
+  constexpr int kG = kRows / kW;
+  FusedBars* B = cx.B;
+  int* abort_flag = cx.abort_flag;
+  unsigned int* dev_status = a.dev_status;
+  const int b = bh / a.Hkv, h = bh % a.Hkv;
+  const int warp = cx.warp, lane = cx.lane;
+  const uint32_t tmem = cx.tmem;   // buffer s: S' at s*256, C' at s*256 + 128
+  const int n = a.n;
+
+  if (warp == 0) {
+    if (lane == 0 && T > 0) {
+      fence_proxy_async_all();   // O' and the constant strip were written with ordinary stores by other CTAs
+      mbar_arrive_expect_tx(&B->const_full, kTileBytes + kAugBytes);
+      tma_load_3d(cx.gen_base + kOffO, tmO, &B->const_full, 0, 0, bh);
+      tma_load_3d(cx.gen_base + kOffO + kBoxBytes, tmO, &B->const_full, 64, 0, bh);
+      tma_load_3d(cx.gen_base + kOffAug, tmAug, &B->const_full, 0, 0, bh);
+      for (int it = pre; it < T; ++it) {   // the first `pre` tiles were requested before the group barriers
+        const int s = it & 1;
+        if (it >= 2 && !mbar_wait(&B->kv_empty[s], ((it >> 1) - 1) & 1, abort_flag, dev_status, kDevTimeout)) break;
+        load_stage_c(cx, tmK, tmV, b, h, (tile0 + it) * kTile, s);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && T > 0) {
+      bool ok = mbar_wait(&B->const_full, 0, abort_flag, dev_status, kDevTimeout);
+      const uint32_t sQ = cx.smem_base + kOffQ, sO = cx.smem_base + kOffO, sAug = cx.smem_base + kOffAug;
+      const uint64_t ones_desc = make_smem_desc(cx.smem_base + kOffOnes, 16, 0);   // every 8-row group reads the same block
+      const uint64_t aug_s = kmajor_desc(sAug), aug_c = kmajor_desc(sAug + 32u);
+      for (int it = 0; ok && it < T; ++it) {
+        const int s = it & 1;
+        if (!mbar_wait(&B->kv_full[s], (it >> 1) & 1, abort_flag, dev_status, kDevTimeout)) break;
+        if (it >= 2 && !mbar_wait(&B->acc_empty[s], ((it >> 1) - 1) & 1, abort_flag, dev_status, kDevTimeout)) break;
+        tc_fence_after();
+        const uint32_t sK = cx.smem_base + k_slot_off(2 * s), sV = sK + kTileBytes;
+        const uint32_t tS = tmem + (uint32_t)s * 256u, tC = tS + 128u;
+        mma_tile_kk(tS, sK, sQ, false);                       // S^T = K Q^T
+        umma_ss(tS, ones_desc, aug_s, kIdescKK, true);        //   + row constant
+        mma_tile_kk(tC, sV, sO, false);                       // C^T = V (-2 O)^T
+        umma_ss(tC, ones_desc, aug_c, kIdescKK, true);        //   + ||o||^2
+        umma_commit(&B->acc_full[s]);
+        umma_commit(&B->kv_empty[s]);
+      }
+    }
+  } else if (warp >= kFFirstWorker) {
+    const int cgp = (warp - kFFirstWorker) >> 2;     // column group 0..3
+    const int quad = warp & 3;                       // TMEM lane quarter this warp may touch
+    const int t = quad * 32 + lane;
+    const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+    const float ema_decay = a.ema_decay;
+    const float neg_c2 = -a.scale * kLog2e;
+    const float heavy_thr = log2f(1.f / kHeavyA) / neg_c2;   // S' above this <=> A > kHeavyA
+    const float alpha = 1.f - ema_decay;                     // > 0 on this path
+    // Eq. 9 over a run of consecutive window positions i_a..i_b as a Horner chain H = sum c_i I_i decay^(i_b - i),
+    // c_0 = 1/alpha (the seed), c_i = 1: the run contributes alpha * decay^(w-1-i_b) * H.  Even and odd columns
+    // of a run are chained separately in decay^2 (one packed FMA per column pair): H = decay * H_even + H_odd.
+    constexpr int kRun = kW < 32 ? kW : 32;                  // columns of one run inside this warpgroup
+    const int i_first = (cgp * 32) % kW;
+    const float seed_coef = (i_first == 0) ? 1.f / alpha : 1.f;
+    const float fin_scale = alpha * powf(ema_decay, (float)(kW - 1 - (i_first + kRun - 1))) / (float)kG;
+    const f32x2 d2 = f2_make(ema_decay * ema_decay, ema_decay * ema_decay);
+    const f32x2 nc2 = f2_make(neg_c2, neg_c2), m1 = f2_make(-1.f, -1.f), tiny2 = f2_make(1e-36f, 1e-36f);
+    const f32x2 seed2 = f2_make(seed_coef, 1.f);
+    const float* O_head = a.O_f32 + (long long)bh * kRows * kHeadDim;
+    const __nv_bfloat16* V_head = a.V + (long long)b * a.vsb + (long long)h * a.vsh;
+    const float* vn_head = a.vnorm + (long long)bh * a.n_kv;
+    float* I_head = a.I_hat + (long long)bh * n;
+    bool ok = true;
+    const int nt_all = (a.n_kv + kTile - 1) / kTile;
+    const uint4* hv_head = reinterpret_cast<const uint4*>(a.heavy) + (long long)bh * nt_all;
+    float vn_next = 0.f;
+    uint4 hv_next = make_uint4(0, 0, 0, 0);
+    if (T > 0) {
+      const int j = tile0 * kTile + t;
+      vn_next = (j < n) ? vn_head[j] : 1.f;
+      hv_next = hv_head[tile0];
+    }
+
+    for (int it = 0; it < T; ++it) {
+      const int s = it & 1;
+      const uint32_t par = (uint32_t)(it >> 1) & 1u;
+      const float vn = vn_next;
+      const bool tile_heavy = (hv_next.x | hv_next.y | hv_next.z | hv_next.w) != 0;   // same for the whole CTA
+      if (it + 1 < T) {   // next tile's ||v||^2 and flags, well ahead of their use
+        const int jn = (tile0 + it + 1) * kTile + t;
+        vn_next = (jn < n) ? vn_head[jn] : 1.f;
+        hv_next = hv_head[tile0 + it + 1];
+      }
+      // The shares of the previous tile are summed in a fixed order by warpgroup 0 once all sixteen warps have
+      // stored theirs.  A slot of `red` is rewritten four tiles later, which the two accumulator buffers only
+      // allow after every warp has moved past this point.
+      if (it > 0 && cgp == 0) {
+        const int rs = (it - 1) & 3;
+        ok = ok && mbar_wait(&B->red_full[rs], (uint32_t)((it - 1) >> 2) & 1u, abort_flag, dev_status, kDevTimeout);
+        const int jp = (tile0 + it - 1) * kTile + t;
+        if (ok && jp < n) I_head[jp] = (red[rs][0][t] + red[rs][1][t]) + (red[rs][2][t] + red[rs][3][t]);
+      }
+      ok = ok && mbar_wait(&B->acc_full[s], par, abort_flag, dev_status, kDevTimeout);
+      float tot = 0.f;
+      if (ok) {
+        tc_fence_after();
+        const int j = (tile0 + it) * kTile + t;
+        const uint32_t tS = tmem + (uint32_t)s * 256u + lane_base + (uint32_t)cgp * 32u, tC = tS + 128u;
+        // ||o - v||^2 = C' + ||v||^2 is formed with ||v||^2 raised by 2^-16 of itself: a bias of ~1e-5 that keeps
+        // the sum positive when the expansion cancels, so that no clamp is needed.
+        const float vnb = vn * 1.0000152587890625f;
+        const f32x2 vn2 = f2_make(vnb, vnb);
+        f32x2 h2 = f2_make(0.f, 0.f);
+        if (!tile_heavy) {
+          float sv0[16], cv0[16], sv1[16], cv1[16];
+          tmem_ld16(tS, sv0);
+          tmem_ld16(tC, cv0);
+          tmem_wait_ld();
+          tmem_ld16(tS + 16, sv1);   // the second half of the columns travels while the first is worked on
+          tmem_ld16(tC + 16, cv1);
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+            const float* sv = c == 0 ? sv0 : sv1;
+            const float* cv = c == 0 ? cv0 : cv1;
+            if (c == 1) {
+              tmem_wait_ld();
+              // every tensor-memory read of this tile is done: the MMA warp may refill the accumulators
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(&B->acc_empty[s]);
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              const f32x2 nt = f2_mul(f2_make(sv[2 * q], sv[2 * q + 1]), nc2);
+              const f32x2 um = f2_add(f2_make(ex2_approx(f2_lo(nt)), ex2_approx(f2_hi(nt))), m1);   // 1/A - 1
+              const f32x2 x = f2_add(f2_make(cv[2 * q], cv[2 * q + 1]), vn2);                       // ||o - v||^2
+              const f32x2 bq = f2_fma(f2_mul(x, um), um, tiny2);                                    // x (1/A - 1)^2
+              f32x2 Iq = f2_mul(x, f2_make(rsqrt_approx(f2_lo(bq)), rsqrt_approx(f2_hi(bq))));
+              if (q == 0 && (c * 16) % kRun == 0) Iq = f2_mul(Iq, seed2);
+              h2 = f2_fma(h2, d2, Iq);
+            }
+            if ((c * 16 + 16) % kRun == 0) {   // end of a run
+              tot += fmaf(f2_lo(h2), ema_decay, f2_hi(h2));
+              h2 = f2_make(0.f, 0.f);
+            }
+          }
+        } else {
+          // rare: the tile may hold large attention weights; those entries take the exact distance
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            float sv[8], cv[8], I[8];
+            tmem_ld8(tS + c * 8, sv);
+            tmem_ld8(tC + c * 8, cv);
+            tmem_wait_ld();
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const float um = ex2_approx(sv[u] * neg_c2) - 1.f;
+              float x = cv[u] + vnb;
+              if (sv[u] > heavy_thr && j < n)
+                x = exact_dist2(O_head + (cgp * 32 + c * 8 + u) * kHeadDim, V_head + (long long)j * a.vsn);
+              I[u] = x * rsqrt_approx(fmaf(x * um, um, 1e-36f));
+            }
+            if ((c * 8) % kRun == 0) I[0] *= seed_coef;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) h2 = f2_fma(h2, d2, f2_make(I[2 * q], I[2 * q + 1]));
+            if ((c * 8 + 8) % kRun == 0) {   // end of a run
+              tot += fmaf(f2_lo(h2), ema_decay, f2_hi(h2));
+              h2 = f2_make(0.f, 0.f);
+            }
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&B->acc_empty[s]);
+        }
+      } else {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&B->acc_empty[s]);
+      }
+      red[it & 3][cgp][t] = tot * fin_scale;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&B->red_full[it & 3]);
+    }
+    if (T > 0 && cgp == 0) {
+      const int rs = (T - 1) & 3;
+      ok = ok && mbar_wait(&B->red_full[rs], (uint32_t)((T - 1) >> 2) & 1u, abort_flag, dev_status, kDevTimeout);
+      const int jl = (tile0 + T - 1) * kTile + t;
+      if (ok && jl < n) I_head[jl] = (red[rs][0][t] + red[rs][1][t]) + (red[rs][2][t] + red[rs][3][t]);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+template <int kW>
+__global__ void __launch_bounds__(kFThreads, 1)
+tc_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                const __grid_constant__ CUtensorMap tmAug, const FusedArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) FusedBars bars;
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  __shared__ float sm_stats[2 * kRows];
+  __shared__ float red[4][4][kTile];   // [tile & 3][warpgroup][token]: each warpgroup's share of the score
+
+  const int group = blockIdx.x / a.cpg, rank = blockIdx.x % a.cpg;
+  if (group >= a.groups) return;   // CTAs beyond groups * cpg have no work (uniform per CTA)
+
+  Ctx cx;
+  cx.smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  cx.gen_base = smem_raw + (cx.smem_base - smem_u32(smem_raw));
+  cx.B = &bars;
+  cx.abort_flag = &abort_flag;
+  cx.sm_stats = sm_stats;
+  cx.warp = threadIdx.x >> 5;
+  cx.lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    init_bars(&bars, true);
+    prefetch_tensormap(&tmQ);
+    prefetch_tensormap(&tmK);
+    prefetch_tensormap(&tmV);
+    prefetch_tensormap(&tmO);
+    prefetch_tensormap(&tmAug);
+  }
+  if (cx.warp == 1) {
+    tmem_alloc(&tmem_slot, 512);
+    tmem_relinquish();
+  }
+  if (threadIdx.x >= 128 && threadIdx.x < 128 + (int)(kOnesBytes / 4))   // the block of ones (bf16 1.0 = 0x3F80)
+    reinterpret_cast<uint32_t*>(cx.gen_base + kOffOnes)[threadIdx.x - 128] = 0x3F803F80u;
+  fence_proxy_async_smem();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  cx.tmem = tmem_slot;
+
+  // the same split of the token tiles in both phases (phase C covers only the scored rows)
+  const int nt1 = (a.n_kv + kTile - 1) / kTile, nt2 = (a.n + kTile - 1) / kTile;
+  const int per = (nt1 + a.cpg - 1) / a.cpg;
+  const int tile0 = rank * per;
+  const int T1 = max(0, min(nt1, tile0 + per) - tile0);
+  const int T2 = max(0, min(nt2, tile0 + per) - tile0);
+  unsigned int* counter = a.counters + group;
+  unsigned int epoch = 0;
+  bool alive = true;
+
+  for (int bh = group; bh < a.BH && alive; bh += a.groups) {
+    if (bh != group) {   // fresh barriers for every phase: nothing is in flight between two __syncthreads
+      if (threadIdx.x == 0) init_bars(&bars, false);
+      __syncthreads();
+    }
+    phase_a(cx, a, &tmQ, &tmK, &tmV, bh, rank, tile0, T1);
+    // Phase A no longer needs the tile ring: request phase C's first two K/V stages now, so that they arrive
+    // while the group merges its partials (K and V are inputs; only O' depends on the merge).
+    __syncthreads();
+    const int pre = T2 < 2 ? T2 : 2;
+    if (threadIdx.x == 0)
+      for (int it = 0; it < pre; ++it)
+        load_stage_c(cx, &tmK, &tmV, bh / a.Hkv, bh % a.Hkv, (tile0 + it) * kTile, it);
+    alive = group_barrier(counter, (++epoch) * (unsigned int)a.cpg, &abort_flag, a.dev_status);
+    if (!alive) break;
+    // ---- phase B: rows rank, rank + cpg, ... of the head; the sixteen worker warps share them ----
+    if (cx.warp >= kFFirstWorker) {
+      const int wq = cx.warp - kFFirstWorker;
+      const int rows_max = (kRows + a.cpg - 1) / a.cpg;          // rows of the busiest CTA of the group
+      int wpr = kFWorkerWarps;                                    // warps per row: 16, 8, 4, 2 or 1
+      while (wpr > 1 && kFWorkerWarps / wpr < rows_max) wpr >>= 1;
+      const int rows_at_once = kFWorkerWarps / wpr;
+      float (*xch)[kHeadDim + 4] = reinterpret_cast<float (*)[kHeadDim + 4]>(cx.gen_base + kOffAug);
+      for (int k0 = 0; k0 < rows_max; k0 += rows_at_once) {
+        const int r = rank + (k0 + wq / wpr) * a.cpg;
+        combine_rows(a, bh, group, r < kRows ? r : -1, wq % wpr, wpr, wq, cx.lane, xch);
+        named_barrier_sync(2, kFWorkerWarps * 32);   // the exchange buffer is reused by the next batch of rows
+      }
+      fence_proxy_async_smem();   // the exchange buffer is overwritten by a TMA load in phase C
+    }
+    alive = group_barrier(counter, (++epoch) * (unsigned int)a.cpg, &abort_flag, a.dev_status);
+    if (!alive) break;
+    tc_fence_after();
+    phase_c<kW>(cx, a, &tmO, &tmAug, &tmK, &tmV, bh, tile0, T2, pre, red);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (cx.warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(cx.tmem, 512);
+  }
+}
+
+}  // namespace
+
+// Number of CTA groups: as many heads in flight as fit a 72 MB share of L2 (phase C re-reads the head from there),
+// chosen to minimise rounds x tiles per CTA; ties go to more groups (fewer barrier rounds).
+void fused_plan(const Problem& p, int sm_count, int* groups, int* cpg) {
+  const long long head_bytes = 2ll * p.n_kv * p.d * 2;
+  long long limit = (72ll << 20) / (head_bytes > 0 ? head_bytes : 1);
+  if (limit < 1) limit = 1;
+  const int tiles = (p.n_kv + kTile - 1) / kTile;
+  int best_g = 1;
+  long long best_cost = -1;
+  for (int g = 1; g <= p.BH && g <= limit && g <= sm_count && g <= 256; ++g) {
+    const int c = sm_count / g;
+    const long long cost = (long long)((p.BH + g - 1) / g) * ((tiles + c - 1) / c);
+    if (best_cost < 0 || cost <= best_cost) { best_cost = cost; best_g = g; }
+  }
+  *groups = best_g;
+  *cpg = sm_count / best_g;
+}
+
+cudaError_t tc_fused_init() {
+  cudaError_t e = cudaFuncSetAttribute(tc_fused_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fused_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fused_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fused_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmem);
+  return e;
+}
+
+// One launch for pass 1, the merge and pass 2 of every head.  Cooperative launch: the CTAs of a group wait for one
+// another, so all of them must be resident.  ws.counters must be zero (the caller enqueues the memset).
+cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
+                            const void* V, float ema_decay, int sm_count, unsigned int* dev_status, cudaStream_t st) {
+  TcState* ts = (TcState*)state;
+  CUtensorMap tmQ, tmK, tmV, tmO, tmAug;
+  if (!make_rows_map(ts, &tmQ, Q, p.BH) || !make_rows_map(ts, &tmO, ws.O_m2, p.BH) ||
+      !make_aug_map(ts, &tmAug, ws.aug, p.BH) || !make_kv_map(ts, &tmK, K, p, p.ksb, p.ksh, p.ksn) ||
+      !make_kv_map(ts, &tmV, V, p, p.vsb, p.vsh, p.vsn))
+    return cudaErrorInvalidValue;
+  FusedArgs a{};
+  a.Hkv = p.Hkv; a.BH = p.BH; a.n = p.n; a.n_kv = p.n_kv; a.w = p.w;
+  a.scale = p.scale; a.ema_decay = ema_decay;
+  fused_plan(p, sm_count, &a.groups, &a.cpg);
+  a.part_m = ws.part_m; a.part_l = ws.part_l; a.part_O = ws.part_O;
+  a.O_f32 = ws.O_f32; a.O_m2 = ws.O_m2; a.aug = ws.aug; a.vnorm = ws.vnorm; a.I_hat = ws.I_hat;
+  a.V = (const __nv_bfloat16*)V; a.vsb = p.vsb; a.vsh = p.vsh; a.vsn = p.vsn;
+  a.counters = ws.counters; a.heavy = ws.heavy; a.dev_status = dev_status;
+  cudaError_t e = cudaMemsetAsync(ws.counters, 0, 1024, st);
+  if (e != cudaSuccess) return e;
+  void* args[] = {&tmQ, &tmK, &tmV, &tmO, &tmAug, &a};
+  const dim3 grid(a.groups * a.cpg), block(kFThreads);
+  switch (p.w) {
+    case 16: return cudaLaunchCooperativeKernel((void*)tc_fused_kernel<16>, grid, block, args, kFSmem, st);
+    case 32: return cudaLaunchCooperativeKernel((void*)tc_fused_kernel<32>, grid, block, args, kFSmem, st);
+    case 64: return cudaLaunchCooperativeKernel((void*)tc_fused_kernel<64>, grid, block, args, kFSmem, st);
+    case 128: return cudaLaunchCooperativeKernel((void*)tc_fused_kernel<128>, grid, block, args, kFSmem, st);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+}  // namespace restkv

@@ -91,7 +91,7 @@ def test_config1_adaptive_window(handle, tail):
 
 
 # ------------------------------------------------------------------ config 2 (8B-shaped layer)
-@pytest.mark.parametrize("path", [rk.PATH_AUTO, rk.PATH_SIMT])
+@pytest.mark.parametrize("path", [rk.PATH_AUTO, rk.PATH_SIMT, rk.PATH_HEAD_SEQUENTIAL])
 def test_config2(handle, path):
     inp = make_inputs(CONFIGS["cfg2"])
     worst, exact = full_check(handle, inp, path=path)
@@ -103,8 +103,29 @@ def test_config2(handle, path):
     assert recall > 0.9
 
 
-def test_config2_causal_tail(handle):
-    full_check(handle, make_inputs(CONFIGS["cfg2"].with_(causal_tail=32)))
+@pytest.mark.parametrize("path", [rk.PATH_AUTO, rk.PATH_HEAD_SEQUENTIAL])
+def test_config2_causal_tail(handle, path):
+    full_check(handle, make_inputs(CONFIGS["cfg2"].with_(causal_tail=32)), path=path)
+
+
+@pytest.mark.parametrize("spec", [(2, 8, 2, 1000, 32, 0), (1, 8, 1, 700, 16, 0), (2, 4, 1, 4097, 32, 32), (3, 4, 1, 129, 32, 0)])
+def test_head_sequential_kernel_on_ragged_shapes(handle, spec):
+    b, Hq, Hkv, n, w, tail = spec
+    case = Case("headseq", b, Hq, Hkv, 128, n, w, 64, 5, 0, 0.8, "bf16", tail, "normal", 91)
+    full_check(handle, make_inputs(case), path=rk.PATH_HEAD_SEQUENTIAL)
+
+
+def test_head_sequential_kernel_at_full_size(handle):
+    inp = make_inputs(CONFIGS["cfg4"])
+    run = GpuRun(handle, inp)
+    ref = run.score().copy()                      # default tensor-core kernels, checked against the oracle elsewhere
+    handle.set_kernel_path(rk.PATH_HEAD_SEQUENTIAL)
+    try:
+        got = run.score()
+    finally:
+        handle.set_kernel_path(rk.PATH_AUTO)
+    assert handle.poll_status() == rk.RESTKV_OK
+    np.testing.assert_allclose(got, ref, rtol=1e-3, atol=0)
 
 
 def test_config2_is_deterministic(handle):
