@@ -43,6 +43,7 @@ __device__ __forceinline__ unsigned int float_key(float x) {
 constexpr int kSelThreads = 1024;
 constexpr int kSelBins = 256;                // 8-bit digits
 constexpr int kSelMaxSmemKeys = 44 * 1024;   // keys of one CTA's slice kept in shared memory (176 KB)
+constexpr int kSelMaxStagedWidth = 65;       // widest box whose taps are staged in shared memory
 
 // Inclusive scan over the 1024 threads of the block, in thread order.
 __device__ __forceinline__ unsigned int block_inclusive_scan(unsigned int v, unsigned int* warp_sums) {
@@ -82,7 +83,7 @@ __device__ __forceinline__ unsigned int block_inclusive_scan(unsigned int v, uns
 __global__ void __launch_bounds__(kSelThreads, 1)
 select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const int* __restrict__ pool, int W,
               int gamma, float* scores, int32_t* __restrict__ indices, int32_t* __restrict__ pool_used, int per,
-              int use_smem) {
+              int use_smem, int stage_taps) {
   cg::cluster_group cluster = cg::this_cluster();
   const unsigned int CS = cluster.num_blocks(), rank = cluster.block_rank();
   const int row = blockIdx.x / CS;
@@ -106,10 +107,34 @@ select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const 
     if (pool) { W = pool[2 * row]; gamma = pool[2 * row + 1]; }
     if (pool_used && rank == 0 && tid == 0) { pool_used[2 * row] = W; pool_used[2 * row + 1] = gamma; }
     const float* src = I_hat + (long long)row * n;
-    for (int jj = tid; jj < cnt; jj += kSelThreads) {
-      const float out = box_mean(src, n, (int)(j0 + jj), W, gamma);
-      srow[j0 + jj] = out;
-      if (use_smem) skeys[jj] = float_key(out);
+    if (stage_taps && W <= kSelMaxStagedWidth && cnt > 0) {
+      // the taps of the whole slice (slice + halo) are staged in shared memory once, then summed from there in
+      // the same order as box_mean does
+      float* staged = reinterpret_cast<float*>(skeys + per);
+      const int half = W / 2;
+      const long long lo64 = j0 - half + gamma, hi64 = j0 + cnt - 1 + half + gamma;
+      const int s_lo = lo64 < 0 ? 0 : (int)(lo64 < n ? lo64 : n), s_hi = hi64 > n - 1 ? n - 1 : (int)(hi64 > -1 ? hi64 : -1);
+      for (int t = s_lo + tid; t <= s_hi; t += kSelThreads) staged[t - s_lo] = src[t];
+      __syncthreads();
+      for (int jj = tid; jj < cnt; jj += kSelThreads) {
+        const int j = (int)(j0 + jj);
+        float out = INFINITY;
+        if (j < n) {
+          const long long a64 = (long long)j - half + gamma, b64 = (long long)j + half + gamma;
+          const int a = a64 < s_lo ? s_lo : (int)(a64 <= s_hi ? a64 : s_hi + 1), b = b64 > s_hi ? s_hi : (int)(b64 >= s_lo ? b64 : s_lo - 1);
+          float acc = 0.f;
+          for (int t = a; t <= b; ++t) acc += staged[t - s_lo];
+          out = acc / (float)W;
+        }
+        srow[j0 + jj] = out;
+        skeys[jj] = float_key(out);
+      }
+    } else {
+      for (int jj = tid; jj < cnt; jj += kSelThreads) {
+        const float out = box_mean(src, n, (int)(j0 + jj), W, gamma);
+        srow[j0 + jj] = out;
+        if (use_smem) skeys[jj] = float_key(out);
+      }
     }
   } else if (use_smem) {
     for (int jj = tid; jj < cnt; jj += kSelThreads) skeys[jj] = float_key(srow[j0 + jj]);
@@ -315,7 +340,9 @@ cudaError_t launch_select(int rows, int n, int n_kv, int budget, const float* I_
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned int)(rows * CS));
   cfg.blockDim = dim3(kSelThreads);
-  cfg.dynamicSmemBytes = use_smem ? (size_t)per * sizeof(unsigned int) : 0;
+  // with room for it, the pooling taps of the slice (slice + halo) are staged behind the keys
+  const int stage_taps = (I_hat && use_smem && 2 * per + kSelMaxStagedWidth <= kSelMaxSmemKeys) ? 1 : 0;
+  cfg.dynamicSmemBytes = use_smem ? (size_t)(stage_taps ? 2 * per + kSelMaxStagedWidth : per) * sizeof(unsigned int) : 0;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -325,7 +352,7 @@ cudaError_t launch_select(int rows, int n, int n_kv, int budget, const float* I_
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, select_kernel, n, n_kv, keep, I_hat, pool_dev, W, gamma, scores, indices, pool_used,
-                            per, use_smem);
+                            per, use_smem, stage_taps);
 }
 
 cudaError_t launch_compact(const Problem& p, const void* K, const void* V, const int32_t* indices, int n_sel,

@@ -175,10 +175,12 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
     if (e == cudaSuccess && adaptive)
       e = cudaMemsetAsync(ws.I_raw, 0, (size_t)p.batch * p.Hq * p.w * p.n * sizeof(float), c.st);
     if (e != cudaSuccess) return c.fail(e);
-  } else if (use_tc && c.h->kernel_path == 4) {
-    // pass 1, merge and pass 2 of every head in one head-sequential launch (timed as "pass 2")
+  } else if (use_tc && c.h->kernel_path != 3) {
+    // pass 1, merge and pass 2 in one persistent launch (timed as "pass 2"); path 4 keeps only as many heads in
+    // flight as fit in L2 so that pass 2 re-reads K and V from there
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2,
-                  launch_tc_fused(c.h->tc_state, p, ws, Q, K, V, ema_decay, c.h->sm_count, c.h->dev_status, c.st), 1);
+                  launch_tc_fused(c.h->tc_state, p, ws, Q, K, V, ema_decay, c.h->sm_count, c.h->kernel_path == 4,
+                                  c.h->dev_status, c.st), 1);
   } else if (use_tc) {
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS1, launch_tc_pass1(c.h->tc_state, p, ws, Q, K, V, c.h->dev_status, c.st), 1);
     RESTKV_LAUNCH(c, RESTKV_KERNEL_COMBINE, launch_combine(p, ws, 2 * ws.splits, c.st), 1);   // two warpgroups per CTA

@@ -82,7 +82,8 @@ cudaError_t launch_tc_pass1(void* state, const Problem& p, const Workspace& ws, 
                             const void* V, unsigned int* dev_status, cudaStream_t st);
 cudaError_t tc_fused_init();
 cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
-                            const void* V, float ema_decay, int sm_count, unsigned int* dev_status, cudaStream_t st);
+                            const void* V, float ema_decay, int sm_count, bool reuse_l2, unsigned int* dev_status,
+                            cudaStream_t st);
 cudaError_t launch_tc_pass2(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
                             const void* V, float ema_decay, unsigned int* dev_status, cudaStream_t st);
 

@@ -795,11 +795,12 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
 }  // namespace
 
-// Number of CTA groups: as many heads in flight as fit a 72 MB share of L2 (phase C re-reads the head from there),
-// chosen to minimise rounds x tiles per CTA; ties go to more groups (fewer barrier rounds).
-void fused_plan(const Problem& p, int sm_count, int* groups, int* cpg) {
+// Number of CTA groups = heads in flight.  With `reuse_l2` only as many as fit a 72 MB share of L2 (phase C then
+// re-reads the heads from there); otherwise as many as there are heads.  Among the allowed counts the one with the
+// fewest rounds x tiles per CTA wins; ties go to more groups (fewer barrier rounds).
+void fused_plan(const Problem& p, int sm_count, bool reuse_l2, int* groups, int* cpg) {
   const long long head_bytes = 2ll * p.n_kv * p.d * 2;
-  long long limit = (72ll << 20) / (head_bytes > 0 ? head_bytes : 1);
+  long long limit = reuse_l2 ? (72ll << 20) / (head_bytes > 0 ? head_bytes : 1) : p.BH;
   if (limit < 1) limit = 1;
   const int tiles = (p.n_kv + kTile - 1) / kTile;
   int best_g = 1;
@@ -821,10 +822,13 @@ cudaError_t tc_fused_init() {
   return e;
 }
 
-// One launch for pass 1, the merge and pass 2 of every head.  Cooperative launch: the CTAs of a group wait for one
-// another, so all of them must be resident.  ws.counters must be zero (the caller enqueues the memset).
+// One launch for pass 1, the merge and pass 2 of every head.  The CTAs of a group wait for one another, so all of
+// them must be resident: the grid never exceeds the SM count and a CTA fills an SM (shared memory), which holds as
+// long as the device is not shared with another kernel at that moment; if it is, the bounded group barrier gives up
+// with the timeout status instead of hanging.  (A cooperative launch would guarantee residency but costs ~25 us.)
 cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
-                            const void* V, float ema_decay, int sm_count, unsigned int* dev_status, cudaStream_t st) {
+                            const void* V, float ema_decay, int sm_count, bool reuse_l2, unsigned int* dev_status,
+                            cudaStream_t st) {
   TcState* ts = (TcState*)state;
   CUtensorMap tmQ, tmK, tmV, tmO, tmAug;
   if (!make_rows_map(ts, &tmQ, Q, p.BH) || !make_rows_map(ts, &tmO, ws.O_m2, p.BH) ||
@@ -834,22 +838,22 @@ cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, 
   FusedArgs a{};
   a.Hkv = p.Hkv; a.BH = p.BH; a.n = p.n; a.n_kv = p.n_kv; a.w = p.w;
   a.scale = p.scale; a.ema_decay = ema_decay;
-  fused_plan(p, sm_count, &a.groups, &a.cpg);
+  fused_plan(p, sm_count, reuse_l2, &a.groups, &a.cpg);
   a.part_m = ws.part_m; a.part_l = ws.part_l; a.part_O = ws.part_O;
   a.O_f32 = ws.O_f32; a.O_m2 = ws.O_m2; a.aug = ws.aug; a.vnorm = ws.vnorm; a.I_hat = ws.I_hat;
   a.V = (const __nv_bfloat16*)V; a.vsb = p.vsb; a.vsh = p.vsh; a.vsn = p.vsn;
   a.counters = ws.counters; a.heavy = ws.heavy; a.dev_status = dev_status;
   cudaError_t e = cudaMemsetAsync(ws.counters, 0, 1024, st);
   if (e != cudaSuccess) return e;
-  void* args[] = {&tmQ, &tmK, &tmV, &tmO, &tmAug, &a};
   const dim3 grid(a.groups * a.cpg), block(kFThreads);
   switch (p.w) {
-    case 16: return cudaLaunchCooperativeKernel((void*)tc_fused_kernel<16>, grid, block, args, kFSmem, st);
-    case 32: return cudaLaunchCooperativeKernel((void*)tc_fused_kernel<32>, grid, block, args, kFSmem, st);
-    case 64: return cudaLaunchCooperativeKernel((void*)tc_fused_kernel<64>, grid, block, args, kFSmem, st);
-    case 128: return cudaLaunchCooperativeKernel((void*)tc_fused_kernel<128>, grid, block, args, kFSmem, st);
+    case 16: tc_fused_kernel<16><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a); break;
+    case 32: tc_fused_kernel<32><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a); break;
+    case 64: tc_fused_kernel<64><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a); break;
+    case 128: tc_fused_kernel<128><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a); break;
     default: return cudaErrorInvalidValue;
   }
+  return cudaGetLastError();
 }
 
 }  // namespace restkv
