@@ -207,11 +207,11 @@ typedef enum {
 } restkv_kernel_id;
 restkv_status restkv_set_profile_events(restkv_handle* h, int which, void* start, void* stop);
 
-/* Kernel choice: 0 = automatic, 1 = force the fp32 SIMT kernels, 2 or 3 = require the tensor-core kernels (pass 1
- * and pass 2 as separate launches over all heads; what 0 picks when the shape qualifies), 4 = require the
- * head-sequential tensor-core kernel: one persistent launch that runs pass 1, the merge and pass 2 of one head
- * back to back so that pass 2 reads the head's K and V from L2 (needs a cooperative launch; it halves the DRAM
- * reads but pays two grid barriers per head, and is the slower of the two on today's shapes). */
+/* Kernel choice: 0 = automatic, 1 = force the fp32 SIMT kernels, 2 = require the tensor-core kernel (one persistent
+ * launch that runs pass 1, the merge of the partial softmax results and pass 2 with every head in flight; what 0
+ * picks when the shape qualifies), 3 = require the tensor-core kernel in its head-sequential form: only as many
+ * heads in flight as fit in L2, so that pass 2 re-reads K and V from there (half the DRAM reads, but two grid
+ * barriers per head; the slower of the two on today's shapes). */
 restkv_status restkv_set_kernel_path(restkv_handle* h, int path);
 
 #ifdef __cplusplus

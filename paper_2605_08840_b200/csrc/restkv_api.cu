@@ -49,15 +49,14 @@ size_t plan_workspace(const Problem& p, int budget, int sm_count, bool adaptive,
   Workspace w{};
   w.splits = pass1_splits(p, sm_count);
   const size_t BH = (size_t)p.BH, R = (size_t)p.R, d = (size_t)p.d;
-  w.parts = w.splits;
-  // partial slots: two per (head, split) for the two-kernel paths, one per CTA for the head-sequential kernel
-  size_t slots = BH * 2 * w.splits;
+  // partial slots: one per (head, split) on the SIMT path, one per CTA in the persistent tensor-core kernel
+  size_t slots = BH * w.splits;
   if (slots < (size_t)sm_count) slots = (size_t)sm_count;
   w.part_m = (float*)take(slots * R * sizeof(float));
   w.part_l = (float*)take(slots * R * sizeof(float));
   w.part_O = (float*)take(slots * R * d * sizeof(float));
   w.counters = (unsigned int*)take(1024);
-  w.heavy = (unsigned int*)take(BH * (size_t)((p.n_kv + 127) / 128) * 4 * sizeof(unsigned int));
+  w.heavy = (unsigned int*)take(BH * (size_t)((p.n_kv + 127) / 128) * 8 * sizeof(unsigned int));
   w.vnorm = (float*)take(BH * (size_t)p.n_kv * sizeof(float));
   w.fin_m = (float*)take(BH * R * sizeof(float));
   w.fin_l = (float*)take(BH * R * sizeof(float));
@@ -175,19 +174,15 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
     if (e == cudaSuccess && adaptive)
       e = cudaMemsetAsync(ws.I_raw, 0, (size_t)p.batch * p.Hq * p.w * p.n * sizeof(float), c.st);
     if (e != cudaSuccess) return c.fail(e);
-  } else if (use_tc && c.h->kernel_path != 3) {
-    // pass 1, merge and pass 2 in one persistent launch (timed as "pass 2"); path 4 keeps only as many heads in
+  } else if (use_tc) {
+    // pass 1, merge and pass 2 in one persistent launch (timed as "pass 2"); path 3 keeps only as many heads in
     // flight as fit in L2 so that pass 2 re-reads K and V from there
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2,
-                  launch_tc_fused(c.h->tc_state, p, ws, Q, K, V, ema_decay, c.h->sm_count, c.h->kernel_path == 4,
+                  launch_tc_fused(c.h->tc_state, p, ws, Q, K, V, ema_decay, c.h->sm_count, c.h->kernel_path == 3,
                                   c.h->dev_status, c.st), 1);
-  } else if (use_tc) {
-    RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS1, launch_tc_pass1(c.h->tc_state, p, ws, Q, K, V, c.h->dev_status, c.st), 1);
-    RESTKV_LAUNCH(c, RESTKV_KERNEL_COMBINE, launch_combine(p, ws, 2 * ws.splits, c.st), 1);   // two warpgroups per CTA
-    RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2, launch_tc_pass2(c.h->tc_state, p, ws, Q, K, V, ema_decay, c.h->dev_status, c.st), 1);
   } else {
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS1, launch_simt_pass1(p, ws, Q, K, V, c.st), 1);
-    RESTKV_LAUNCH(c, RESTKV_KERNEL_COMBINE, launch_combine(p, ws, ws.splits, c.st), 1);
+    RESTKV_LAUNCH(c, RESTKV_KERNEL_COMBINE, launch_combine(p, ws, c.st), 1);
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2, launch_simt_pass2(p, ws, Q, K, V, ema_decay, adaptive ? ws.I_raw : nullptr, c.st), 1);
   }
   if (adaptive) {
@@ -437,7 +432,7 @@ restkv_status restkv_set_profile_events(restkv_handle* h, int which, void* start
 }
 
 restkv_status restkv_set_kernel_path(restkv_handle* h, int path) {
-  if (!h || path < 0 || path > 4) return RESTKV_ERR_INVALID_ARG;
+  if (!h || path < 0 || path > 3) return RESTKV_ERR_INVALID_ARG;
   h->kernel_path = path;
   return RESTKV_OK;
 }

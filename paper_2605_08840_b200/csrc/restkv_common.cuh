@@ -29,13 +29,12 @@ struct Problem {
 // Workspace carve-up (all offsets 256-byte aligned).
 struct Workspace {
   int splits;             // token splits (CTAs) of the score passes per (batch, KV head)
-  int parts;              // partials per (batch, KV head) that pass 1 writes and combine merges
-  float* part_m;          // [BH, parts, R]   (room for 2 * splits)
-  float* part_l;          // [BH, parts, R]
-  float* part_O;          // [BH, parts, R, d]
+  float* part_m;          // [slots, R]     partial softmax results: one slot per (head, split) on the SIMT path,
+  float* part_l;          // [slots, R]      one per CTA in the persistent tensor-core kernel
+  float* part_O;          // [slots, R, d]
   float* vnorm;           // [BH, n_kv]  ||v_j||^2 (tensor-core path)
   unsigned int* counters; // [256] group barrier counters of the head-sequential kernel
-  unsigned int* heavy;    // [BH, tiles, 4] per-tile flags of the head-sequential kernel
+  unsigned int* heavy;    // [BH, tiles, 8] per-tile flags of the persistent score kernel
   float* fin_m;           // [BH, R]    row max of the scaled logits (natural units)
   float* fin_l;           // [BH, R]    sum of exp(s - m)
   float* O_f32;           // [BH, R, d]
@@ -61,7 +60,7 @@ size_t plan_workspace(const Problem& p, int budget, int sm_count, bool adaptive,
 // ---- launches (each returns the cudaError_t of the launch) -------------------------------------
 cudaError_t launch_simt_pass1(const Problem& p, const Workspace& ws, const void* Q, const void* K, const void* V,
                               cudaStream_t st);
-cudaError_t launch_combine(const Problem& p, const Workspace& ws, int parts, cudaStream_t st);
+cudaError_t launch_combine(const Problem& p, const Workspace& ws, cudaStream_t st);
 cudaError_t launch_simt_pass2(const Problem& p, const Workspace& ws, const void* Q, const void* K, const void* V,
                               float ema_decay, float* I_raw, cudaStream_t st);
 cudaError_t launch_pool(const Problem& p, const Workspace& ws, const int* pool_dev, int W, int gamma, float* scores,
@@ -78,14 +77,10 @@ cudaError_t launch_adaptive_params(const Problem& p, const Workspace& ws, int bu
 // Tensor-core (tcgen05 / TMEM / TMA) score kernels.  `supported` says whether the shape qualifies.
 bool tc_supported(const Problem& p);
 cudaError_t tc_init(void** state);   // resolves the driver entry point for tensor-map encoding
-cudaError_t launch_tc_pass1(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
-                            const void* V, unsigned int* dev_status, cudaStream_t st);
 cudaError_t tc_fused_init();
 cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
                             const void* V, float ema_decay, int sm_count, bool reuse_l2, unsigned int* dev_status,
                             cudaStream_t st);
-cudaError_t launch_tc_pass2(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
-                            const void* V, float ema_decay, unsigned int* dev_status, cudaStream_t st);
 
 // ---- small device helpers ------------------------------------------------------------------------
 template <typename T> __device__ __forceinline__ float to_f32(T x);

@@ -116,26 +116,10 @@ __global__ void simt_pass1_kernel(Problem p, const T* __restrict__ Q, const T* _
 }
 
 // ------------------------------------------------------------------------------------------------
-// x = hi + mid + lo with three bf16 pieces (24 significant bits): lets an fp32 constant ride through a
-// bf16 tensor-core contraction against a column of ones.
-__device__ __forceinline__ void split3_bf16(float x, __nv_bfloat16* out) {
-  const __nv_bfloat16 hi = __float2bfloat16_rn(x);
-  const float r1 = x - __bfloat162float(hi);
-  const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
-  const float r2 = r1 - __bfloat162float(mid);
-  out[0] = hi;
-  out[1] = mid;
-  out[2] = __float2bfloat16_rn(r2);
-}
-
 // Combine the token splits.  grid (R, BH), block 128: one block per query row.
-// Besides the final (m, l, O) it prepares what the tensor-core pass 2 consumes: O_m2 = -2 * bf16(O) and, per
-// row, a 64-column bf16 strip `aug` whose columns 0-2 hold the pieces of -(m*log2e + log2 l) / (scale*log2e)
-// and columns 16-18 the pieces of ||bf16(O)||^2 (all other columns zero).
-__global__ void combine_kernel(int R, int d, int splits, float scale, const float* __restrict__ part_m,
+__global__ void combine_kernel(int R, int d, int splits, const float* __restrict__ part_m,
                                const float* __restrict__ part_l, const float* __restrict__ part_O,
-                               float* __restrict__ fin_m, float* __restrict__ fin_l, float* __restrict__ O_f32,
-                               __nv_bfloat16* __restrict__ O_m2, __nv_bfloat16* __restrict__ aug) {
+                               float* __restrict__ fin_m, float* __restrict__ fin_l, float* __restrict__ O_f32) {
   const int r = blockIdx.x, bh = blockIdx.y;
   const long long base = (long long)bh * splits * R + r;   // + s * R
   float m = -INFINITY;
@@ -146,37 +130,17 @@ __global__ void combine_kernel(int R, int d, int splits, float scale, const floa
     if (ms != -INFINITY) l += part_l[base + (long long)s * R] * expf(ms - m);
   }
   const float inv_l = 1.f / l;
-  float on = 0.f;
   for (int k = threadIdx.x; k < d; k += blockDim.x) {
     float acc = 0.f;
     for (int s = 0; s < splits; ++s) {
       const float ms = part_m[base + (long long)s * R];
       if (ms != -INFINITY) acc += part_O[(base + (long long)s * R) * d + k] * expf(ms - m);
     }
-    const float o = acc * inv_l;
-    const long long oi = ((long long)bh * R + r) * d + k;
-    O_f32[oi] = o;
-    const float of = __bfloat162float(__float2bfloat16_rn(o));
-    O_m2[oi] = __float2bfloat16_rn(-2.f * of);   // exact: a power-of-two multiple of a bf16 value
-    on += of * of;
+    O_f32[((long long)bh * R + r) * d + k] = acc * inv_l;
   }
-  const long long ri = (long long)bh * R + r;
-  __nv_bfloat16* arow = aug + ri * 64;
-  if (threadIdx.x < 64) arow[threadIdx.x] = __float2bfloat16_rn(0.f);
-  // block reduction of the squared norm
-  __shared__ float red[32];
-  for (int off = 16; off > 0; off >>= 1) on += __shfl_xor_sync(0xffffffffu, on, off);
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = on;
-  __syncthreads();
   if (threadIdx.x == 0) {
-    float tot = 0.f;
-    for (int wv = 0; wv < (int)(blockDim.x >> 5); ++wv) tot += red[wv];
-    fin_m[ri] = m;
-    fin_l[ri] = l;
-    const float c2 = scale * 1.4426950408889634f;
-    const float M2 = m * 1.4426950408889634f + log2f(l);   // A = exp2(s * c2 - M2)
-    split3_bf16(-M2 / c2, arow);
-    split3_bf16(tot, arow + 16);
+    fin_m[(long long)bh * R + r] = m;
+    fin_l[(long long)bh * R + r] = l;
   }
 }
 
@@ -273,10 +237,10 @@ cudaError_t launch_simt_pass1(const Problem& p, const Workspace& ws, const void*
   return cudaGetLastError();
 }
 
-cudaError_t launch_combine(const Problem& p, const Workspace& ws, int parts, cudaStream_t st) {
+cudaError_t launch_combine(const Problem& p, const Workspace& ws, cudaStream_t st) {
   dim3 grid(p.R, p.BH);
-  combine_kernel<<<grid, 128, 0, st>>>(p.R, p.d, parts, p.scale, ws.part_m, ws.part_l, ws.part_O, ws.fin_m,
-                                       ws.fin_l, ws.O_f32, ws.O_m2, ws.aug);
+  combine_kernel<<<grid, 128, 0, st>>>(p.R, p.d, ws.splits, ws.part_m, ws.part_l, ws.part_O, ws.fin_m, ws.fin_l,
+                                       ws.O_f32);
   return cudaGetLastError();
 }
 

@@ -18,7 +18,8 @@ namespace {
 
 constexpr int kFFirstWorker = 2;                  // warp 0: TMA producer, warp 1: MMA issuer
 constexpr int kFWorkerWarps = 16;                 // warps 2..17
-constexpr int kFThreads = (kFFirstWorker + kFWorkerWarps) * 32;
+constexpr int kFNormWarps = 2;                    // warps 18, 19: ||v||^2 of the tokens during phase A
+constexpr int kFThreads = (kFFirstWorker + kFWorkerWarps + kFNormWarps) * 32;
 constexpr int kFRing = 4;                         // 32 KB tile slots after Q | O' | aug | ones
 constexpr size_t kFSmem = 2 * kTileBytes + kAugBytes + kOnesBytes + kFRing * kTileBytes + 1024;
 constexpr int kFVSlots = 3;                       // phase A: V slots = ring 2, ring 3 and the (then unused) O' tile
@@ -34,7 +35,7 @@ struct FusedArgs {
   __nv_bfloat16* O_m2;               // [BH, 128, 128]  -2 * bf16(O)
   __nv_bfloat16* aug;                // [BH, 128, 64]
   float* vnorm;                      // [BH, n_kv]
-  unsigned int* heavy;               // [BH, tiles]: bit per softmax warp, set if the tile may hold a weight > kHeavyA
+  unsigned int* heavy;               // [BH, tiles, 8]: one word per softmax warp, set if the tile may hold a weight > kHeavyA
   float* I_hat;                      // [BH, n]
   const __nv_bfloat16* V;
   long long vsb, vsh, vsn;
@@ -73,7 +74,7 @@ __device__ void init_bars(FusedBars* B, bool first) {
     mbar_init(&B->k_full[i], 1);
     mbar_init(&B->k_empty[i], 1);
     mbar_init(&B->s_full[i], 1);
-    mbar_init(&B->p_full[i], 128);
+    mbar_init(&B->p_full[i], 256);
     mbar_init(&B->pv_done[i], 1);
     mbar_init(&B->kv_full[i], 1);
     mbar_init(&B->kv_empty[i], 1);
@@ -82,7 +83,7 @@ __device__ void init_bars(FusedBars* B, bool first) {
   }
   for (int i = 0; i < kFVSlots; ++i) {
     mbar_init(&B->v_full[i], 1);
-    mbar_init(&B->v_empty[i], 1 + 4);   // MMA commit + the four warps that reduce ||v||^2
+    mbar_init(&B->v_empty[i], 1 + 1);   // MMA commit + the warp that reduces ||v||^2
   }
   mbar_init(&B->const_full, 1);
   for (int i = 0; i < 4; ++i) mbar_init(&B->red_full[i], kFWorkerWarps);
@@ -116,7 +117,7 @@ struct Ctx {
   uint32_t tmem;
   FusedBars* B;
   int* abort_flag;
-  float* sm_stats;         // [2][128] floats: (m, l) of warpgroup 1 for the in-CTA merge
+  float* sm_stats;         // [6][128] floats: row maxima of the column halves [slot][half], then (m, l) hand-over
   int warp, lane;
 };
 
@@ -186,7 +187,9 @@ __device__ void phase_a(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tm
 #pragma unroll
           for (int k = 0; k < 8; ++k) {
             const uint64_t bdesc = make_smem_desc(vaddr + (uint32_t)k * 2048u, kBoxBytes, 1024);
-            umma_ts(tmem + 256u + (uint32_t)g * 128u, tmem + (uint32_t)g * 128u + (uint32_t)k * 8u, bdesc, kIdescKMN,
+            // tokens 0-63 of P_g sit in columns [0, 32) of S_g, tokens 64-127 in columns [64, 96)
+            const uint32_t pcol = (uint32_t)(k < 4 ? k * 8 : 64 + (k - 4) * 8);
+            umma_ts(tmem + 256u + (uint32_t)g * 128u, tmem + (uint32_t)g * 128u + pcol, bdesc, kIdescKMN,
                     pt >= 2 || k > 0);
           }
           umma_commit(&B->pv_done[g]);
@@ -194,60 +197,72 @@ __device__ void phase_a(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tm
         }
       }
     }
-  } else if (warp >= kFFirstWorker + 8) {
-    // ---------------- ||v||^2: worker warpgroup 2 takes the even tiles, 3 the odd ones ----------------
-    const int vg = (warp - kFFirstWorker - 8) >> 2;
-    const int row = ((warp - kFFirstWorker - 8) & 3) * 32 + lane;
+  } else if (warp >= kFFirstWorker + kFWorkerWarps) {
+    // ---------------- ||v||^2: one warp takes the even tiles, the other the odd ones; lane = 4 tokens ----------------
+    const int vg = warp - (kFFirstWorker + kFWorkerWarps);
     bool ok = true;
     for (int it = 0; it < T && ok; ++it) {
       const int vs = it % kFVSlots;
-      // both warpgroups wait for every tile so that neither falls a whole phase behind a slot's barrier
+      // both warps wait for every tile so that neither falls a whole phase behind a slot's barrier
       ok = mbar_wait(&B->v_full[vs], (it / kFVSlots) & 1, abort_flag, dev_status, kDevTimeout);
       if (!ok || (it & 1) != vg) continue;
-      // 16-byte chunk c of row r of a 128-byte-swizzled box sits at chunk c ^ (r & 7)
       const uint8_t* vt = cx.gen_base + v_slot_off(vs);
-      float2 acc = make_float2(0.f, 0.f);
+      float vn[4];
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        const uint8_t* rowp = vt + half * kBoxBytes + (row >> 3) * 1024 + (row & 7) * 128;
+      for (int rr = 0; rr < 4; ++rr) {
+        const int row = rr * 32 + lane;
+        float2 acc = make_float2(0.f, 0.f);
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const uint4 u = *reinterpret_cast<const uint4*>(rowp + ((c ^ (row & 7)) << 4));
-          const unsigned int wv[4] = {u.x, u.y, u.z, u.w};
+        for (int half = 0; half < 2; ++half) {
+          // 16-byte chunk c of row r of a 128-byte-swizzled box sits at chunk c ^ (r & 7)
+          const uint8_t* rowp = vt + half * kBoxBytes + (row >> 3) * 1024 + (row & 7) * 128;
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const float2 e = make_float2(__uint_as_float(wv[q] << 16), __uint_as_float(wv[q] & 0xFFFF0000u));
-            acc = ffma2(e, e, acc);
+          for (int c = 0; c < 8; ++c) {
+            const uint4 u = *reinterpret_cast<const uint4*>(rowp + ((c ^ (row & 7)) << 4));
+            const unsigned int wv[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const float2 e = make_float2(__uint_as_float(wv[q] << 16), __uint_as_float(wv[q] & 0xFFFF0000u));
+              acc = ffma2(e, e, acc);
+            }
           }
         }
+        vn[rr] = acc.x + acc.y;
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&B->v_empty[vs]);
-      const int j = (tile0 + it) * kTile + row;
-      if (j < a.n_kv) a.vnorm[(long long)bh * a.n_kv + j] = acc.x + acc.y;
+#pragma unroll
+      for (int rr = 0; rr < 4; ++rr) {
+        const int j = (tile0 + it) * kTile + rr * 32 + lane;
+        if (j < a.n_kv) a.vnorm[(long long)bh * a.n_kv + j] = vn[rr];
+      }
     }
   } else {
-    // ---------------- softmax warpgroups: thread = query row ----------------
-    const int g = (warp - kFFirstWorker) >> 2;
+    // ---------------- four softmax warpgroups: thread = query row; warpgroups g and g + 2 share tile slot g,
+    //                  the first takes tokens 0-63 of the tile, the second tokens 64-127 ----------------
+    const int wgi = (warp - kFFirstWorker) >> 2;
+    const int g = wgi & 1, hf = wgi >> 1;
     const int quad = warp & 3;
     const int row = quad * 32 + lane;
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-    const uint32_t tS = tmem + (uint32_t)g * 128u + lane_base, tO = tmem + 256u + (uint32_t)g * 128u + lane_base;
+    const uint32_t tS = tmem + (uint32_t)g * 128u + lane_base + (uint32_t)hf * 64u;   // this half's 64 logits
+    const uint32_t tP = tS;                                                           // and where its P goes
+    const uint32_t tO = tmem + 256u + (uint32_t)g * 128u + lane_base + (uint32_t)hf * 64u;
     const int i_q = row % a.w;                // window position of this row (row = group * w + i)
     const float c2 = a.scale * kLog2e;
     const int n = a.n, n_kv = a.n_kv;
     const int nt_all = (n_kv + kTile - 1) / kTile;
+    float* my_max = cx.sm_stats + (g * 2 + hf) * kRows;
+    const float* other_max = cx.sm_stats + (g * 2 + (hf ^ 1)) * kRows;
     float m_ref = -INFINITY;
     float2 l2 = make_float2(0.f, 0.f);
     bool ok = true;
     int uses = 0;                             // tiles this warpgroup has processed
     for (int it = g; it < T; it += 2, ++uses) {
       ok = ok && mbar_wait(&B->s_full[g], (uint32_t)uses & 1u, abort_flag, dev_status, kDevTimeout);
-      if (!ok) break;
-      tc_fence_after();
-      const int j0 = (tile0 + it) * kTile;
-      const bool ragged = j0 + kTile > n;   // rows past the scored prefix: window rows (causal) or padding
-      // Both sweeps keep the next 16 columns in flight from tensor memory while the current ones are worked on.
+      if (ok) tc_fence_after();
+      const int j0 = (tile0 + it) * kTile + hf * 64;
+      const bool ragged = j0 + 64 > n;   // rows past the scored prefix: window rows (causal) or padding
       auto mask = [&](float* s, int c) {
 #pragma unroll
         for (int u = 0; u < 16; ++u) {
@@ -257,19 +272,26 @@ __device__ void phase_a(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tm
         }
       };
       float sa[16], sb[16];
-      // ---- sweep 1: row maximum of the tile ----
+      // ---- sweep 1: row maximum of this half of the tile; the next 16 columns travel while 16 are reduced ----
       float tmax = -INFINITY;
-      tmem_ld16(tS, sa);
+      if (ok) {
+        tmem_ld16(tS, sa);
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        float* cur = (c & 1) ? sb : sa;
-        float* nxt = (c & 1) ? sa : sb;
-        tmem_wait_ld();
-        tmem_ld16(tS + ((c + 1) & 7) * 16, nxt);   // after the last chunk: chunk 0 again, for sweep 2
-        if (ragged) mask(cur, c);
+        for (int c = 0; c < 4; ++c) {
+          float* cur = (c & 1) ? sb : sa;
+          float* nxt = (c & 1) ? sa : sb;
+          tmem_wait_ld();
+          tmem_ld16(tS + ((c + 1) & 3) * 16, nxt);   // after the last chunk: chunk 0 again, for sweep 2
+          if (ragged) mask(cur, c);
 #pragma unroll
-        for (int u = 0; u < 16; ++u) tmax = fmaxf(tmax, cur[u]);
+          for (int u = 0; u < 16; ++u) tmax = fmaxf(tmax, cur[u]);
+        }
       }
+      my_max[row] = tmax;
+      named_barrier_sync(3 + g, 256);            // the two halves of the slot exchange their row maxima
+      tmax = fmaxf(tmax, other_max[row]);
+      named_barrier_sync(3 + g, 256);            // both have read before the next tile overwrites
+      if (!ok) continue;
       const float m_tile = tmax * c2;
       const bool need = m_tile > m_ref + kRescaleThreshold;   // also true for the first visible entries (m_ref = -inf)
       float factor = 1.f;
@@ -279,11 +301,12 @@ __device__ void phase_a(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tm
         l2.y *= factor;
         m_ref = m_tile;
       }
-      // S(it) has landed, so O += P V of this warpgroup's previous tile (issued before it) is complete
+      // S(it) has landed, so O += P V of this slot's previous tile (issued before it) is complete; each half
+      // rescales its 64 columns of O_g
       if (uses > 0 && __any_sync(0xffffffffu, need)) {
         tmem_wait_ld();
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
+        for (int c = 0; c < 4; ++c) {
           float o[16];
           tmem_ld16(tO + c * 16, o);
           tmem_wait_ld();
@@ -292,17 +315,17 @@ __device__ void phase_a(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tm
           tmem_st16(tO + c * 16, reinterpret_cast<const uint32_t*>(o));
         }
       }
-      // ---- sweep 2: P = exp2(s*c2 - m_ref) as bf16 over the first 64 columns of S_g.  Chunk c of P lands on
-      //      columns [8c, 8c + 8), which belong to a chunk of S that is already in registers. ----
+      // ---- sweep 2: P = exp2(s*c2 - m_ref) as bf16 over the first 32 columns of this half.  Chunk c of P lands
+      //      on columns [8c, 8c + 8) of the half, which belong to a chunk of S that is already in registers. ----
       const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
       const float2 c22 = make_float2(c2, c2), nm2 = make_float2(-m_use, -m_use);
       __nv_bfloat162 pmax2 = __float2bfloat162_rn(0.f);
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
+      for (int c = 0; c < 4; ++c) {
         float* cur = (c & 1) ? sb : sa;     // chunk 0 sits in sa (loaded at the end of sweep 1)
         float* nxt = (c & 1) ? sa : sb;
         tmem_wait_ld();
-        if (c < 7) tmem_ld16(tS + (c + 1) * 16, nxt);
+        if (c < 3) tmem_ld16(tS + (c + 1) * 16, nxt);
         if (ragged) mask(cur, c);
         uint32_t packed[8];
 #pragma unroll
@@ -313,7 +336,7 @@ __device__ void phase_a(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tm
           packed[u] = pack_bf16x2(pp.x, pp.y);
           pmax2 = __hmax2(pmax2, *reinterpret_cast<const __nv_bfloat162*>(&packed[u]));
         }
-        tmem_st8(tS + c * 8, packed);
+        tmem_st8(tP + c * 8, packed);
       }
       // The final attention weight of an entry is p / l_final with both taken against the same reference, and
       // l_final is at least the sum this warpgroup has so far: a tile without p > kHeavyA * l needs no exact
@@ -321,7 +344,7 @@ __device__ void phase_a(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tm
       {
         const bool hv = fmaxf(__low2float(pmax2), __high2float(pmax2)) > kHeavyA * (l2.x + l2.y);
         const unsigned int any = __any_sync(0xffffffffu, hv) ? 1u : 0u;
-        if (lane == 0) a.heavy[((long long)bh * nt_all + tile0 + it) * 4 + quad] = any;
+        if (lane == 0) a.heavy[((long long)bh * nt_all + tile0 + it) * 8 + hf * 4 + quad] = any;
       }
       tmem_wait_st();
       tc_fence_before();
@@ -332,53 +355,61 @@ __device__ void phase_a(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tm
     const bool have = ok && uses > 0;
     const float m_mine = have ? m_ref : -INFINITY, l_mine = have ? l2.x + l2.y : 0.f;
 
-    // ---- merge the two warpgroups: 1 hands (m, l, O) over through shared memory (the K slots are idle: every
-    //      MMA of this phase has completed once both warpgroups have seen their last O += P V) ----
+    // ---- merge: the halves add their l, then slot 1 hands (m, l, O) to slot 0 through shared memory (the K
+    //      slots are idle: every MMA of this phase has completed once all warpgroups have seen their last
+    //      O += P V).  Each thread moves the 64 columns of O of its half. ----
     float* xO = reinterpret_cast<float*>(cx.gen_base + k_slot_off(0));   // [128 cols][128 rows] floats, 64 KB
-    named_barrier_sync(1, 256);
+    float* st_l = cx.sm_stats + 4 * kRows;   // [slot][row]: l of the second half
+    float* st_m1 = cx.sm_stats;              // slot 1's m     (the row-maxima exchange is over)
+    float* st_l1 = cx.sm_stats + kRows;      // slot 1's l
+    named_barrier_sync(1, kFWorkerWarps * 32);
+    if (hf == 1) st_l[g * kRows + row] = l_mine;
+    named_barrier_sync(1, kFWorkerWarps * 32);
+    const float l_slot = l_mine + (hf == 0 ? st_l[g * kRows + row] : 0.f);   // meaningful in the first half only
     if (g == 1) {
-      cx.sm_stats[row] = m_mine;
-      cx.sm_stats[128 + row] = l_mine;
+      if (hf == 0) { st_m1[row] = m_mine; st_l1[row] = l_slot; }
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
-        float o[32];
+        float o[16];
         if (have) {
-          tmem_ld32(tO + c * 32, o);
+          tmem_ld16(tO + c * 16, o);
           tmem_wait_ld();
         } else {
 #pragma unroll
-          for (int u = 0; u < 32; ++u) o[u] = 0.f;
+          for (int u = 0; u < 16; ++u) o[u] = 0.f;
         }
 #pragma unroll
-        for (int u = 0; u < 32; ++u) xO[(c * 32 + u) * 128 + row] = o[u];
+        for (int u = 0; u < 16; ++u) xO[(hf * 64 + c * 16 + u) * 128 + row] = o[u];
       }
     }
-    named_barrier_sync(1, 256);
+    named_barrier_sync(1, kFWorkerWarps * 32);
     if (g == 0) {
-      const float m1 = cx.sm_stats[row], l1 = cx.sm_stats[128 + row];
+      const float m1 = st_m1[row], l1 = st_l1[row];
       const float m = fmaxf(m_mine, m1);
       const float a0 = (m_mine == -INFINITY) ? 0.f : ex2_approx(m_mine - m);
       const float a1 = (m1 == -INFINITY) ? 0.f : ex2_approx(m1 - m);
       const long long o_idx = (long long)blockIdx.x * kRows + row;
-      float* Op = a.part_O + o_idx * kHeadDim;
+      float* Op = a.part_O + o_idx * kHeadDim + hf * 64;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
-        float o[32];
+        float o[16];
         if (have) {
-          tmem_ld32(tO + c * 32, o);
+          tmem_ld16(tO + c * 16, o);
           tmem_wait_ld();
         } else {
 #pragma unroll
-          for (int u = 0; u < 32; ++u) o[u] = 0.f;
+          for (int u = 0; u < 16; ++u) o[u] = 0.f;
         }
 #pragma unroll
-        for (int u = 0; u < 32; ++u) o[u] = o[u] * a0 + xO[(c * 32 + u) * 128 + row] * a1;
+        for (int u = 0; u < 16; ++u) o[u] = o[u] * a0 + xO[(hf * 64 + c * 16 + u) * 128 + row] * a1;
 #pragma unroll
-        for (int u = 0; u < 32; u += 4)
-          *reinterpret_cast<float4*>(Op + c * 32 + u) = make_float4(o[u], o[u + 1], o[u + 2], o[u + 3]);
+        for (int u = 0; u < 16; u += 4)
+          *reinterpret_cast<float4*>(Op + c * 16 + u) = make_float4(o[u], o[u + 1], o[u + 2], o[u + 3]);
       }
-      a.part_m[o_idx] = m;
-      a.part_l[o_idx] = l_mine * a0 + l1 * a1;
+      if (hf == 0) {
+        a.part_m[o_idx] = m;
+        a.part_l[o_idx] = l_slot * a0 + l1 * a1;
+      }
     }
     fence_proxy_async_smem();   // the hand-over buffer lies in the tile ring, which TMA loads refill next
     tc_fence_before();
@@ -548,7 +579,7 @@ __device__ void phase_c(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tm
         umma_commit(&B->kv_empty[s]);
       }
     }
-  } else if (warp >= kFFirstWorker) {
+  } else if (warp >= kFFirstWorker && warp < kFFirstWorker + kFWorkerWarps) {
     const int cgp = (warp - kFFirstWorker) >> 2;     // column group 0..3
     const int quad = warp & 3;                       // TMEM lane quarter this warp may touch
     const int t = quad * 32 + lane;
@@ -573,24 +604,26 @@ __device__ void phase_c(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tm
     float* I_head = a.I_hat + (long long)bh * n;
     bool ok = true;
     const int nt_all = (a.n_kv + kTile - 1) / kTile;
-    const uint4* hv_head = reinterpret_cast<const uint4*>(a.heavy) + (long long)bh * nt_all;
+    const uint4* hv_head = reinterpret_cast<const uint4*>(a.heavy) + (long long)bh * nt_all * 2;
     float vn_next = 0.f;
-    uint4 hv_next = make_uint4(0, 0, 0, 0);
+    uint4 hv_next = make_uint4(0, 0, 0, 0), hw_next = make_uint4(0, 0, 0, 0);
     if (T > 0) {
       const int j = tile0 * kTile + t;
       vn_next = (j < n) ? vn_head[j] : 1.f;
-      hv_next = hv_head[tile0];
+      hv_next = hv_head[2 * tile0];
+      hw_next = hv_head[2 * tile0 + 1];
     }
 
     for (int it = 0; it < T; ++it) {
       const int s = it & 1;
       const uint32_t par = (uint32_t)(it >> 1) & 1u;
       const float vn = vn_next;
-      const bool tile_heavy = (hv_next.x | hv_next.y | hv_next.z | hv_next.w) != 0;   // same for the whole CTA
+      const bool tile_heavy = (hv_next.x | hv_next.y | hv_next.z | hv_next.w | hw_next.x | hw_next.y | hw_next.z | hw_next.w) != 0;   // same for the whole CTA
       if (it + 1 < T) {   // next tile's ||v||^2 and flags, well ahead of their use
         const int jn = (tile0 + it + 1) * kTile + t;
         vn_next = (jn < n) ? vn_head[jn] : 1.f;
-        hv_next = hv_head[tile0 + it + 1];
+        hv_next = hv_head[2 * (tile0 + it + 1)];
+        hw_next = hv_head[2 * (tile0 + it + 1) + 1];
       }
       // The shares of the previous tile are summed in a fixed order by warpgroup 0 once all sixteen warps have
       // stored theirs.  A slot of `red` is rewritten four tiles later, which the two accumulator buffers only
@@ -700,7 +733,7 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   __shared__ __align__(8) FusedBars bars;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
-  __shared__ float sm_stats[2 * kRows];
+  __shared__ float sm_stats[6 * kRows];
   __shared__ float red[4][4][kTile];   // [tile & 3][warpgroup][token]: each warpgroup's share of the score
 
   const int group = blockIdx.x / a.cpg, rank = blockIdx.x % a.cpg;
@@ -762,7 +795,7 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     alive = group_barrier(counter, (++epoch) * (unsigned int)a.cpg, &abort_flag, a.dev_status);
     if (!alive) break;
     // ---- phase B: rows rank, rank + cpg, ... of the head; the sixteen worker warps share them ----
-    if (cx.warp >= kFFirstWorker) {
+    if (cx.warp >= kFFirstWorker && cx.warp < kFFirstWorker + kFWorkerWarps) {
       const int wq = cx.warp - kFFirstWorker;
       const int rows_max = (kRows + a.cpg - 1) / a.cpg;          // rows of the busiest CTA of the group
       int wpr = kFWorkerWarps;                                    // warps per row: 16, 8, 4, 2 or 1
@@ -796,22 +829,43 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 }  // namespace
 
 // Number of CTA groups = heads in flight.  With `reuse_l2` only as many as fit a 72 MB share of L2 (phase C then
-// re-reads the heads from there); otherwise as many as there are heads.  Among the allowed counts the one with the
-// fewest rounds x tiles per CTA wins; ties go to more groups (fewer barrier rounds).
+// re-reads the heads from there); otherwise as many as there are heads.  Among the allowed counts the cheapest wins,
+// where a round costs its tiles per CTA plus about eight tiles' worth of pipeline fill, merge and barriers
+// (measured); ties go to more groups.
 void fused_plan(const Problem& p, int sm_count, bool reuse_l2, int* groups, int* cpg) {
   const long long head_bytes = 2ll * p.n_kv * p.d * 2;
   long long limit = reuse_l2 ? (72ll << 20) / (head_bytes > 0 ? head_bytes : 1) : p.BH;
   if (limit < 1) limit = 1;
   const int tiles = (p.n_kv + kTile - 1) / kTile;
+  constexpr int kRoundOverheadTiles = 8;
   int best_g = 1;
   long long best_cost = -1;
   for (int g = 1; g <= p.BH && g <= limit && g <= sm_count && g <= 256; ++g) {
     const int c = sm_count / g;
-    const long long cost = (long long)((p.BH + g - 1) / g) * ((tiles + c - 1) / c);
+    const long long cost = (long long)((p.BH + g - 1) / g) * ((tiles + c - 1) / c + kRoundOverheadTiles);
     if (best_cost < 0 || cost <= best_cost) { best_cost = cost; best_g = g; }
   }
   *groups = best_g;
   *cpg = sm_count / best_g;
+}
+
+bool tc_supported(const Problem& p) {
+  if (p.dtype != RESTKV_BF16 || p.d != kHeadDim || p.R != kRows) return false;
+  if (p.w != 16 && p.w != 32 && p.w != 64 && p.w != 128) return false;
+  return true;
+}
+
+cudaError_t tc_init(void** state) {
+  *state = nullptr;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess) return e;
+  if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+  static TcState the_state;
+  the_state.encode = (EncodeTiledFn)fn;
+  *state = &the_state;
+  return cudaSuccess;
 }
 
 cudaError_t tc_fused_init() {
