@@ -56,7 +56,8 @@ size_t plan_workspace(const Problem& p, int budget, int sm_count, bool adaptive,
   w.part_l = (float*)take(slots * R * sizeof(float));
   w.part_O = (float*)take(slots * R * d * sizeof(float));
   w.counters = (unsigned int*)take(1024);
-  w.heavy = (unsigned int*)take(BH * (size_t)((p.n_kv + 127) / 128) * 8 * sizeof(unsigned int));
+  w.tile_max = (float*)take(BH * (size_t)((p.n_kv + 127) / 128) * 128 * sizeof(float));
+  w.row_M2 = (float*)take(BH * 128 * sizeof(float));
   w.vnorm = (float*)take(BH * (size_t)p.n_kv * sizeof(float));
   w.fin_m = (float*)take(BH * R * sizeof(float));
   w.fin_l = (float*)take(BH * R * sizeof(float));

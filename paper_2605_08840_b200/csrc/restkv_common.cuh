@@ -34,7 +34,8 @@ struct Workspace {
   float* part_O;          // [slots, R, d]
   float* vnorm;           // [BH, n_kv]  ||v_j||^2 (tensor-core path)
   unsigned int* counters; // [256] group barrier counters of the head-sequential kernel
-  unsigned int* heavy;    // [BH, tiles, 8] per-tile flags of the persistent score kernel
+  float* tile_max;        // [BH, tiles, 128] per-tile row maxima of the persistent score kernel
+  float* row_M2;          // [BH, 128] log2 normaliser of each query row
   float* fin_m;           // [BH, R]    row max of the scaled logits (natural units)
   float* fin_l;           // [BH, R]    sum of exp(s - m)
   float* O_f32;           // [BH, R, d]

@@ -35,7 +35,8 @@ struct FusedArgs {
   __nv_bfloat16* O_m2;               // [BH, 128, 128]  -2 * bf16(O)
   __nv_bfloat16* aug;                // [BH, 128, 64]
   float* vnorm;                      // [BH, n_kv]
-  unsigned int* heavy;               // [BH, tiles, 8]: one word per softmax warp, set if the tile may hold a weight > kHeavyA
+  float* tile_max;                   // [BH, tiles, 128] largest scaled logit (log2 units) of each query row in each tile
+  float* row_M2;                     // [BH, 128] m*log2e + log2 l of each query row (written by the merge)
   float* I_hat;                      // [BH, n]
   const __nv_bfloat16* V;
   long long vsb, vsh, vsn;
@@ -293,6 +294,9 @@ __device__ void phase_a(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tm
       named_barrier_sync(3 + g, 256);            // both have read before the next tile overwrites
       if (!ok) continue;
       const float m_tile = tmax * c2;
+      // phase C takes the exact distance only in tiles where some weight can exceed kHeavyA: it compares this
+      // maximum with the row's final normaliser
+      if (hf == 0) a.tile_max[((long long)bh * nt_all + tile0 + it) * kRows + row] = m_tile;
       const bool need = m_tile > m_ref + kRescaleThreshold;   // also true for the first visible entries (m_ref = -inf)
       float factor = 1.f;
       if (need) {
@@ -319,7 +323,6 @@ __device__ void phase_a(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tm
       //      on columns [8c, 8c + 8) of the half, which belong to a chunk of S that is already in registers. ----
       const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
       const float2 c22 = make_float2(c2, c2), nm2 = make_float2(-m_use, -m_use);
-      __nv_bfloat162 pmax2 = __float2bfloat162_rn(0.f);
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         float* cur = (c & 1) ? sb : sa;     // chunk 0 sits in sa (loaded at the end of sweep 1)
@@ -334,17 +337,8 @@ __device__ void phase_a(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tm
           const float2 pp = make_float2(ex2_approx(e.x), ex2_approx(e.y));
           l2 = fadd2(l2, pp);
           packed[u] = pack_bf16x2(pp.x, pp.y);
-          pmax2 = __hmax2(pmax2, *reinterpret_cast<const __nv_bfloat162*>(&packed[u]));
         }
         tmem_st8(tP + c * 8, packed);
-      }
-      // The final attention weight of an entry is p / l_final with both taken against the same reference, and
-      // l_final is at least the sum this warpgroup has so far: a tile without p > kHeavyA * l needs no exact
-      // distances in phase C.
-      {
-        const bool hv = fmaxf(__low2float(pmax2), __high2float(pmax2)) > kHeavyA * (l2.x + l2.y);
-        const unsigned int any = __any_sync(0xffffffffu, hv) ? 1u : 0u;
-        if (lane == 0) a.heavy[((long long)bh * nt_all + tile0 + it) * 8 + hf * 4 + quad] = any;
       }
       tmem_wait_st();
       tc_fence_before();
@@ -508,6 +502,7 @@ __device__ void combine_rows(const FusedArgs& a, int bh, int group, int r, int s
   if (lane == 0) {
     const float c2 = a.scale * kLog2e;
     const float M2 = m + log2f(l);        // A = exp2(s * c2 - M2)
+    a.row_M2[ri] = M2;
     split3(-M2 / c2, arow);
     split3(on, arow + 16);
   }
@@ -604,26 +599,34 @@ __device__ void phase_c(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tm
     float* I_head = a.I_hat + (long long)bh * n;
     bool ok = true;
     const int nt_all = (a.n_kv + kTile - 1) / kTile;
-    const uint4* hv_head = reinterpret_cast<const uint4*>(a.heavy) + (long long)bh * nt_all * 2;
+    // a tile needs exact distances iff some row's largest logit in it reaches that row's M2 - log2(1 / kHeavyA);
+    // every warp checks all 128 rows (lane = rows lane, lane + 32, ...) so that no synchronisation is needed
+    const float* tm_head = a.tile_max + (long long)bh * nt_all * kRows;
+    float m2r[4], tm_next[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      m2r[k] = a.row_M2[(long long)bh * kRows + k * 32 + lane] - log2f(1.f / kHeavyA);
+      tm_next[k] = -INFINITY;
+    }
     float vn_next = 0.f;
-    uint4 hv_next = make_uint4(0, 0, 0, 0), hw_next = make_uint4(0, 0, 0, 0);
     if (T > 0) {
       const int j = tile0 * kTile + t;
       vn_next = (j < n) ? vn_head[j] : 1.f;
-      hv_next = hv_head[2 * tile0];
-      hw_next = hv_head[2 * tile0 + 1];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) tm_next[k] = tm_head[(long long)tile0 * kRows + k * 32 + lane];
     }
 
     for (int it = 0; it < T; ++it) {
       const int s = it & 1;
       const uint32_t par = (uint32_t)(it >> 1) & 1u;
       const float vn = vn_next;
-      const bool tile_heavy = (hv_next.x | hv_next.y | hv_next.z | hv_next.w | hw_next.x | hw_next.y | hw_next.z | hw_next.w) != 0;   // same for the whole CTA
-      if (it + 1 < T) {   // next tile's ||v||^2 and flags, well ahead of their use
+      const bool tile_heavy = __any_sync(0xffffffffu, tm_next[0] > m2r[0] || tm_next[1] > m2r[1] ||
+                                                          tm_next[2] > m2r[2] || tm_next[3] > m2r[3]);
+      if (it + 1 < T) {   // next tile's ||v||^2 and row maxima, well ahead of their use
         const int jn = (tile0 + it + 1) * kTile + t;
         vn_next = (jn < n) ? vn_head[jn] : 1.f;
-        hv_next = hv_head[2 * (tile0 + it + 1)];
-        hw_next = hv_head[2 * (tile0 + it + 1) + 1];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) tm_next[k] = tm_head[(long long)(tile0 + it + 1) * kRows + k * 32 + lane];
       }
       // The shares of the previous tile are summed in a fixed order by warpgroup 0 once all sixteen warps have
       // stored theirs.  A slot of `red` is rewritten four tiles later, which the two accumulator buffers only
@@ -896,7 +899,7 @@ cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, 
   a.part_m = ws.part_m; a.part_l = ws.part_l; a.part_O = ws.part_O;
   a.O_f32 = ws.O_f32; a.O_m2 = ws.O_m2; a.aug = ws.aug; a.vnorm = ws.vnorm; a.I_hat = ws.I_hat;
   a.V = (const __nv_bfloat16*)V; a.vsb = p.vsb; a.vsh = p.vsh; a.vsn = p.vsn;
-  a.counters = ws.counters; a.heavy = ws.heavy; a.dev_status = dev_status;
+  a.counters = ws.counters; a.tile_max = ws.tile_max; a.row_M2 = ws.row_M2; a.dev_status = dev_status;
   cudaError_t e = cudaMemsetAsync(ws.counters, 0, 1024, st);
   if (e != cudaSuccess) return e;
   const dim3 grid(a.groups * a.cpg), block(kFThreads);
