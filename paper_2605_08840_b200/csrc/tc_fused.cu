@@ -16,10 +16,15 @@ namespace restkv {
 
 namespace {
 
-constexpr int kFFirstWorker = 2;                  // warp 0: TMA producer, warp 1: MMA issuer
-constexpr int kFWorkerWarps = 16;                 // warps 2..17
-constexpr int kFNormWarps = 2;                    // warps 18, 19: ||v||^2 of the tokens during phase A
-constexpr int kFThreads = (kFFirstWorker + kFWorkerWarps + kFNormWarps) * 32;
+constexpr int kFFirstWorker = 4;                  // warp 0: TMA producer, 1: MMA issuer, 2-3: ||v||^2 during phase A
+constexpr int kFWorkerWarps = 16;                 // warps 4..19
+constexpr int kFThreads = (kFFirstWorker + kFWorkerWarps) * 32;
+// Registers per thread: 96 at launch (640 threads), i.e. a pool of 20 warps x 32 x 96 = 61440 for the CTA.  The control
+// warpgroup then shrinks to 32 and the sixteen worker warps grow to 112: 4*32*32 + 16*32*112 = 61440, exactly the pool
+// (a larger request would block for ever: the pool is what the CTA was launched with, not the SM's register file).
+constexpr int kFRegsLaunch = 96, kFRegsControl = 32, kFRegsWorker = 112;
+static_assert(kFFirstWorker * kFRegsControl + kFWorkerWarps * kFRegsWorker <= (kFFirstWorker + kFWorkerWarps) * kFRegsLaunch,
+              "the register split must fit the pool the CTA is launched with");
 constexpr int kFRing = 4;                         // 32 KB tile slots after Q | O' | aug | ones
 constexpr size_t kFSmem = 2 * kTileBytes + kAugBytes + kOnesBytes + kFRing * kTileBytes + 1024;
 constexpr int kFVSlots = 3;                       // phase A: V slots = ring 2, ring 3 and the (then unused) O' tile
@@ -91,8 +96,10 @@ __device__ void init_bars(FusedBars* B, bool first) {
   fence_mbar_init();
 }
 
-// All CTAs of a group arrive and wait until `target` arrivals have been counted.  Bounded.
-__device__ bool group_barrier(unsigned int* counter, unsigned int target, volatile int* abort_flag,
+// All CTAs of a group arrive and wait until `target` arrivals have been counted.  Bounded.  Thread 0 runs the
+// counter; every other thread calls group_barrier_follow at the same point.  Both return the same verdict (one
+// shared word written between the two synchronisations): false once any wait of the CTA has run out.
+__device__ bool group_barrier(unsigned int* counter, unsigned int target, volatile int* abort_flag, volatile int* go,
                               unsigned int* dev_status) {
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -107,9 +114,15 @@ __device__ bool group_barrier(unsigned int* counter, unsigned int target, volati
         break;
       }
     }
+    *go = (*abort_flag == 0);
   }
   __syncthreads();
-  return *abort_flag == 0;
+  return *go != 0;
+}
+__device__ bool group_barrier_follow(volatile int* go) {
+  __syncthreads();
+  __syncthreads();
+  return *go != 0;
 }
 
 struct Ctx {
@@ -133,7 +146,7 @@ __device__ __forceinline__ uint32_t v_slot_off(int i) { return i < 2 ? kOffRing 
 // maximum and its own O accumulator), worker warps 8-15 reduce ||v_j||^2 of the tokens from the V tiles.
 // Tensor memory: S_g at g*128 (bf16 P_g overwrites its first 64 columns), O_g at 256 + g*128.
 // At the end the two warpgroups' (m, l, O) are merged and written as the CTA's partial.
-__device__ void phase_a(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tmQ, const CUtensorMap* tmK,
+__device__ void phase_a_control(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tmQ, const CUtensorMap* tmK,
                         const CUtensorMap* tmV, int bh, int rank, int tile0, int T) {
   FusedBars* B = cx.B;
   int* abort_flag = cx.abort_flag;
@@ -198,9 +211,9 @@ __device__ void phase_a(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tm
         }
       }
     }
-  } else if (warp >= kFFirstWorker + kFWorkerWarps) {
+  } else if (warp < kFFirstWorker) {
     // ---------------- ||v||^2: one warp takes the even tiles, the other the odd ones; lane = 4 tokens ----------------
-    const int vg = warp - (kFFirstWorker + kFWorkerWarps);
+    const int vg = warp - 2;
     bool ok = true;
     for (int it = 0; it < T && ok; ++it) {
       const int vs = it % kFVSlots;
@@ -238,176 +251,186 @@ __device__ void phase_a(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tm
         if (j < a.n_kv) a.vnorm[(long long)bh * a.n_kv + j] = vn[rr];
       }
     }
-  } else {
-    // ---------------- four softmax warpgroups: thread = query row; warpgroups g and g + 2 share tile slot g,
-    //                  the first takes tokens 0-63 of the tile, the second tokens 64-127 ----------------
-    const int wgi = (warp - kFFirstWorker) >> 2;
-    const int g = wgi & 1, hf = wgi >> 1;
-    const int quad = warp & 3;
-    const int row = quad * 32 + lane;
-    const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-    const uint32_t tS = tmem + (uint32_t)g * 128u + lane_base + (uint32_t)hf * 64u;   // this half's 64 logits
-    const uint32_t tP = tS;                                                           // and where its P goes
-    const uint32_t tO = tmem + 256u + (uint32_t)g * 128u + lane_base + (uint32_t)hf * 64u;
-    const int i_q = row % a.w;                // window position of this row (row = group * w + i)
-    const float c2 = a.scale * kLog2e;
-    const int n = a.n, n_kv = a.n_kv;
-    const int nt_all = (n_kv + kTile - 1) / kTile;
-    float* my_max = cx.sm_stats + (g * 2 + hf) * kRows;
-    const float* other_max = cx.sm_stats + (g * 2 + (hf ^ 1)) * kRows;
-    float m_ref = -INFINITY;
-    float2 l2 = make_float2(0.f, 0.f);
-    bool ok = true;
-    int uses = 0;                             // tiles this warpgroup has processed
-    for (int it = g; it < T; it += 2, ++uses) {
-      ok = ok && mbar_wait(&B->s_full[g], (uint32_t)uses & 1u, abort_flag, dev_status, kDevTimeout);
-      if (ok) tc_fence_after();
-      const int j0 = (tile0 + it) * kTile + hf * 64;
-      const bool ragged = j0 + 64 > n;   // rows past the scored prefix: window rows (causal) or padding
-      auto mask = [&](float* s, int c) {
+  }
+}
+
+__device__ void phase_a_worker(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tmQ, const CUtensorMap* tmK,
+                        const CUtensorMap* tmV, int bh, int rank, int tile0, int T) {
+  FusedBars* B = cx.B;
+  int* abort_flag = cx.abort_flag;
+  unsigned int* dev_status = a.dev_status;
+  const int b = bh / a.Hkv, h = bh % a.Hkv;
+  const int warp = cx.warp, lane = cx.lane;
+  const uint32_t tmem = cx.tmem;
+
+  // ---------------- four softmax warpgroups: thread = query row; warpgroups g and g + 2 share tile slot g,
+  //                  the first takes tokens 0-63 of the tile, the second tokens 64-127 ----------------
+  const int wgi = (warp - kFFirstWorker) >> 2;
+  const int g = wgi & 1, hf = wgi >> 1;
+  const int quad = warp & 3;
+  const int row = quad * 32 + lane;
+  const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+  const uint32_t tS = tmem + (uint32_t)g * 128u + lane_base + (uint32_t)hf * 64u;   // this half's 64 logits
+  const uint32_t tP = tS;                                                           // and where its P goes
+  const uint32_t tO = tmem + 256u + (uint32_t)g * 128u + lane_base + (uint32_t)hf * 64u;
+  const int i_q = row % a.w;                // window position of this row (row = group * w + i)
+  const float c2 = a.scale * kLog2e;
+  const int n = a.n, n_kv = a.n_kv;
+  const int nt_all = (n_kv + kTile - 1) / kTile;
+  float* my_max = cx.sm_stats + (g * 2 + hf) * kRows;
+  const float* other_max = cx.sm_stats + (g * 2 + (hf ^ 1)) * kRows;
+  float m_ref = -INFINITY;
+  float2 l2 = make_float2(0.f, 0.f);
+  bool ok = true;
+  int uses = 0;                             // tiles this warpgroup has processed
+  for (int it = g; it < T; it += 2, ++uses) {
+    ok = ok && mbar_wait(&B->s_full[g], (uint32_t)uses & 1u, abort_flag, dev_status, kDevTimeout);
+    if (ok) tc_fence_after();
+    const int j0 = (tile0 + it) * kTile + hf * 64;
+    const bool ragged = j0 + 64 > n;   // rows past the scored prefix: window rows (causal) or padding
+    auto mask = [&](float* s, int c) {
 #pragma unroll
-        for (int u = 0; u < 16; ++u) {
-          const int j = j0 + c * 16 + u;
-          const bool vis = (j < n_kv) && (j < n || (j - n) <= i_q);
-          s[u] = vis ? s[u] : -INFINITY;
-        }
-      };
-      float sa[16], sb[16];
-      // ---- sweep 1: row maximum of this half of the tile; the next 16 columns travel while 16 are reduced ----
-      float tmax = -INFINITY;
-      if (ok) {
-        tmem_ld16(tS, sa);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          float* cur = (c & 1) ? sb : sa;
-          float* nxt = (c & 1) ? sa : sb;
-          tmem_wait_ld();
-          tmem_ld16(tS + ((c + 1) & 3) * 16, nxt);   // after the last chunk: chunk 0 again, for sweep 2
-          if (ragged) mask(cur, c);
-#pragma unroll
-          for (int u = 0; u < 16; ++u) tmax = fmaxf(tmax, cur[u]);
-        }
+      for (int u = 0; u < 16; ++u) {
+        const int j = j0 + c * 16 + u;
+        const bool vis = (j < n_kv) && (j < n || (j - n) <= i_q);
+        s[u] = vis ? s[u] : -INFINITY;
       }
-      my_max[row] = tmax;
-      named_barrier_sync(3 + g, 256);            // the two halves of the slot exchange their row maxima
-      tmax = fmaxf(tmax, other_max[row]);
-      named_barrier_sync(3 + g, 256);            // both have read before the next tile overwrites
-      if (!ok) continue;
-      const float m_tile = tmax * c2;
-      // phase C takes the exact distance only in tiles where some weight can exceed kHeavyA: it compares this
-      // maximum with the row's final normaliser
-      if (hf == 0) a.tile_max[((long long)bh * nt_all + tile0 + it) * kRows + row] = m_tile;
-      const bool need = m_tile > m_ref + kRescaleThreshold;   // also true for the first visible entries (m_ref = -inf)
-      float factor = 1.f;
-      if (need) {
-        factor = ex2_approx(m_ref - m_tile);   // 0 when m_ref = -inf
-        l2.x *= factor;
-        l2.y *= factor;
-        m_ref = m_tile;
-      }
-      // S(it) has landed, so O += P V of this slot's previous tile (issued before it) is complete; each half
-      // rescales its 64 columns of O_g
-      if (uses > 0 && __any_sync(0xffffffffu, need)) {
-        tmem_wait_ld();
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          float o[16];
-          tmem_ld16(tO + c * 16, o);
-          tmem_wait_ld();
-#pragma unroll
-          for (int u = 0; u < 16; ++u) o[u] *= factor;
-          tmem_st16(tO + c * 16, reinterpret_cast<const uint32_t*>(o));
-        }
-      }
-      // ---- sweep 2: P = exp2(s*c2 - m_ref) as bf16 over the first 32 columns of this half.  Chunk c of P lands
-      //      on columns [8c, 8c + 8) of the half, which belong to a chunk of S that is already in registers. ----
-      const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-      const float2 c22 = make_float2(c2, c2), nm2 = make_float2(-m_use, -m_use);
+    };
+    float sa[16], sb[16];
+    // ---- sweep 1: row maximum of this half of the tile; the next 16 columns travel while 16 are reduced ----
+    float tmax = -INFINITY;
+    if (ok) {
+      tmem_ld16(tS, sa);
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
-        float* cur = (c & 1) ? sb : sa;     // chunk 0 sits in sa (loaded at the end of sweep 1)
+        float* cur = (c & 1) ? sb : sa;
         float* nxt = (c & 1) ? sa : sb;
         tmem_wait_ld();
-        if (c < 3) tmem_ld16(tS + (c + 1) * 16, nxt);
+        tmem_ld16(tS + ((c + 1) & 3) * 16, nxt);   // after the last chunk: chunk 0 again, for sweep 2
         if (ragged) mask(cur, c);
-        uint32_t packed[8];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const float2 e = ffma2(make_float2(cur[2 * u], cur[2 * u + 1]), c22, nm2);
-          const float2 pp = make_float2(ex2_approx(e.x), ex2_approx(e.y));
-          l2 = fadd2(l2, pp);
-          packed[u] = pack_bf16x2(pp.x, pp.y);
-        }
-        tmem_st8(tP + c * 8, packed);
+        for (int u = 0; u < 16; ++u) tmax = fmaxf(tmax, cur[u]);
       }
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(&B->p_full[g]);
     }
-    if (uses > 0 && ok) ok = mbar_wait(&B->pv_done[g], (uint32_t)(uses - 1) & 1u, abort_flag, dev_status, kDevTimeout);
-    if (ok && uses > 0) tc_fence_after();
-    const bool have = ok && uses > 0;
-    const float m_mine = have ? m_ref : -INFINITY, l_mine = have ? l2.x + l2.y : 0.f;
-
-    // ---- merge: the halves add their l, then slot 1 hands (m, l, O) to slot 0 through shared memory (the K
-    //      slots are idle: every MMA of this phase has completed once all warpgroups have seen their last
-    //      O += P V).  Each thread moves the 64 columns of O of its half. ----
-    float* xO = reinterpret_cast<float*>(cx.gen_base + k_slot_off(0));   // [128 cols][128 rows] floats, 64 KB
-    float* st_l = cx.sm_stats + 4 * kRows;   // [slot][row]: l of the second half
-    float* st_m1 = cx.sm_stats;              // slot 1's m     (the row-maxima exchange is over)
-    float* st_l1 = cx.sm_stats + kRows;      // slot 1's l
-    named_barrier_sync(1, kFWorkerWarps * 32);
-    if (hf == 1) st_l[g * kRows + row] = l_mine;
-    named_barrier_sync(1, kFWorkerWarps * 32);
-    const float l_slot = l_mine + (hf == 0 ? st_l[g * kRows + row] : 0.f);   // meaningful in the first half only
-    if (g == 1) {
-      if (hf == 0) { st_m1[row] = m_mine; st_l1[row] = l_slot; }
+    my_max[row] = tmax;
+    named_barrier_sync(3 + g, 256);            // the two halves of the slot exchange their row maxima
+    tmax = fmaxf(tmax, other_max[row]);
+    named_barrier_sync(3 + g, 256);            // both have read before the next tile overwrites
+    if (!ok) continue;
+    const float m_tile = tmax * c2;
+    // phase C takes the exact distance only in tiles where some weight can exceed kHeavyA: it compares this
+    // maximum with the row's final normaliser
+    if (hf == 0) a.tile_max[((long long)bh * nt_all + tile0 + it) * kRows + row] = m_tile;
+    const bool need = m_tile > m_ref + kRescaleThreshold;   // also true for the first visible entries (m_ref = -inf)
+    float factor = 1.f;
+    if (need) {
+      factor = ex2_approx(m_ref - m_tile);   // 0 when m_ref = -inf
+      l2.x *= factor;
+      l2.y *= factor;
+      m_ref = m_tile;
+    }
+    // S(it) has landed, so O += P V of this slot's previous tile (issued before it) is complete; each half
+    // rescales its 64 columns of O_g
+    if (uses > 0 && __any_sync(0xffffffffu, need)) {
+      tmem_wait_ld();
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         float o[16];
-        if (have) {
-          tmem_ld16(tO + c * 16, o);
-          tmem_wait_ld();
-        } else {
+        tmem_ld16(tO + c * 16, o);
+        tmem_wait_ld();
 #pragma unroll
-          for (int u = 0; u < 16; ++u) o[u] = 0.f;
-        }
-#pragma unroll
-        for (int u = 0; u < 16; ++u) xO[(hf * 64 + c * 16 + u) * 128 + row] = o[u];
+        for (int u = 0; u < 16; ++u) o[u] *= factor;
+        tmem_st16(tO + c * 16, reinterpret_cast<const uint32_t*>(o));
       }
     }
-    named_barrier_sync(1, kFWorkerWarps * 32);
-    if (g == 0) {
-      const float m1 = st_m1[row], l1 = st_l1[row];
-      const float m = fmaxf(m_mine, m1);
-      const float a0 = (m_mine == -INFINITY) ? 0.f : ex2_approx(m_mine - m);
-      const float a1 = (m1 == -INFINITY) ? 0.f : ex2_approx(m1 - m);
-      const long long o_idx = (long long)blockIdx.x * kRows + row;
-      float* Op = a.part_O + o_idx * kHeadDim + hf * 64;
+    // ---- sweep 2: P = exp2(s*c2 - m_ref) as bf16 over the first 32 columns of this half.  Chunk c of P lands
+    //      on columns [8c, 8c + 8) of the half, which belong to a chunk of S that is already in registers. ----
+    const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+    const float2 c22 = make_float2(c2, c2), nm2 = make_float2(-m_use, -m_use);
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        float o[16];
-        if (have) {
-          tmem_ld16(tO + c * 16, o);
-          tmem_wait_ld();
-        } else {
+    for (int c = 0; c < 4; ++c) {
+      float* cur = (c & 1) ? sb : sa;     // chunk 0 sits in sa (loaded at the end of sweep 1)
+      float* nxt = (c & 1) ? sa : sb;
+      tmem_wait_ld();
+      if (c < 3) tmem_ld16(tS + (c + 1) * 16, nxt);
+      if (ragged) mask(cur, c);
+      uint32_t packed[8];
 #pragma unroll
-          for (int u = 0; u < 16; ++u) o[u] = 0.f;
-        }
-#pragma unroll
-        for (int u = 0; u < 16; ++u) o[u] = o[u] * a0 + xO[(hf * 64 + c * 16 + u) * 128 + row] * a1;
-#pragma unroll
-        for (int u = 0; u < 16; u += 4)
-          *reinterpret_cast<float4*>(Op + c * 16 + u) = make_float4(o[u], o[u + 1], o[u + 2], o[u + 3]);
+      for (int u = 0; u < 8; ++u) {
+        const float2 e = ffma2(make_float2(cur[2 * u], cur[2 * u + 1]), c22, nm2);
+        const float2 pp = make_float2(ex2_approx(e.x), ex2_approx(e.y));
+        l2 = fadd2(l2, pp);
+        packed[u] = pack_bf16x2(pp.x, pp.y);
       }
-      if (hf == 0) {
-        a.part_m[o_idx] = m;
-        a.part_l[o_idx] = l_slot * a0 + l1 * a1;
-      }
+      tmem_st8(tP + c * 8, packed);
     }
-    fence_proxy_async_smem();   // the hand-over buffer lies in the tile ring, which TMA loads refill next
+    tmem_wait_st();
     tc_fence_before();
+    mbar_arrive(&B->p_full[g]);
   }
+  if (uses > 0 && ok) ok = mbar_wait(&B->pv_done[g], (uint32_t)(uses - 1) & 1u, abort_flag, dev_status, kDevTimeout);
+  if (ok && uses > 0) tc_fence_after();
+  const bool have = ok && uses > 0;
+  const float m_mine = have ? m_ref : -INFINITY, l_mine = have ? l2.x + l2.y : 0.f;
+
+  // ---- merge: the halves add their l, then slot 1 hands (m, l, O) to slot 0 through shared memory (the K
+  //      slots are idle: every MMA of this phase has completed once all warpgroups have seen their last
+  //      O += P V).  Each thread moves the 64 columns of O of its half. ----
+  float* xO = reinterpret_cast<float*>(cx.gen_base + k_slot_off(0));   // [128 cols][128 rows] floats, 64 KB
+  float* st_l = cx.sm_stats + 4 * kRows;   // [slot][row]: l of the second half
+  float* st_m1 = cx.sm_stats;              // slot 1's m     (the row-maxima exchange is over)
+  float* st_l1 = cx.sm_stats + kRows;      // slot 1's l
+  named_barrier_sync(1, kFWorkerWarps * 32);
+  if (hf == 1) st_l[g * kRows + row] = l_mine;
+  named_barrier_sync(1, kFWorkerWarps * 32);
+  const float l_slot = l_mine + (hf == 0 ? st_l[g * kRows + row] : 0.f);   // meaningful in the first half only
+  if (g == 1) {
+    if (hf == 0) { st_m1[row] = m_mine; st_l1[row] = l_slot; }
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      float o[16];
+      if (have) {
+        tmem_ld16(tO + c * 16, o);
+        tmem_wait_ld();
+      } else {
+#pragma unroll
+        for (int u = 0; u < 16; ++u) o[u] = 0.f;
+      }
+#pragma unroll
+      for (int u = 0; u < 16; ++u) xO[(hf * 64 + c * 16 + u) * 128 + row] = o[u];
+    }
+  }
+  named_barrier_sync(1, kFWorkerWarps * 32);
+  if (g == 0) {
+    const float m1 = st_m1[row], l1 = st_l1[row];
+    const float m = fmaxf(m_mine, m1);
+    const float a0 = (m_mine == -INFINITY) ? 0.f : ex2_approx(m_mine - m);
+    const float a1 = (m1 == -INFINITY) ? 0.f : ex2_approx(m1 - m);
+    const long long o_idx = (long long)blockIdx.x * kRows + row;
+    float* Op = a.part_O + o_idx * kHeadDim + hf * 64;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      float o[16];
+      if (have) {
+        tmem_ld16(tO + c * 16, o);
+        tmem_wait_ld();
+      } else {
+#pragma unroll
+        for (int u = 0; u < 16; ++u) o[u] = 0.f;
+      }
+#pragma unroll
+      for (int u = 0; u < 16; ++u) o[u] = o[u] * a0 + xO[(hf * 64 + c * 16 + u) * 128 + row] * a1;
+#pragma unroll
+      for (int u = 0; u < 16; u += 4)
+        *reinterpret_cast<float4*>(Op + c * 16 + u) = make_float4(o[u], o[u + 1], o[u + 2], o[u + 3]);
+    }
+    if (hf == 0) {
+      a.part_m[o_idx] = m;
+      a.part_l[o_idx] = l_slot * a0 + l1 * a1;
+    }
+  }
+  fence_proxy_async_smem();   // the hand-over buffer lies in the tile ring, which TMA loads refill next
+  tc_fence_before();
 }
 
 // x = hi + mid + lo with three bf16 pieces (24 significant bits).
@@ -528,9 +551,8 @@ __device__ __forceinline__ void load_stage_c(const Ctx& cx, const CUtensorMap* t
 // tensor core (one extra K = 16 step against a block of ones), so with u = exp2(-scale*log2e * S') = 1/A and
 // x = C' + ||v||^2 = ||o - v||^2 the indicator is x * rsqrt(x * (u - 1)^2).
 template <int kW>
-__device__ void phase_c(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tmO, const CUtensorMap* tmAug,
-                        const CUtensorMap* tmK, const CUtensorMap* tmV, int bh, int tile0, int T, int pre,
-                        float (*red)[4][kTile]) {
+__device__ void phase_c_control(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tmO, const CUtensorMap* tmAug,
+                                const CUtensorMap* tmK, const CUtensorMap* tmV, int bh, int tile0, int T, int pre) {
   constexpr int kG = kRows / kW;
   FusedBars* B = cx.B;
   int* abort_flag = cx.abort_flag;
@@ -574,155 +596,242 @@ __device__ void phase_c(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tm
         umma_commit(&B->kv_empty[s]);
       }
     }
-  } else if (warp >= kFFirstWorker && warp < kFFirstWorker + kFWorkerWarps) {
-    const int cgp = (warp - kFFirstWorker) >> 2;     // column group 0..3
-    const int quad = warp & 3;                       // TMEM lane quarter this warp may touch
-    const int t = quad * 32 + lane;
-    const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-    const float ema_decay = a.ema_decay;
-    const float neg_c2 = -a.scale * kLog2e;
-    const float heavy_thr = log2f(1.f / kHeavyA) / neg_c2;   // S' above this <=> A > kHeavyA
-    const float alpha = 1.f - ema_decay;                     // > 0 on this path
-    // Eq. 9 over a run of consecutive window positions i_a..i_b as a Horner chain H = sum c_i I_i decay^(i_b - i),
-    // c_0 = 1/alpha (the seed), c_i = 1: the run contributes alpha * decay^(w-1-i_b) * H.  Even and odd columns
-    // of a run are chained separately in decay^2 (one packed FMA per column pair): H = decay * H_even + H_odd.
-    constexpr int kRun = kW < 32 ? kW : 32;                  // columns of one run inside this warpgroup
-    const int i_first = (cgp * 32) % kW;
-    const float seed_coef = (i_first == 0) ? 1.f / alpha : 1.f;
-    const float fin_scale = alpha * powf(ema_decay, (float)(kW - 1 - (i_first + kRun - 1))) / (float)kG;
-    const f32x2 d2 = f2_make(ema_decay * ema_decay, ema_decay * ema_decay);
-    const f32x2 nc2 = f2_make(neg_c2, neg_c2), m1 = f2_make(-1.f, -1.f), tiny2 = f2_make(1e-36f, 1e-36f);
-    const f32x2 seed2 = f2_make(seed_coef, 1.f);
-    const float* O_head = a.O_f32 + (long long)bh * kRows * kHeadDim;
-    const __nv_bfloat16* V_head = a.V + (long long)b * a.vsb + (long long)h * a.vsh;
-    const float* vn_head = a.vnorm + (long long)bh * a.n_kv;
-    float* I_head = a.I_hat + (long long)bh * n;
-    bool ok = true;
-    const int nt_all = (a.n_kv + kTile - 1) / kTile;
-    // a tile needs exact distances iff some row's largest logit in it reaches that row's M2 - log2(1 / kHeavyA);
-    // every warp checks all 128 rows (lane = rows lane, lane + 32, ...) so that no synchronisation is needed
-    const float* tm_head = a.tile_max + (long long)bh * nt_all * kRows;
-    float m2r[4], tm_next[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      m2r[k] = a.row_M2[(long long)bh * kRows + k * 32 + lane] - log2f(1.f / kHeavyA);
-      tm_next[k] = -INFINITY;
-    }
-    float vn_next = 0.f;
-    if (T > 0) {
-      const int j = tile0 * kTile + t;
-      vn_next = (j < n) ? vn_head[j] : 1.f;
-#pragma unroll
-      for (int k = 0; k < 4; ++k) tm_next[k] = tm_head[(long long)tile0 * kRows + k * 32 + lane];
-    }
+  }
+}
 
-    for (int it = 0; it < T; ++it) {
-      const int s = it & 1;
-      const uint32_t par = (uint32_t)(it >> 1) & 1u;
-      const float vn = vn_next;
-      const bool tile_heavy = __any_sync(0xffffffffu, tm_next[0] > m2r[0] || tm_next[1] > m2r[1] ||
-                                                          tm_next[2] > m2r[2] || tm_next[3] > m2r[3]);
-      if (it + 1 < T) {   // next tile's ||v||^2 and row maxima, well ahead of their use
-        const int jn = (tile0 + it + 1) * kTile + t;
-        vn_next = (jn < n) ? vn_head[jn] : 1.f;
+template <int kW>
+__device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tmO, const CUtensorMap* tmAug,
+                        const CUtensorMap* tmK, const CUtensorMap* tmV, int bh, int tile0, int T, int pre,
+                        float (*red)[4][kTile]) {
+  constexpr int kG = kRows / kW;
+  FusedBars* B = cx.B;
+  int* abort_flag = cx.abort_flag;
+  unsigned int* dev_status = a.dev_status;
+  const int b = bh / a.Hkv, h = bh % a.Hkv;
+  const int warp = cx.warp, lane = cx.lane;
+  const uint32_t tmem = cx.tmem;   // buffer s: S' at s*256, C' at s*256 + 128
+  const int n = a.n;
+
+  const int cgp = (warp - kFFirstWorker) >> 2;     // column group 0..3
+  const int quad = warp & 3;                       // TMEM lane quarter this warp may touch
+  const int t = quad * 32 + lane;
+  const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+  const float ema_decay = a.ema_decay;
+  const float neg_c2 = -a.scale * kLog2e;
+  const float heavy_thr = log2f(1.f / kHeavyA) / neg_c2;   // S' above this <=> A > kHeavyA
+  const float alpha = 1.f - ema_decay;                     // > 0 on this path
+  // Eq. 9 over a run of consecutive window positions i_a..i_b as a Horner chain H = sum c_i I_i decay^(i_b - i),
+  // c_0 = 1/alpha (the seed), c_i = 1: the run contributes alpha * decay^(w-1-i_b) * H.  Even and odd columns
+  // of a run are chained separately in decay^2 (one packed FMA per column pair): H = decay * H_even + H_odd.
+  constexpr int kRun = kW < 32 ? kW : 32;                  // columns of one run inside this warpgroup
+  const int i_first = (cgp * 32) % kW;
+  const float seed_coef = (i_first == 0) ? 1.f / alpha : 1.f;
+  const float fin_scale = alpha * powf(ema_decay, (float)(kW - 1 - (i_first + kRun - 1))) / (float)kG;
+  const f32x2 d2 = f2_make(ema_decay * ema_decay, ema_decay * ema_decay);
+  const f32x2 nc2 = f2_make(neg_c2, neg_c2), m1 = f2_make(-1.f, -1.f), tiny2 = f2_make(1e-36f, 1e-36f);
+  const f32x2 seed2 = f2_make(seed_coef, 1.f);
+  const float* O_head = a.O_f32 + (long long)bh * kRows * kHeadDim;
+  const __nv_bfloat16* V_head = a.V + (long long)b * a.vsb + (long long)h * a.vsh;
+  const float* vn_head = a.vnorm + (long long)bh * a.n_kv;
+  float* I_head = a.I_hat + (long long)bh * n;
+  bool ok = true;
+  const int nt_all = (a.n_kv + kTile - 1) / kTile;
+  // a tile needs exact distances iff some row's largest logit in it reaches that row's M2 - log2(1 / kHeavyA);
+  // every warp checks all 128 rows (lane = rows lane, lane + 32, ...) so that no synchronisation is needed
+  const float* tm_head = a.tile_max + (long long)bh * nt_all * kRows;
+  float m2r[4], tm_next[4];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) tm_next[k] = tm_head[(long long)(tile0 + it + 1) * kRows + k * 32 + lane];
-      }
-      // The shares of the previous tile are summed in a fixed order by warpgroup 0 once all sixteen warps have
-      // stored theirs.  A slot of `red` is rewritten four tiles later, which the two accumulator buffers only
-      // allow after every warp has moved past this point.
-      if (it > 0 && cgp == 0) {
-        const int rs = (it - 1) & 3;
-        ok = ok && mbar_wait(&B->red_full[rs], (uint32_t)((it - 1) >> 2) & 1u, abort_flag, dev_status, kDevTimeout);
-        const int jp = (tile0 + it - 1) * kTile + t;
-        if (ok && jp < n) I_head[jp] = (red[rs][0][t] + red[rs][1][t]) + (red[rs][2][t] + red[rs][3][t]);
-      }
-      ok = ok && mbar_wait(&B->acc_full[s], par, abort_flag, dev_status, kDevTimeout);
-      float tot = 0.f;
-      if (ok) {
-        tc_fence_after();
-        const int j = (tile0 + it) * kTile + t;
-        const uint32_t tS = tmem + (uint32_t)s * 256u + lane_base + (uint32_t)cgp * 32u, tC = tS + 128u;
-        // ||o - v||^2 = C' + ||v||^2 is formed with ||v||^2 raised by 2^-16 of itself: a bias of ~1e-5 that keeps
-        // the sum positive when the expansion cancels, so that no clamp is needed.
-        const float vnb = vn * 1.0000152587890625f;
-        const f32x2 vn2 = f2_make(vnb, vnb);
-        f32x2 h2 = f2_make(0.f, 0.f);
-        if (!tile_heavy) {
-          float sv0[16], cv0[16], sv1[16], cv1[16];
-          tmem_ld16(tS, sv0);
-          tmem_ld16(tC, cv0);
-          tmem_wait_ld();
-          tmem_ld16(tS + 16, sv1);   // the second half of the columns travels while the first is worked on
-          tmem_ld16(tC + 16, cv1);
+  for (int k = 0; k < 4; ++k) {
+    m2r[k] = a.row_M2[(long long)bh * kRows + k * 32 + lane] - log2f(1.f / kHeavyA);
+    tm_next[k] = -INFINITY;
+  }
+  float vn_next = 0.f;
+  if (T > 0) {
+    const int j = tile0 * kTile + t;
+    vn_next = (j < n) ? vn_head[j] : 1.f;
 #pragma unroll
-          for (int c = 0; c < 2; ++c) {
-            const float* sv = c == 0 ? sv0 : sv1;
-            const float* cv = c == 0 ? cv0 : cv1;
-            if (c == 1) {
-              tmem_wait_ld();
-              // every tensor-memory read of this tile is done: the MMA warp may refill the accumulators
-              tc_fence_before();
-              __syncwarp();
-              if (lane == 0) mbar_arrive(&B->acc_empty[s]);
-            }
+    for (int k = 0; k < 4; ++k) tm_next[k] = tm_head[(long long)tile0 * kRows + k * 32 + lane];
+  }
+
+  for (int it = 0; it < T; ++it) {
+    const int s = it & 1;
+    const uint32_t par = (uint32_t)(it >> 1) & 1u;
+    const float vn = vn_next;
+    const bool tile_heavy = __any_sync(0xffffffffu, tm_next[0] > m2r[0] || tm_next[1] > m2r[1] ||
+                                                        tm_next[2] > m2r[2] || tm_next[3] > m2r[3]);
+    if (it + 1 < T) {   // next tile's ||v||^2 and row maxima, well ahead of their use
+      const int jn = (tile0 + it + 1) * kTile + t;
+      vn_next = (jn < n) ? vn_head[jn] : 1.f;
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              const f32x2 nt = f2_mul(f2_make(sv[2 * q], sv[2 * q + 1]), nc2);
-              const f32x2 um = f2_add(f2_make(ex2_approx(f2_lo(nt)), ex2_approx(f2_hi(nt))), m1);   // 1/A - 1
-              const f32x2 x = f2_add(f2_make(cv[2 * q], cv[2 * q + 1]), vn2);                       // ||o - v||^2
-              const f32x2 bq = f2_fma(f2_mul(x, um), um, tiny2);                                    // x (1/A - 1)^2
-              f32x2 Iq = f2_mul(x, f2_make(rsqrt_approx(f2_lo(bq)), rsqrt_approx(f2_hi(bq))));
-              if (q == 0 && (c * 16) % kRun == 0) Iq = f2_mul(Iq, seed2);
-              h2 = f2_fma(h2, d2, Iq);
-            }
-            if ((c * 16 + 16) % kRun == 0) {   // end of a run
-              tot += fmaf(f2_lo(h2), ema_decay, f2_hi(h2));
-              h2 = f2_make(0.f, 0.f);
-            }
-          }
-        } else {
-          // rare: the tile may hold large attention weights; those entries take the exact distance
-#pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
-            float sv[8], cv[8], I[8];
-            tmem_ld8(tS + c * 8, sv);
-            tmem_ld8(tC + c * 8, cv);
+      for (int k = 0; k < 4; ++k) tm_next[k] = tm_head[(long long)(tile0 + it + 1) * kRows + k * 32 + lane];
+    }
+    // The shares of the previous tile are summed in a fixed order by warpgroup 0 once all sixteen warps have
+    // stored theirs.  A slot of `red` is rewritten four tiles later, which the two accumulator buffers only
+    // allow after every warp has moved past this point.
+    if (it > 0 && cgp == 0) {
+      const int rs = (it - 1) & 3;
+      ok = ok && mbar_wait(&B->red_full[rs], (uint32_t)((it - 1) >> 2) & 1u, abort_flag, dev_status, kDevTimeout);
+      const int jp = (tile0 + it - 1) * kTile + t;
+      if (ok && jp < n) I_head[jp] = (red[rs][0][t] + red[rs][1][t]) + (red[rs][2][t] + red[rs][3][t]);
+    }
+    ok = ok && mbar_wait(&B->acc_full[s], par, abort_flag, dev_status, kDevTimeout);
+    float tot = 0.f;
+    if (ok) {
+      tc_fence_after();
+      const int j = (tile0 + it) * kTile + t;
+      const uint32_t tS = tmem + (uint32_t)s * 256u + lane_base + (uint32_t)cgp * 32u, tC = tS + 128u;
+      // ||o - v||^2 = C' + ||v||^2 is formed with ||v||^2 raised by 2^-16 of itself: a bias of ~1e-5 that keeps
+      // the sum positive when the expansion cancels, so that no clamp is needed.
+      const float vnb = vn * 1.0000152587890625f;
+      const f32x2 vn2 = f2_make(vnb, vnb);
+      f32x2 h2 = f2_make(0.f, 0.f);
+      if (!tile_heavy) {
+        float sv0[16], cv0[16], sv1[16], cv1[16];
+        tmem_ld16(tS, sv0);
+        tmem_ld16(tC, cv0);
+        tmem_wait_ld();
+        tmem_ld16(tS + 16, sv1);   // the second half of the columns travels while the first is worked on
+        tmem_ld16(tC + 16, cv1);
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          const float* sv = c == 0 ? sv0 : sv1;
+          const float* cv = c == 0 ? cv0 : cv1;
+          if (c == 1) {
             tmem_wait_ld();
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-              const float um = ex2_approx(sv[u] * neg_c2) - 1.f;
-              float x = cv[u] + vnb;
-              if (sv[u] > heavy_thr && j < n)
-                x = exact_dist2(O_head + (cgp * 32 + c * 8 + u) * kHeadDim, V_head + (long long)j * a.vsn);
-              I[u] = x * rsqrt_approx(fmaf(x * um, um, 1e-36f));
-            }
-            if ((c * 8) % kRun == 0) I[0] *= seed_coef;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) h2 = f2_fma(h2, d2, f2_make(I[2 * q], I[2 * q + 1]));
-            if ((c * 8 + 8) % kRun == 0) {   // end of a run
-              tot += fmaf(f2_lo(h2), ema_decay, f2_hi(h2));
-              h2 = f2_make(0.f, 0.f);
-            }
+            // every tensor-memory read of this tile is done: the MMA warp may refill the accumulators
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&B->acc_empty[s]);
           }
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&B->acc_empty[s]);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const f32x2 nt = f2_mul(f2_make(sv[2 * q], sv[2 * q + 1]), nc2);
+            const f32x2 um = f2_add(f2_make(ex2_approx(f2_lo(nt)), ex2_approx(f2_hi(nt))), m1);   // 1/A - 1
+            const f32x2 x = f2_add(f2_make(cv[2 * q], cv[2 * q + 1]), vn2);                       // ||o - v||^2
+            const f32x2 bq = f2_fma(f2_mul(x, um), um, tiny2);                                    // x (1/A - 1)^2
+            f32x2 Iq = f2_mul(x, f2_make(rsqrt_approx(f2_lo(bq)), rsqrt_approx(f2_hi(bq))));
+            if (q == 0 && (c * 16) % kRun == 0) Iq = f2_mul(Iq, seed2);
+            h2 = f2_fma(h2, d2, Iq);
+          }
+          if ((c * 16 + 16) % kRun == 0) {   // end of a run
+            tot += fmaf(f2_lo(h2), ema_decay, f2_hi(h2));
+            h2 = f2_make(0.f, 0.f);
+          }
         }
       } else {
+        // rare: the tile may hold large attention weights; those entries take the exact distance
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          float sv[8], cv[8], I[8];
+          tmem_ld8(tS + c * 8, sv);
+          tmem_ld8(tC + c * 8, cv);
+          tmem_wait_ld();
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const float um = ex2_approx(sv[u] * neg_c2) - 1.f;
+            float x = cv[u] + vnb;
+            if (sv[u] > heavy_thr && j < n)
+              x = exact_dist2(O_head + (cgp * 32 + c * 8 + u) * kHeadDim, V_head + (long long)j * a.vsn);
+            I[u] = x * rsqrt_approx(fmaf(x * um, um, 1e-36f));
+          }
+          if ((c * 8) % kRun == 0) I[0] *= seed_coef;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) h2 = f2_fma(h2, d2, f2_make(I[2 * q], I[2 * q + 1]));
+          if ((c * 8 + 8) % kRun == 0) {   // end of a run
+            tot += fmaf(f2_lo(h2), ema_decay, f2_hi(h2));
+            h2 = f2_make(0.f, 0.f);
+          }
+        }
+        tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&B->acc_empty[s]);
       }
-      red[it & 3][cgp][t] = tot * fin_scale;
+    } else {
       __syncwarp();
-      if (lane == 0) mbar_arrive(&B->red_full[it & 3]);
+      if (lane == 0) mbar_arrive(&B->acc_empty[s]);
     }
-    if (T > 0 && cgp == 0) {
-      const int rs = (T - 1) & 3;
-      ok = ok && mbar_wait(&B->red_full[rs], (uint32_t)((T - 1) >> 2) & 1u, abort_flag, dev_status, kDevTimeout);
-      const int jl = (tile0 + T - 1) * kTile + t;
-      if (ok && jl < n) I_head[jl] = (red[rs][0][t] + red[rs][1][t]) + (red[rs][2][t] + red[rs][3][t]);
+    red[it & 3][cgp][t] = tot * fin_scale;
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&B->red_full[it & 3]);
+  }
+  if (T > 0 && cgp == 0) {
+    const int rs = (T - 1) & 3;
+    ok = ok && mbar_wait(&B->red_full[rs], (uint32_t)((T - 1) >> 2) & 1u, abort_flag, dev_status, kDevTimeout);
+    const int jl = (tile0 + T - 1) * kTile + t;
+    if (ok && jl < n) I_head[jl] = (red[rs][0][t] + red[rs][1][t]) + (red[rs][2][t] + red[rs][3][t]);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+struct Plan {
+  int group, rank, tile0, T1, T2;
+};
+
+// The two role loops below run through the same sequence of CTA-wide synchronisations: per head a barrier
+// re-initialisation (from the second head on), phase A, the prefetch point, group barrier, phase B, group
+// barrier, phase C, and a closing __syncthreads.
+
+// Warps 0-3: TMA producer, MMA issuer, the two ||v||^2 warps; thread 0 also runs the group barriers.
+template <int kW>
+__device__ void control_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, const CUtensorMap* tmQ,
+                             const CUtensorMap* tmK, const CUtensorMap* tmV, const CUtensorMap* tmO,
+                             const CUtensorMap* tmAug, FusedBars* bars, int* abort_flag, int* go) {
+  unsigned int* counter = a.counters + pl.group;
+  unsigned int epoch = 0;
+  for (int bh = pl.group; bh < a.BH; bh += a.groups) {
+    if (bh != pl.group) {   // fresh barriers for every head: nothing is in flight between two __syncthreads
+      if (threadIdx.x == 0) init_bars(bars, false);
+      __syncthreads();
     }
+    phase_a_control(cx, a, tmQ, tmK, tmV, bh, pl.rank, pl.tile0, pl.T1);
+    // Phase A no longer needs the tile ring: request phase C's first two K/V stages now, so that they arrive
+    // while the group merges its partials (K and V are inputs; only O' depends on the merge).
+    __syncthreads();
+    const int pre = pl.T2 < 2 ? pl.T2 : 2;
+    if (threadIdx.x == 0)
+      for (int it = 0; it < pre; ++it)
+        load_stage_c(cx, tmK, tmV, bh / a.Hkv, bh % a.Hkv, (pl.tile0 + it) * kTile, it);
+    if (!group_barrier(counter, (++epoch) * (unsigned int)a.cpg, abort_flag, go, a.dev_status)) break;
+    // phase B belongs to the worker warps
+    if (!group_barrier(counter, (++epoch) * (unsigned int)a.cpg, abort_flag, go, a.dev_status)) break;
+    tc_fence_after();
+    phase_c_control<kW>(cx, a, tmO, tmAug, tmK, tmV, bh, pl.tile0, pl.T2, pre);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+  }
+}
+
+// Warps 4-19: softmax in phase A, the merge of the partials in phase B, the indicator epilogue in phase C.
+template <int kW>
+__device__ void worker_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, const CUtensorMap* tmQ,
+                            const CUtensorMap* tmK, const CUtensorMap* tmV, const CUtensorMap* tmO,
+                            const CUtensorMap* tmAug, int* go, float (*red)[4][kTile]) {
+  for (int bh = pl.group; bh < a.BH; bh += a.groups) {
+    if (bh != pl.group) __syncthreads();
+    phase_a_worker(cx, a, tmQ, tmK, tmV, bh, pl.rank, pl.tile0, pl.T1);
+    __syncthreads();
+    if (!group_barrier_follow(go)) break;
+    {
+      const int wq = cx.warp - kFFirstWorker;
+      const int rows_max = (kRows + a.cpg - 1) / a.cpg;          // rows of the busiest CTA of the group
+      int wpr = kFWorkerWarps;                                    // warps per row: 16, 8, 4, 2 or 1
+      while (wpr > 1 && kFWorkerWarps / wpr < rows_max) wpr >>= 1;
+      const int rows_at_once = kFWorkerWarps / wpr;
+      float (*xch)[kHeadDim + 4] = reinterpret_cast<float (*)[kHeadDim + 4]>(cx.gen_base + kOffAug);
+      for (int k0 = 0; k0 < rows_max; k0 += rows_at_once) {
+        const int r = pl.rank + (k0 + wq / wpr) * a.cpg;
+        combine_rows(a, bh, pl.group, r < kRows ? r : -1, wq % wpr, wpr, wq, cx.lane, xch);
+        named_barrier_sync(2, kFWorkerWarps * 32);   // the exchange buffer is reused by the next batch of rows
+      }
+      fence_proxy_async_smem();   // the exchange buffer is overwritten by a TMA load in phase C
+    }
+    if (!group_barrier_follow(go)) break;
+    tc_fence_after();
+    phase_c_worker<kW>(cx, a, tmO, tmAug, tmK, tmV, bh, pl.tile0, pl.T2, 0, red);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
   }
 }
 
@@ -735,7 +844,7 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) FusedBars bars;
   __shared__ uint32_t tmem_slot;
-  __shared__ int abort_flag;
+  __shared__ int abort_flag, go_flag;
   __shared__ float sm_stats[6 * kRows];
   __shared__ float red[4][4][kTile];   // [tile & 3][warpgroup][token]: each warpgroup's share of the score
 
@@ -771,54 +880,24 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   cx.tmem = tmem_slot;
-
   // the same split of the token tiles in both phases (phase C covers only the scored rows)
+  Plan pl;
+  pl.group = group;
+  pl.rank = rank;
   const int nt1 = (a.n_kv + kTile - 1) / kTile, nt2 = (a.n + kTile - 1) / kTile;
   const int per = (nt1 + a.cpg - 1) / a.cpg;
-  const int tile0 = rank * per;
-  const int T1 = max(0, min(nt1, tile0 + per) - tile0);
-  const int T2 = max(0, min(nt2, tile0 + per) - tile0);
-  unsigned int* counter = a.counters + group;
-  unsigned int epoch = 0;
-  bool alive = true;
+  pl.tile0 = rank * per;
+  pl.T1 = max(0, min(nt1, pl.tile0 + per) - pl.tile0);
+  pl.T2 = max(0, min(nt2, pl.tile0 + per) - pl.tile0);
 
-  for (int bh = group; bh < a.BH && alive; bh += a.groups) {
-    if (bh != group) {   // fresh barriers for every phase: nothing is in flight between two __syncthreads
-      if (threadIdx.x == 0) init_bars(&bars, false);
-      __syncthreads();
-    }
-    phase_a(cx, a, &tmQ, &tmK, &tmV, bh, rank, tile0, T1);
-    // Phase A no longer needs the tile ring: request phase C's first two K/V stages now, so that they arrive
-    // while the group merges its partials (K and V are inputs; only O' depends on the merge).
-    __syncthreads();
-    const int pre = T2 < 2 ? T2 : 2;
-    if (threadIdx.x == 0)
-      for (int it = 0; it < pre; ++it)
-        load_stage_c(cx, &tmK, &tmV, bh / a.Hkv, bh % a.Hkv, (tile0 + it) * kTile, it);
-    alive = group_barrier(counter, (++epoch) * (unsigned int)a.cpg, &abort_flag, a.dev_status);
-    if (!alive) break;
-    // ---- phase B: rows rank, rank + cpg, ... of the head; the sixteen worker warps share them ----
-    if (cx.warp >= kFFirstWorker && cx.warp < kFFirstWorker + kFWorkerWarps) {
-      const int wq = cx.warp - kFFirstWorker;
-      const int rows_max = (kRows + a.cpg - 1) / a.cpg;          // rows of the busiest CTA of the group
-      int wpr = kFWorkerWarps;                                    // warps per row: 16, 8, 4, 2 or 1
-      while (wpr > 1 && kFWorkerWarps / wpr < rows_max) wpr >>= 1;
-      const int rows_at_once = kFWorkerWarps / wpr;
-      float (*xch)[kHeadDim + 4] = reinterpret_cast<float (*)[kHeadDim + 4]>(cx.gen_base + kOffAug);
-      for (int k0 = 0; k0 < rows_max; k0 += rows_at_once) {
-        const int r = rank + (k0 + wq / wpr) * a.cpg;
-        combine_rows(a, bh, group, r < kRows ? r : -1, wq % wpr, wpr, wq, cx.lane, xch);
-        named_barrier_sync(2, kFWorkerWarps * 32);   // the exchange buffer is reused by the next batch of rows
-      }
-      fence_proxy_async_smem();   // the exchange buffer is overwritten by a TMA load in phase C
-    }
-    alive = group_barrier(counter, (++epoch) * (unsigned int)a.cpg, &abort_flag, a.dev_status);
-    if (!alive) break;
-    tc_fence_after();
-    phase_c<kW>(cx, a, &tmO, &tmAug, &tmK, &tmV, bh, tile0, T2, pre, red);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
+  // Each role's code sits behind its own register-budget change, so that the sixteen worker warps can be
+  // compiled for more registers than the launch gives every thread.
+  if (cx.warp < kFFirstWorker) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kFRegsControl));
+    control_main<kW>(cx, a, pl, &tmQ, &tmK, &tmV, &tmO, &tmAug, &bars, &abort_flag, &go_flag);
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kFRegsWorker));
+    worker_main<kW>(cx, a, pl, &tmQ, &tmK, &tmV, &tmO, &tmAug, &go_flag, red);
   }
 
   tc_fence_before();
@@ -871,7 +950,23 @@ cudaError_t tc_init(void** state) {
   return cudaSuccess;
 }
 
+// The register split inside the kernel assumes that it was compiled for exactly kFRegsLaunch registers per thread.
+template <typename K>
+static cudaError_t check_launch_regs(K kernel) {
+  cudaFuncAttributes fa;
+  cudaError_t e = cudaFuncGetAttributes(&fa, kernel);
+  if (e != cudaSuccess) return e;
+  return fa.numRegs == kFRegsLaunch ? cudaSuccess : cudaErrorInvalidConfiguration;
+}
+
 cudaError_t tc_fused_init() {
+  {
+    cudaError_t c = check_launch_regs(tc_fused_kernel<16>);
+    if (c == cudaSuccess) c = check_launch_regs(tc_fused_kernel<32>);
+    if (c == cudaSuccess) c = check_launch_regs(tc_fused_kernel<64>);
+    if (c == cudaSuccess) c = check_launch_regs(tc_fused_kernel<128>);
+    if (c != cudaSuccess) return c;
+  }
   cudaError_t e = cudaFuncSetAttribute(tc_fused_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmem);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fused_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmem);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fused_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmem);
