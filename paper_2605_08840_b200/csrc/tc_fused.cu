@@ -545,7 +545,8 @@ __device__ __forceinline__ void load_stage_c(const Ctx& cx, const CUtensorMap* t
 }
 
 // ------------------------------------------------------------------------------------------------
-// Phase C: this CTA's share [tile0, tile0 + T) of the scored rows of one head.  Warp 0 loads, warp 1 issues the
+// Phase C: this CTA's share [tile0, tile0 + T) of the scored rows of one head, walked from the last tile to the
+// first (the tiles phase A read last are the likeliest to still be in L2).  Warp 0 loads, warp 1 issues the
 // MMAs, the sixteen worker warps are four epilogue warpgroups (thread = token, warpgroup c = accumulator columns
 // [32c, 32c + 32)).  Q is still in shared memory from phase A.  The per-query-row constants ride through the
 // tensor core (one extra K = 16 step against a block of ones), so with u = exp2(-scale*log2e * S') = 1/A and
@@ -572,7 +573,7 @@ __device__ void phase_c_control(const Ctx& cx, const FusedArgs& a, const CUtenso
       for (int it = pre; it < T; ++it) {   // the first `pre` tiles were requested before the group barriers
         const int s = it & 1;
         if (it >= 2 && !mbar_wait(&B->kv_empty[s], ((it >> 1) - 1) & 1, abort_flag, dev_status, kDevTimeout)) break;
-        load_stage_c(cx, tmK, tmV, b, h, (tile0 + it) * kTile, s);
+        load_stage_c(cx, tmK, tmV, b, h, (tile0 + T - 1 - it) * kTile, s);
       }
     }
   } else if (warp == 1) {
@@ -647,10 +648,10 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
   }
   float vn_next = 0.f;
   if (T > 0) {
-    const int j = tile0 * kTile + t;
+    const int j = (tile0 + T - 1) * kTile + t;
     vn_next = (j < n) ? vn_head[j] : 1.f;
 #pragma unroll
-    for (int k = 0; k < 4; ++k) tm_next[k] = tm_head[(long long)tile0 * kRows + k * 32 + lane];
+    for (int k = 0; k < 4; ++k) tm_next[k] = tm_head[(long long)(tile0 + T - 1) * kRows + k * 32 + lane];
   }
 
   for (int it = 0; it < T; ++it) {
@@ -660,10 +661,10 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
     const bool tile_heavy = __any_sync(0xffffffffu, tm_next[0] > m2r[0] || tm_next[1] > m2r[1] ||
                                                         tm_next[2] > m2r[2] || tm_next[3] > m2r[3]);
     if (it + 1 < T) {   // next tile's ||v||^2 and row maxima, well ahead of their use
-      const int jn = (tile0 + it + 1) * kTile + t;
+      const int jn = (tile0 + T - 2 - it) * kTile + t;
       vn_next = (jn < n) ? vn_head[jn] : 1.f;
 #pragma unroll
-      for (int k = 0; k < 4; ++k) tm_next[k] = tm_head[(long long)(tile0 + it + 1) * kRows + k * 32 + lane];
+      for (int k = 0; k < 4; ++k) tm_next[k] = tm_head[(long long)(tile0 + T - 2 - it) * kRows + k * 32 + lane];
     }
     // The shares of the previous tile are summed in a fixed order by warpgroup 0 once all sixteen warps have
     // stored theirs.  A slot of `red` is rewritten four tiles later, which the two accumulator buffers only
@@ -671,14 +672,14 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
     if (it > 0 && cgp == 0) {
       const int rs = (it - 1) & 3;
       ok = ok && mbar_wait(&B->red_full[rs], (uint32_t)((it - 1) >> 2) & 1u, abort_flag, dev_status, kDevTimeout);
-      const int jp = (tile0 + it - 1) * kTile + t;
+      const int jp = (tile0 + T - it) * kTile + t;
       if (ok && jp < n) I_head[jp] = (red[rs][0][t] + red[rs][1][t]) + (red[rs][2][t] + red[rs][3][t]);
     }
     ok = ok && mbar_wait(&B->acc_full[s], par, abort_flag, dev_status, kDevTimeout);
     float tot = 0.f;
     if (ok) {
       tc_fence_after();
-      const int j = (tile0 + it) * kTile + t;
+      const int j = (tile0 + T - 1 - it) * kTile + t;
       const uint32_t tS = tmem + (uint32_t)s * 256u + lane_base + (uint32_t)cgp * 32u, tC = tS + 128u;
       // ||o - v||^2 = C' + ||v||^2 is formed with ||v||^2 raised by 2^-16 of itself: a bias of ~1e-5 that keeps
       // the sum positive when the expansion cancels, so that no clamp is needed.
@@ -757,7 +758,7 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
   if (T > 0 && cgp == 0) {
     const int rs = (T - 1) & 3;
     ok = ok && mbar_wait(&B->red_full[rs], (uint32_t)((T - 1) >> 2) & 1u, abort_flag, dev_status, kDevTimeout);
-    const int jl = (tile0 + T - 1) * kTile + t;
+    const int jl = tile0 * kTile + t;   // the last tile processed is the first of the share
     if (ok && jl < n) I_head[jl] = (red[rs][0][t] + red[rs][1][t]) + (red[rs][2][t] + red[rs][3][t]);
   }
 }
@@ -790,7 +791,7 @@ __device__ void control_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, 
     const int pre = pl.T2 < 2 ? pl.T2 : 2;
     if (threadIdx.x == 0)
       for (int it = 0; it < pre; ++it)
-        load_stage_c(cx, tmK, tmV, bh / a.Hkv, bh % a.Hkv, (pl.tile0 + it) * kTile, it);
+        load_stage_c(cx, tmK, tmV, bh / a.Hkv, bh % a.Hkv, (pl.tile0 + pl.T2 - 1 - it) * kTile, it);
     if (!group_barrier(counter, (++epoch) * (unsigned int)a.cpg, abort_flag, go, a.dev_status)) break;
     // phase B belongs to the worker warps
     if (!group_barrier(counter, (++epoch) * (unsigned int)a.cpg, abort_flag, go, a.dev_status)) break;
