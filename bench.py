@@ -246,8 +246,9 @@ def main():
     def step():
         handle.evict(shape, Q, K, V, case.ema_decay, pool, case.budget, indices, K_out, V_out, ws)
 
-    # the tensor-core path runs pass 1, the merge and pass 2 in one launch; pooling runs inside the select kernel
-    kernel_ids = {"score": rk.KERNEL_PASS2, "pool_select": rk.KERNEL_SELECT, "compact": rk.KERNEL_COMPACT}
+    # the tensor-core path runs pass 1, the merge and pass 2 in one launch; pooling and the gather run inside the
+    # select kernel
+    kernel_ids = {"score": rk.KERNEL_PASS2, "pool_select_compact": rk.KERNEL_SELECT}
     prof = {}
     for name, kid in kernel_ids.items():
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

@@ -57,7 +57,8 @@ cudaError_t launch_adaptive_params(const Problem& p, const Workspace& ws, int bu
   if (Bp > p.n) Bp = p.n;
   const int rows = p.batch * p.Hq * p.w;
   *n_launches = 0;
-  cudaError_t e = launch_select(rows, p.n, p.n, Bp, nullptr, nullptr, 1, 0, ws.I_raw, ws.adaptive_idx, nullptr, st);
+  cudaError_t e = launch_select(rows, p.n, p.n, Bp, nullptr, nullptr, 1, 0, ws.I_raw, ws.adaptive_idx, nullptr, nullptr, nullptr,
+                                nullptr, nullptr, nullptr, st);
   if (e != cudaSuccess) return e;
   ++*n_launches;
   zero_sums_kernel<<<(2 * p.BH + 127) / 128, 128, 0, st>>>(ws.adaptive_sums, 2 * p.BH);

@@ -40,6 +40,17 @@ __device__ __forceinline__ unsigned int float_key(float x) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// Optional gather fused into the select kernel (all pointers null: indices only).  K, V addressed by element strides;
+// K_out, V_out [rows, keep, row_chunks * 16 bytes] contiguous.
+struct GatherArgs {
+  const unsigned char* K;
+  const unsigned char* V;
+  unsigned char* K_out;
+  unsigned char* V_out;
+  long long ksb, ksh, ksn, vsb, vsh, vsn;   // element strides
+  int Hkv, esize, row_chunks;
+};
+
 constexpr int kSelThreads = 1024;
 constexpr int kSelBins = 256;                // 8-bit digits
 constexpr int kSelMaxSmemKeys = 44 * 1024;   // keys of one CTA's slice kept in shared memory (176 KB)
@@ -83,7 +94,7 @@ __device__ __forceinline__ unsigned int block_inclusive_scan(unsigned int v, uns
 __global__ void __launch_bounds__(kSelThreads, 1)
 select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const int* __restrict__ pool, int W,
               int gamma, float* scores, int32_t* __restrict__ indices, int32_t* __restrict__ pool_used, int per,
-              int use_smem, int stage_taps) {
+              int use_smem, int stage_taps, GatherArgs ga) {
   cg::cluster_group cluster = cg::this_cluster();
   const unsigned int CS = cluster.num_blocks(), rank = cluster.block_rank();
   const int row = blockIdx.x / CS;
@@ -144,6 +155,22 @@ select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const 
 
   if (keep >= n_kv) {   // budget covers everything: identity (uniform over the cluster)
     for (int jj = tid; jj < cnt; jj += kSelThreads) dst[j0 + jj] = (int32_t)(j0 + jj);
+    if (ga.K) {
+      const int b = row / ga.Hkv, h = row % ga.Hkv;
+      const unsigned char* Kh = ga.K + ((long long)b * ga.ksb + (long long)h * ga.ksh) * ga.esize;
+      const unsigned char* Vh = ga.V + ((long long)b * ga.vsb + (long long)h * ga.vsh) * ga.esize;
+      const int rc2 = 2 * ga.row_chunks;
+      for (long long e = tid; e < (long long)cnt * rc2; e += kSelThreads) {
+        const long long r = e / rc2;
+        const int c = (int)(e - r * rc2);
+        const bool isV = c >= ga.row_chunks;
+        const int chunk = isV ? c - ga.row_chunks : c;
+        const long long j = j0 + r;
+        const uint4* src = reinterpret_cast<const uint4*>((isV ? Vh + j * ga.vsn * ga.esize : Kh + j * ga.ksn * ga.esize)) + chunk;
+        uint4* out = reinterpret_cast<uint4*>((isV ? ga.V_out : ga.K_out) + ((long long)row * keep + j) * ga.row_chunks * 16) + chunk;
+        *out = __ldg(src);
+      }
+    }
     return;
   }
 
@@ -285,6 +312,33 @@ select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const 
     run_gt += __popc(mgt);
     run_eq += __popc(meq);
   }
+  if (ga.K) {
+    // ---- gather the rows this CTA selected: its indices are the contiguous run dst[first, first + mine) ----
+    unsigned int g_before = 0, e_before = 0;
+    for (unsigned int r = 0; r < rank; ++r) {
+      const unsigned int* rc = cluster.map_shared_rank(cta_counts, r);
+      g_before += rc[0];
+      e_before += rc[1];
+    }
+    const unsigned int first = g_before + min(e_before, need_eq);
+    const unsigned int mine = cta_counts[0] + (min(e_before + cta_counts[1], need_eq) - min(e_before, need_eq));
+    __syncthreads();   // the indices written above are visible to the whole CTA
+    const int b = row / ga.Hkv, h = row % ga.Hkv;
+    const unsigned char* Kh = ga.K + ((long long)b * ga.ksb + (long long)h * ga.ksh) * ga.esize;
+    const unsigned char* Vh = ga.V + ((long long)b * ga.vsb + (long long)h * ga.vsh) * ga.esize;
+    const long long out_row0 = (long long)row * keep;
+    const int rc2 = 2 * ga.row_chunks;
+    for (unsigned int e = tid; e < mine * (unsigned int)rc2; e += kSelThreads) {
+      const unsigned int r = e / rc2;
+      const int c = (int)(e - r * rc2);
+      const bool isV = c >= ga.row_chunks;
+      const int chunk = isV ? c - ga.row_chunks : c;
+      const long long j = dst[first + r];
+      const uint4* src = reinterpret_cast<const uint4*>((isV ? Vh + j * ga.vsn * ga.esize : Kh + j * ga.ksn * ga.esize)) + chunk;
+      uint4* out = reinterpret_cast<uint4*>((isV ? ga.V_out : ga.K_out) + (out_row0 + first + r) * ga.row_chunks * 16) + chunk;
+      *out = __ldg(src);
+    }
+  }
   cluster.sync();   // shared memory stays alive until every peer has read cta_counts
 }
 
@@ -328,7 +382,16 @@ cudaError_t launch_pool(const Problem& p, const Workspace& ws, const int* pool_d
 // rows x n_kv scores -> rows x min(budget, n_kv) indices.  I_hat non-null: pool first (n scored rows per row of
 // I_hat, window from pool_dev or (W, gamma)) and write the pooled scores.
 cudaError_t launch_select(int rows, int n, int n_kv, int budget, const float* I_hat, const int* pool_dev, int W,
-                          int gamma, float* scores, int32_t* indices, int32_t* pool_used, cudaStream_t st) {
+                          int gamma, float* scores, int32_t* indices, int32_t* pool_used, const Problem* gather,
+                          const void* K, const void* V, void* K_out, void* V_out, cudaStream_t st) {
+  GatherArgs ga{};
+  if (gather) {
+    ga.K = (const unsigned char*)K; ga.V = (const unsigned char*)V;
+    ga.K_out = (unsigned char*)K_out; ga.V_out = (unsigned char*)V_out;
+    ga.ksb = gather->ksb; ga.ksh = gather->ksh; ga.ksn = gather->ksn;
+    ga.vsb = gather->vsb; ga.vsh = gather->vsh; ga.vsn = gather->vsn;
+    ga.Hkv = gather->Hkv; ga.esize = gather->dtype == RESTKV_BF16 ? 2 : 4; ga.row_chunks = gather->d * ga.esize / 16;
+  }
   const int keep = budget < n_kv ? budget : n_kv;
   int CS = n_kv > 4096 ? 8 : 1;
   cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -352,7 +415,7 @@ cudaError_t launch_select(int rows, int n, int n_kv, int budget, const float* I_
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, select_kernel, n, n_kv, keep, I_hat, pool_dev, W, gamma, scores, indices, pool_used,
-                            per, use_smem, stage_taps);
+                            per, use_smem, stage_taps, ga);
 }
 
 cudaError_t launch_compact(const Problem& p, const void* K, const void* V, const int32_t* indices, int n_sel,
