@@ -1,15 +1,16 @@
-// Head-sequential tensor-core score kernel for sm_100a (bf16, head_dim 128, w * group = 128 query rows).
+// Persistent tensor-core score kernel for sm_100a (bf16, head_dim 128, w * group = 128 query rows).
 //
-// One persistent CTA per SM.  The CTAs are divided into groups; a group takes one (batch, KV head) at a time and
-// runs, back to back,
+// One CTA per SM.  The CTAs are divided into groups; a group takes one (batch, KV head) at a time and runs, back
+// to back,
 //   phase A  (Eq. 3)    every CTA of the group: S = Q K^T, online softmax, O += P V over its share of the tiles
-//   phase B             the group's partial (m, l, O) are merged row by row (one warp per query row)
+//   phase B             the group's partial (m, l, O) are merged row by row
 //   phase C  (Eq. 7-9)  every CTA: S^T = K Q^T, C^T = V (-2 O)^T over its share of the tiles, indicator, EMA,
 //                       group mean
-// so that phase C finds the head's K and V in L2 (a head is 64 MiB at 128k tokens; L2 holds 126 MB) and HBM sees
-// each row once.  The CTAs of a group meet at two counter barriers per head (after A and after B); different
-// groups never wait for one another.  Every wait is bounded: a wait that runs out sets the sticky timeout bit,
-// and the CTA skips the rest of its work and still releases its tensor memory.
+// The CTAs of a group meet at two counter barriers per head (after A and after B); different groups never wait
+// for one another.  By default there are as many groups as heads (every head in flight, one round); with
+// reuse_l2 only as many heads are in flight as fit in L2, so that phase C re-reads K and V from there.
+// Every wait on data is bounded: a wait that runs out sets the sticky timeout bit, and the CTA skips the rest of
+// its work and still releases its tensor memory.
 #include "tc_common.cuh"
 
 namespace restkv {
@@ -141,11 +142,11 @@ __device__ __forceinline__ uint32_t k_slot_off(int i) { return kOffRing + (uint3
 __device__ __forceinline__ uint32_t v_slot_off(int i) { return i < 2 ? kOffRing + (uint32_t)(2 + i) * kTileBytes : kOffO; }
 
 // ------------------------------------------------------------------------------------------------
-// Phase A: this CTA's share [tile0, tile0 + T) of one head.  Warp 0 loads, warp 1 issues the MMAs, worker warps
-// 0-7 are two softmax warpgroups (thread = query row; warpgroup g owns tiles g, g+2, ... with its own running
-// maximum and its own O accumulator), worker warps 8-15 reduce ||v_j||^2 of the tokens from the V tiles.
-// Tensor memory: S_g at g*128 (bf16 P_g overwrites its first 64 columns), O_g at 256 + g*128.
-// At the end the two warpgroups' (m, l, O) are merged and written as the CTA's partial.
+// Phase A: this CTA's share [tile0, tile0 + T) of one head.
+// Control warps: warp 0 loads (K ring of 2 slots, V ring of 3), warp 1 issues the MMAs (S(it), then O += P V of tile
+// it - 1), warps 2 and 3 reduce ||v_j||^2 of the tokens from the V tiles (even / odd tiles).
+// Tensor memory: tile slot g = it & 1 holds S_g at g*128 (the bf16 P_g overwrites columns [0,32) and [64,96) of
+// it) and O_g at 256 + g*128.
 __device__ void phase_a_control(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tmQ, const CUtensorMap* tmK,
                         const CUtensorMap* tmV, int bh, int rank, int tile0, int T) {
   FusedBars* B = cx.B;
@@ -254,6 +255,9 @@ __device__ void phase_a_control(const Ctx& cx, const FusedArgs& a, const CUtenso
   }
 }
 
+// Worker warps in phase A: four softmax warpgroups, thread = query row; warpgroups g and g + 2 share tile slot g
+// (tokens 0-63 and 64-127 of the tile).  At the end the two slots' (m, l, O) are merged and written as the CTA's
+// partial.
 __device__ void phase_a_worker(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tmQ, const CUtensorMap* tmK,
                         const CUtensorMap* tmV, int bh, int rank, int tile0, int T) {
   FusedBars* B = cx.B;
