@@ -53,6 +53,28 @@ def algorithmic_flops(case):
     return 3 * 2 * R * case.head_dim * case.batch * case.n_kv_heads * case.n
 
 
+def max_over_ranks(total_ms, world, device):
+    """The slowest rank's time for the timed region (the job ends when the last replica ends)."""
+    if world <= 1:
+        return float(total_ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([total_ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(tokens_per_rank_step, world, steps, total_ms):
+    """Prefix tokens per second over all replicas: every rank processes its own layer in every step."""
+    return world * tokens_per_rank_step * steps / (total_ms / 1e3)
+
+
+# DRAM bytes (read + write) per launch of the score kernel, from the ncu capture summarised in
+# profiles/tc_fused_select_compact_cfg4_ncu_full.md; valid for the kernel as it stood then (set to None when
+# csrc/tc_fused.cu changes in more than comments).
+SCORE_KERNEL_TRAFFIC = {"cfg4": 1009.68e6 + 25.99e6}
+
+
 class ClockSampler:
     """Samples nvidia-smi SM clocks and throttle reasons while the timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -284,14 +306,34 @@ def main():
         handle.set_profile_events(kid, None, None)
     assert handle.poll_status() == rk.RESTKV_OK
 
-    total_ms = float(sum(step_ms))
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(float(sum(step_ms)), world, "cuda")
     tokens_per_step = world * case.batch * case.n
-    value = tokens_per_step * args.steps / (total_ms / 1e3)
+    value = whole_job_value(case.batch * case.n, world, args.steps, total_ms)
     ms_per_step = total_ms / args.steps
+
+    # ---- one decode step over the compacted cache and over the full cache (context for the paper's 10.61x) ----
+    decode = None
+    if rank == 0:
+        qd = torch.randn(case.batch, case.n_q_heads, case.head_dim, device="cuda").to(tdt)
+        dout = torch.empty(case.batch, case.n_q_heads, case.head_dim, dtype=torch.float32, device="cuda")
+
+        def time_decode(Kc, Vc, rows):
+            for _ in range(3):
+                handle.decode(shape, qd, Kc, Vc, rows, dout, ws)
+            ts = []
+            for _ in range(10):
+                flush.zero_()
+                ev0.record()
+                handle.decode(shape, qd, Kc, Vc, rows, dout, ws)
+                ev1.record()
+                torch.cuda.synchronize()
+                ts.append(ev0.elapsed_time(ev1))
+            return float(np.median(ts)) * 1e3
+        us_c = time_decode(K_out, V_out, keep)
+        us_f = time_decode(K, V, case.n_kv)
+        decode = {"compact_us": us_c, "full_us": us_f, "ratio": us_f / us_c, "rows_compact": keep,
+                  "rows_full": case.n_kv, "note": "one layer, one token, this kernel only; the paper's 10.61x is the "
+                  "whole model's per-token latency on an A800 with FlashAttention-2"}
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----
     e2e = None
@@ -316,10 +358,7 @@ def main():
             torch.cuda.synchronize()
             ms += ev0.elapsed_time(ev1)
         barrier()
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = max_over_ranks(ms, world, "cuda")
         h2d = sum(x.numel() * x.element_size() for x in (hQ, hK, hV))
         d2h = sum(x.numel() * x.element_size() for x in (h_idx, h_Ko, h_Vo))
         e2e = {"value": tokens_per_step * e2e_steps / (ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
@@ -339,7 +378,8 @@ def main():
     dom_bytes = kv_bytes + 4 * case.batch * case.n_kv_heads * case.n
     achieved = dom_bytes / (kmean[dominant] * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "tc_fused_kernel (score: pass 1 + merge + pass 2)", "achieved": achieved,
-                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                "traffic": SCORE_KERNEL_TRAFFIC.get(args.workload) if args.path == 0 else None,
                 "peak_source": peaks["source"], "algorithmic_bytes_per_launch": dom_bytes,
                 "ms_per_launch": kmean[dominant]}
     t_roof_ms = max((kv_bytes + out_bytes) / (peaks["hbm_gbs"] * 1e9), flops / (peaks["bf16_tflops"] * 1e12)) * 1e3
@@ -352,7 +392,7 @@ def main():
         "dtype": case.dtype, "data": "synthetic",
         "config": workload_config(case, l2="flushed between steps (256 MiB write); inputs 537 MB > 126 MB L2"),
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-        "roofline": roofline, "path_roofline": path_roofline, "kernels_ms": kmean,
+        "roofline": roofline, "path_roofline": path_roofline, "kernels_ms": kmean, "decode": decode,
     }
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(inp, case.budget)
