@@ -331,8 +331,10 @@ def main():
             return float(np.median(ts)) * 1e3
         us_c = time_decode(K_out, V_out, keep)
         us_f = time_decode(K, V, case.n_kv)
+        row_bytes = 2 * case.batch * case.n_kv_heads * case.head_dim * (2 if case.dtype == "bf16" else 4)
         decode = {"compact_us": us_c, "full_us": us_f, "ratio": us_f / us_c, "rows_compact": keep,
-                  "rows_full": case.n_kv, "note": "one layer, one token, this kernel only; the paper's 10.61x is the "
+                  "rows_full": case.n_kv, "compact_gbs": row_bytes * keep / us_c / 1e3,
+                  "full_gbs": row_bytes * case.n_kv / us_f / 1e3, "note": "one layer, one token, this kernel only; the paper's 10.61x is the "
                   "whole model's per-token latency on an A800 with FlashAttention-2"}
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----

@@ -107,43 +107,55 @@ __global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(
     }
   }
 
-  // merge the lane groups of this block
-  __shared__ float sm_m[kGroups][G], sm_l[kGroups][G];
-  __shared__ float sm_scale[kGroups][G];
-  __shared__ float sm_o[G][LPR * EPL];
-  if (sub == 0) {
+  // ---- merge, in a fixed order (no atomics: the result is bit-reproducible) ----
+  // 1. the lane groups of a warp, by butterfly exchange: afterwards every group holds the warp's result
 #pragma unroll
-    for (int g = 0; g < G; ++g) { sm_m[grp][g] = m[g]; sm_l[grp][g] = l[g]; }
+  for (int off = LPR; off < 32; off <<= 1) {
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      const float m_o = __shfl_xor_sync(0xffffffffu, m[g], off);
+      const float l_o = __shfl_xor_sync(0xffffffffu, l[g], off);
+      const float mm = fmaxf(m[g], m_o);
+      const float sa = (m[g] == -INFINITY) ? 0.f : __expf(m[g] - mm);
+      const float sb = (m_o == -INFINITY) ? 0.f : __expf(m_o - mm);
+      l[g] = l[g] * sa + l_o * sb;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) o[g][e] = o[g][e] * sa + __shfl_xor_sync(0xffffffffu, o[g][e], off) * sb;
+      m[g] = mm;
+    }
   }
-  for (int e = threadIdx.x; e < G * LPR * EPL; e += kDecThreads) (&sm_o[0][0])[e] = 0.f;
+  // 2. the warps, through shared memory: w_ml [warps][G][2], w_o [warps][G][d]
+  extern __shared__ float dec_smem[];
+  constexpr int kWarps = kDecThreads / 32;
+  float* w_ml = dec_smem;
+  float* w_o = dec_smem + kWarps * G * 2;
+  if (lane < LPR) {
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      if (sub == 0) { w_ml[(wid * G + g) * 2] = m[g]; w_ml[(wid * G + g) * 2 + 1] = l[g]; }
+#pragma unroll
+      for (int c = 0; c < CPL; ++c)
+#pragma unroll
+        for (int e = 0; e < E; ++e) w_o[((long long)wid * G + g) * d + (c * LPR + sub) * E + e] = o[g][c * E + e];
+    }
+  }
   __syncthreads();
   float* my_part = part + ((long long)bh * splits + split) * G * (d + 2);
-  if (threadIdx.x < G) {
-    const int g = threadIdx.x;
-    float mm = -INFINITY;
-    for (int k = 0; k < kGroups; ++k) mm = fmaxf(mm, sm_m[k][g]);
-    float ll = 0.f;
-    for (int k = 0; k < kGroups; ++k) {
-      const float sc = (sm_m[k][g] == -INFINITY) ? 0.f : __expf(sm_m[k][g] - mm);
-      sm_scale[k][g] = sc;
-      ll += sm_l[k][g] * sc;
-    }
-    my_part[g * (d + 2) + 0] = mm;
-    my_part[g * (d + 2) + 1] = ll;
-  }
-  __syncthreads();
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    const float sc = sm_scale[grp][g];
-#pragma unroll
-    for (int c = 0; c < CPL; ++c)
-#pragma unroll
-      for (int e = 0; e < E; ++e) atomicAdd(&sm_o[g][(c * LPR + sub) * E + e], o[g][c * E + e] * sc);
-  }
-  __syncthreads();
   for (int e = threadIdx.x; e < G * d; e += kDecThreads) {
     const int g = e / d, k = e - g * d;
-    my_part[g * (d + 2) + 2 + k] = sm_o[g][k];
+    float mm = -INFINITY;
+#pragma unroll
+    for (int wv = 0; wv < kWarps; ++wv) mm = fmaxf(mm, w_ml[(wv * G + g) * 2]);
+    float acc = 0.f, ll = 0.f;
+#pragma unroll
+    for (int wv = 0; wv < kWarps; ++wv) {
+      const float mw = w_ml[(wv * G + g) * 2];
+      const float sc = (mw == -INFINITY) ? 0.f : __expf(mw - mm);
+      acc = fmaf(w_o[((long long)wv * G + g) * d + k], sc, acc);
+      ll = fmaf(w_ml[(wv * G + g) * 2 + 1], sc, ll);
+    }
+    my_part[g * (d + 2) + 2 + k] = acc;
+    if (k == 0) { my_part[g * (d + 2)] = mm; my_part[g * (d + 2) + 1] = ll; }
   }
 }
 
@@ -178,12 +190,21 @@ cudaError_t launch_partial(const Problem& p, const void* q, const void* Kc, cons
   constexpr int E = Chunk<T>::kElems;
   dim3 grid(splits, p.BH);
   const int chunks = p.d / E;   // 16-byte chunks per row
-#define RESTKV_DEC(LPR, CPL)                                                                              \
-  decode_partial_kernel<T, G, LPR, CPL><<<grid, kDecThreads, 0, st>>>(p.Hq, p.Hkv, p.d, n_rows, p.scale, \
-                                                                      (const T*)q, (const T*)Kc, (const T*)Vc, part, splits)
+  const size_t smem = (size_t)(kDecThreads / 32) * G * (p.d + 2) * sizeof(float);
+#define RESTKV_DEC(LPR, CPL)                                                                                    \
+  do {                                                                                                          \
+    if (smem > 48 * 1024) {                                                                                     \
+      cudaError_t e_ = cudaFuncSetAttribute(decode_partial_kernel<T, G, LPR, CPL>,                              \
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);            \
+      if (e_ != cudaSuccess) return e_;                                                                         \
+    }                                                                                                           \
+    decode_partial_kernel<T, G, LPR, CPL><<<grid, kDecThreads, smem, st>>>(                                     \
+        p.Hq, p.Hkv, p.d, n_rows, p.scale, (const T*)q, (const T*)Kc, (const T*)Vc, part, splits);              \
+  } while (0)
+  // one 16-byte chunk per lane where the row allows it: few registers per thread, several CTAs per SM
   if (chunks == 8) RESTKV_DEC(8, 1);
-  else if (chunks == 16) RESTKV_DEC(8, 2);
-  else if (chunks == 32) RESTKV_DEC(16, 2);
+  else if (chunks == 16) RESTKV_DEC(16, 1);
+  else if (chunks == 32) RESTKV_DEC(32, 1);
   else if (chunks == 64) RESTKV_DEC(32, 2);
   else if (chunks == 4) RESTKV_DEC(4, 1);
   else if (chunks == 2) RESTKV_DEC(2, 1);
