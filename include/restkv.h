@@ -153,6 +153,10 @@ restkv_status restkv_evict_host(restkv_handle* h, const restkv_shape* shape, con
  *   out      device float [batch, n_q_heads, head_dim]
  *   lse      optional device float [batch, n_q_heads] (natural-log sum of exp of the scaled logits)
  * shape->n_kv, w, causal_tail and the strides are ignored.
+ * RESTKV_BF16 with head_dim 128 and up to 128 query heads per KV head runs as plain attention on the tensor-core
+ * kernel (the softmax weights are rounded to bf16 before they meet V) when the workspace has the ~10 MB it needs,
+ * which every restkv_workspace_bytes() result has; everything else runs on fp32 SIMT kernels, which need
+ * batch * n_kv_heads * 64 * group * (head_dim + 2) floats.
  */
 restkv_status restkv_decode(restkv_handle* h, const restkv_shape* shape, const void* q, const void* Kc,
                             const void* Vc, int n_rows, float* out, float* lse, void* workspace,

@@ -242,6 +242,46 @@ cudaError_t launch_decode(const Problem& p, const void* q, const void* Kc, const
 
 }  // namespace restkv
 
+// ------------------------------------------------------------------------------------------------
+// Decode through the tensor-core attention phases: the G queries of a KV head are padded with zero rows to the
+// kernel's 128 query rows, and afterwards the G real rows are copied out.
+namespace restkv {
+namespace {
+
+// grid (128, BH), block 64: q_pad[bh, r, :] = q[b, h*G + r, :] for r < G, else 0 (bf16, head_dim 128).
+__global__ void decode_pad_kernel(int Hq, int Hkv, int G, const __nv_bfloat16* __restrict__ q,
+                                  __nv_bfloat16* __restrict__ q_pad) {
+  const int r = blockIdx.x, bh = blockIdx.y, b = bh / Hkv, h = bh % Hkv;
+  const unsigned int* src = reinterpret_cast<const unsigned int*>(q + ((long long)b * Hq + (long long)h * G + r) * 128);
+  unsigned int* dst = reinterpret_cast<unsigned int*>(q_pad + ((long long)bh * 128 + r) * 128);
+  dst[threadIdx.x] = r < G ? src[threadIdx.x] : 0u;
+}
+
+// grid (G, BH), block 128: out[b, h*G + g, :] = O[bh, g, :]; lse = M2 * ln 2 (M2 is in log2 units).
+__global__ void decode_extract_kernel(int Hq, int Hkv, int G, const float* __restrict__ O_f32,
+                                      const float* __restrict__ row_M2, float* __restrict__ out,
+                                      float* __restrict__ lse) {
+  const int g = blockIdx.x, bh = blockIdx.y, b = bh / Hkv, h = bh % Hkv;
+  const long long hq = (long long)b * Hq + (long long)h * G + g;
+  out[hq * 128 + threadIdx.x] = O_f32[((long long)bh * 128 + g) * 128 + threadIdx.x];
+  if (lse && threadIdx.x == 0) lse[hq] = row_M2[(long long)bh * 128 + g] * 0.6931471805599453f;
+}
+
+}  // namespace
+
+cudaError_t launch_decode_pad(const Problem& p, const void* q, __nv_bfloat16* q_pad, cudaStream_t st) {
+  decode_pad_kernel<<<dim3(128, p.BH), 64, 0, st>>>(p.Hq, p.Hkv, p.G, (const __nv_bfloat16*)q, q_pad);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_decode_extract(const Problem& p, const float* O_f32, const float* row_M2, float* out, float* lse,
+                                  cudaStream_t st) {
+  decode_extract_kernel<<<dim3(p.G, p.BH), 128, 0, st>>>(p.Hq, p.Hkv, p.G, O_f32, row_M2, out, lse);
+  return cudaGetLastError();
+}
+
+}  // namespace restkv
+
 // ================================================================================================
 // restkv_decode_static: the decode step with its split partials in memory that ships with the library.
 // ================================================================================================

@@ -48,7 +48,8 @@ size_t plan_workspace(const Problem& p, int budget, int sm_count, bool adaptive,
   };
   Workspace w{};
   w.splits = pass1_splits(p, sm_count);
-  const size_t BH = (size_t)p.BH, R = (size_t)p.R, d = (size_t)p.d;
+  // at least the tensor-core kernel's 128 query rows, so that restkv_decode can use it whatever w * group is
+  const size_t BH = (size_t)p.BH, R = (size_t)(p.R > 128 ? p.R : 128), d = (size_t)p.d;
   // partial slots: one per (head, split) on the SIMT path, one per CTA in the persistent tensor-core kernel
   size_t slots = BH * w.splits;
   if (slots < (size_t)sm_count) slots = (size_t)sm_count;
@@ -58,6 +59,7 @@ size_t plan_workspace(const Problem& p, int budget, int sm_count, bool adaptive,
   w.counters = (unsigned int*)take(1024);
   w.tile_max = (float*)take(BH * (size_t)((p.n_kv + 127) / 128) * 128 * sizeof(float));
   w.row_M2 = (float*)take(BH * 128 * sizeof(float));
+  w.q_pad = (__nv_bfloat16*)take(BH * 128 * 128 * sizeof(__nv_bfloat16));
   w.vnorm = (float*)take(BH * (size_t)p.n_kv * sizeof(float));
   w.fin_m = (float*)take(BH * R * sizeof(float));
   w.fin_l = (float*)take(BH * R * sizeof(float));
@@ -77,6 +79,30 @@ size_t plan_workspace(const Problem& p, int budget, int sm_count, bool adaptive,
     w.adaptive_idx = (int32_t*)take((size_t)p.batch * p.Hq * p.w * Bp * sizeof(int32_t));
     w.adaptive_sums = (unsigned long long*)take(BH * 2 * sizeof(unsigned long long));
   }
+  w.bytes = off;
+  if (ws) *ws = w;
+  return off;
+}
+
+// The part of the workspace that restkv_decode's tensor-core path uses (phases A and B of the score kernel only).
+static size_t plan_decode_tc(int BH, int sm_count, void* base, Workspace* ws) {
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    void* ptr = base ? (void*)((char*)base + off) : nullptr;
+    off += align256(bytes);
+    return ptr;
+  };
+  Workspace w{};
+  const size_t bh = (size_t)BH, slots = (size_t)sm_count;
+  w.part_m = (float*)take(slots * 128 * sizeof(float));
+  w.part_l = (float*)take(slots * 128 * sizeof(float));
+  w.part_O = (float*)take(slots * 128 * 128 * sizeof(float));
+  w.counters = (unsigned int*)take(1024);
+  w.row_M2 = (float*)take(bh * 128 * sizeof(float));
+  w.q_pad = (__nv_bfloat16*)take(bh * 128 * 128 * sizeof(__nv_bfloat16));
+  w.O_f32 = (float*)take(bh * 128 * 128 * sizeof(float));
+  w.O_m2 = (__nv_bfloat16*)take(bh * 128 * 128 * sizeof(__nv_bfloat16));
+  w.aug = (__nv_bfloat16*)take(bh * 128 * 64 * sizeof(__nv_bfloat16));
   w.bytes = off;
   if (ws) *ws = w;
   return off;
@@ -180,7 +206,7 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
     // flight as fit in L2 so that pass 2 re-reads K and V from there
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2,
                   launch_tc_fused(c.h->tc_state, p, ws, Q, K, V, ema_decay, c.h->sm_count, c.h->kernel_path == 3,
-                                  c.h->dev_status, c.st), 1);
+                                  false, c.h->dev_status, c.st), 1);
   } else {
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS1, launch_simt_pass1(p, ws, Q, K, V, c.st), 1);
     RESTKV_LAUNCH(c, RESTKV_KERNEL_COMBINE, launch_combine(p, ws, c.st), 1);
@@ -386,6 +412,25 @@ restkv_status restkv_decode(restkv_handle* h, const restkv_shape* shape, const v
   const size_t need = align256((size_t)p.BH * kDecodeMaxSplits * p.G * (p.d + 2) * sizeof(float));
   if (!workspace || ((uintptr_t)workspace & 255u) != 0 || workspace_bytes < need) return RESTKV_ERR_WORKSPACE;
   Call c{h, (cudaStream_t)stream};
+  // bf16, head_dim 128: the decode step is plain attention of up to 128 query rows per KV head, i.e. phases A and B
+  // of the tensor-core score kernel with the group's queries padded to its 128 rows.  It needs about 10 MB of
+  // workspace (any restkv_workspace_bytes result has that); with less, or for other shapes, the SIMT kernels run.
+  if (h->tc_state && h->kernel_path != 1 && p.dtype == RESTKV_BF16 && p.d == 128 && p.G <= 128 && n_rows > 1) {
+    Problem pd = p;
+    pd.G = 128; pd.Hq = p.Hkv * 128; pd.w = 1; pd.R = 128; pd.tail = 0; pd.n = pd.n_kv = n_rows;
+    pd.ksn = pd.vsn = p.d;
+    pd.ksh = pd.vsh = (long long)n_rows * p.d;
+    pd.ksb = pd.vsb = (long long)p.Hkv * n_rows * p.d;
+    Workspace ws;
+    if (plan_decode_tc(pd.BH, h->sm_count, workspace, &ws) <= workspace_bytes) {
+      RESTKV_LAUNCH(c, RESTKV_KERNEL_NONE, launch_decode_pad(p, q, ws.q_pad, c.st), 1);
+      RESTKV_LAUNCH(c, RESTKV_KERNEL_NONE,
+                    launch_tc_fused(h->tc_state, pd, ws, ws.q_pad, Kc, Vc, 0.f, h->sm_count, false, true, h->dev_status,
+                                    c.st), 1);
+      RESTKV_LAUNCH(c, RESTKV_KERNEL_NONE, launch_decode_extract(p, ws.O_f32, ws.row_M2, out, lse, c.st), 1);
+      return RESTKV_OK;
+    }
+  }
   int nl = 0;
   cudaError_t e = launch_decode(p, q, Kc, Vc, n_rows, out, lse, (float*)workspace,
                                 decode_splits(p, n_rows, h->sm_count), c.st, &nl);

@@ -36,6 +36,7 @@ struct Workspace {
   unsigned int* counters; // [256] group barrier counters of the head-sequential kernel
   float* tile_max;        // [BH, tiles, 128] per-tile row maxima of the persistent score kernel
   float* row_M2;          // [BH, 128] log2 normaliser of each query row
+  __nv_bfloat16* q_pad;   // [BH, 128, 128] decode queries padded to the kernel's 128 rows
   float* fin_m;           // [BH, R]    row max of the scaled logits (natural units)
   float* fin_l;           // [BH, R]    sum of exp(s - m)
   float* O_f32;           // [BH, R, d]
@@ -81,8 +82,11 @@ bool tc_supported(const Problem& p);
 cudaError_t tc_init(void** state);   // resolves the driver entry point for tensor-map encoding
 cudaError_t tc_fused_init();
 cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
-                            const void* V, float ema_decay, int sm_count, bool reuse_l2, unsigned int* dev_status,
-                            cudaStream_t st);
+                            const void* V, float ema_decay, int sm_count, bool reuse_l2, bool attention_only,
+                            unsigned int* dev_status, cudaStream_t st);
+cudaError_t launch_decode_pad(const Problem& p, const void* q, __nv_bfloat16* q_pad, cudaStream_t st);
+cudaError_t launch_decode_extract(const Problem& p, const float* O_f32, const float* row_M2, float* out, float* lse,
+                                  cudaStream_t st);
 
 // ---- small device helpers ------------------------------------------------------------------------
 template <typename T> __device__ __forceinline__ float to_f32(T x);

@@ -34,6 +34,7 @@ struct FusedArgs {
   int Hkv, BH, n, n_kv, w;
   float scale, ema_decay;
   int groups, cpg;                   // CTA groups and CTAs per group
+  int attention_only;                // 1: stop after the merge (phases A and B): plain attention of the 128 rows
   float* part_m;                     // [CTA, 128]       running maximum, log2 units (one slot per CTA, reused
   float* part_l;                     // [CTA, 128]        from head to head: a group is past phase B of a head
   float* part_O;                     // [CTA, 128, 128]   before any of its CTAs writes the next head's partial)
@@ -249,7 +250,7 @@ __device__ void phase_a_control(const Ctx& cx, const FusedArgs& a, const CUtenso
 #pragma unroll
       for (int rr = 0; rr < 4; ++rr) {
         const int j = (tile0 + it) * kTile + rr * 32 + lane;
-        if (j < a.n_kv) a.vnorm[(long long)bh * a.n_kv + j] = vn[rr];
+        if (j < a.n_kv && !a.attention_only) a.vnorm[(long long)bh * a.n_kv + j] = vn[rr];
       }
     }
   }
@@ -324,7 +325,7 @@ __device__ void phase_a_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
     const float m_tile = tmax * c2;
     // phase C takes the exact distance only in tiles where some weight can exceed kHeavyA: it compares this
     // maximum with the row's final normaliser
-    if (hf == 0) a.tile_max[((long long)bh * nt_all + tile0 + it) * kRows + row] = m_tile;
+    if (hf == 0 && !a.attention_only) a.tile_max[((long long)bh * nt_all + tile0 + it) * kRows + row] = m_tile;
     const bool need = m_tile > m_ref + kRescaleThreshold;   // also true for the first visible entries (m_ref = -inf)
     float factor = 1.f;
     if (need) {
@@ -893,7 +894,7 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const int per = (nt1 + a.cpg - 1) / a.cpg;
   pl.tile0 = rank * per;
   pl.T1 = max(0, min(nt1, pl.tile0 + per) - pl.tile0);
-  pl.T2 = max(0, min(nt2, pl.tile0 + per) - pl.tile0);
+  pl.T2 = a.attention_only ? 0 : max(0, min(nt2, pl.tile0 + per) - pl.tile0);
 
   // Each role's code sits behind its own register-budget change, so that the sixteen worker warps can be
   // compiled for more registers than the launch gives every thread.
@@ -984,8 +985,8 @@ cudaError_t tc_fused_init() {
 // long as the device is not shared with another kernel at that moment; if it is, the bounded group barrier gives up
 // with the timeout status instead of hanging.  (A cooperative launch would guarantee residency but costs ~25 us.)
 cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
-                            const void* V, float ema_decay, int sm_count, bool reuse_l2, unsigned int* dev_status,
-                            cudaStream_t st) {
+                            const void* V, float ema_decay, int sm_count, bool reuse_l2, bool attention_only,
+                            unsigned int* dev_status, cudaStream_t st) {
   TcState* ts = (TcState*)state;
   CUtensorMap tmQ, tmK, tmV, tmO, tmAug;
   if (!make_rows_map(ts, &tmQ, Q, p.BH) || !make_rows_map(ts, &tmO, ws.O_m2, p.BH) ||
@@ -995,6 +996,7 @@ cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, 
   FusedArgs a{};
   a.Hkv = p.Hkv; a.BH = p.BH; a.n = p.n; a.n_kv = p.n_kv; a.w = p.w;
   a.scale = p.scale; a.ema_decay = ema_decay;
+  a.attention_only = attention_only ? 1 : 0;
   fused_plan(p, sm_count, reuse_l2, &a.groups, &a.cpg);
   a.part_m = ws.part_m; a.part_l = ws.part_l; a.part_O = ws.part_O;
   a.O_f32 = ws.O_f32; a.O_m2 = ws.O_m2; a.aug = ws.aug; a.vnorm = ws.vnorm; a.I_hat = ws.I_hat;
@@ -1003,7 +1005,7 @@ cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, 
   cudaError_t e = cudaMemsetAsync(ws.counters, 0, 1024, st);
   if (e != cudaSuccess) return e;
   const dim3 grid(a.groups * a.cpg), block(kFThreads);
-  switch (p.w) {
+  switch (attention_only ? 32 : p.w) {   // the window length only matters to phase C
     case 16: tc_fused_kernel<16><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a); break;
     case 32: tc_fused_kernel<32><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a); break;
     case 64: tc_fused_kernel<64><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a); break;

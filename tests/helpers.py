@@ -10,6 +10,11 @@ from paper_2605_08840_b200.inputs import Case, Inputs
 # relative tolerance of the scores: bf16 inputs with fp32 accumulation / fp32 mode
 TOL = {"bf16": 2e-3, "f32": 1e-5}
 
+# decode (a timing aid): max error of an output row relative to that row's largest element.  The bf16 path feeds the
+# softmax weights to the tensor core as bf16 (relative rounding 2^-9 per weight, random sign): per output element
+# that is ~1.1e-3 of the output's own spread, and the largest of the 128 x n_q_heads elements sits near 2.5x that.
+DECODE_TOL = {"bf16": 4e-3, "f32": 2e-5}
+
 
 def torch_dev(arr: np.ndarray, dtype: str):
     """numpy (int16 bf16 bits | float32) -> CUDA tensor of the library's element type."""

@@ -8,7 +8,7 @@ import oracle
 from paper_2605_08840_b200 import binding as rk
 from paper_2605_08840_b200.inputs import CONFIGS, Case, make_inputs, make_decode_query, round_to_bf16_bits
 
-from helpers import (TOL, GpuRun, assert_compaction_exact, assert_scores_close, assert_selection_valid, shape_of,
+from helpers import (DECODE_TOL, TOL, GpuRun, assert_compaction_exact, assert_scores_close, assert_selection_valid, shape_of,
                      torch_dev)
 
 pytestmark = pytest.mark.gpu
@@ -344,7 +344,7 @@ def test_decode_matches_oracle(handle, spec):
     ws = torch.empty(handle.workspace_bytes(shape, 0), dtype=torch.uint8, device="cuda")
     handle.decode(shape, torch_dev(qd, dtype), torch_dev(Kd, dtype), torch_dev(Vd, dtype), rows, out, ws, lse=lse)
     torch.cuda.synchronize()
-    tol = 2e-3 if dtype == "bf16" else 2e-5
+    tol = DECODE_TOL[dtype]
     scale = np.abs(ref).max(axis=-1, keepdims=True)
     assert np.max(np.abs(out.cpu().numpy() - ref) / scale) < tol
     np.testing.assert_allclose(lse.cpu().numpy(), ref_lse, rtol=1e-5, atol=1e-5)
@@ -364,7 +364,7 @@ def test_decode_over_compacted_cache_of_config2(handle):
     Kc = np.take_along_axis(inp.K, idx[..., None].astype(np.int64), axis=2)
     Vc = np.take_along_axis(inp.V, idx[..., None].astype(np.int64), axis=2)
     ref, _ = oracle.decode(q, Kc, Vc)
-    assert np.max(np.abs(out.cpu().numpy() - ref)) < 2e-3 * np.abs(ref).max()
+    assert np.max(np.abs(out.cpu().numpy() - ref)) < DECODE_TOL["bf16"] * np.abs(ref).max()
 
 
 # ------------------------------------------------------------------ API misuse: error codes, never a fault
