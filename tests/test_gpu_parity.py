@@ -234,6 +234,23 @@ def test_edge_cases(handle, spec):
     full_check(handle, make_inputs(case))
 
 
+def test_more_heads_than_sms(handle):
+    """160 (batch, KV head) pairs: the persistent score kernel runs one CTA per head and two rounds."""
+    case = Case("many_heads", 20, 32, 8, 128, 300, 32, 30, 5, 0, 0.8, "bf16", 0, "normal", 33)
+    inp = make_inputs(case)
+    run = GpuRun(handle, inp)
+    scores, idx, K_out, V_out = run.evict()
+    pick = [(0, 0), (7, 3), (19, 7)]           # the oracle checks three of the 160 heads
+    for b, h in pick:
+        one = _subset_heads(type(inp)(case.with_(batch=1), inp.Q[b:b + 1], inp.K[b:b + 1], inp.V[b:b + 1]), [h])
+        ref = oracle_scores(one).scores[0, 0]
+        assert_scores_close(scores[b, h], ref, TOL["bf16"])
+        assert_selection_valid(idx[b:b + 1, h:h + 1], ref[None, None], case.budget, TOL["bf16"])
+    _, kbits, vbits = inp.device_arrays()
+    assert_compaction_exact(idx, kbits, K_out)
+    assert_compaction_exact(idx, vbits, V_out)
+
+
 @pytest.mark.parametrize("decay", [0.0, 1.0])
 def test_ema_extremes(handle, decay):
     case = Case("ema", 1, 8, 2, 128, 600, 16, 50, 1, 0, decay, "bf16", 0, "normal", 5)
