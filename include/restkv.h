@@ -204,7 +204,9 @@ const char* restkv_error_string(restkv_status s);
 /* Profiling aid: while a pair of events is set for kernel `which` (RESTKV_KERNEL_*, not NONE), every call records
  * `start` right before and `stop` right after that kernel's launch on the call's stream, so a caller can time
  * single kernels of the fused path with CUDA events.  start/stop are cudaEvent_t handles created by the caller
- * with timing enabled; passing NULL for both clears the pair. */
+ * with timing enabled; passing NULL for both clears the pair.  On the tensor-core path pass 1, the merge and pass 2
+ * are one launch, recorded as RESTKV_KERNEL_PASS2 (PASS1 and COMBINE fire on the SIMT path only); in restkv_evict
+ * the pooling and the gather run inside the select kernel, recorded as RESTKV_KERNEL_SELECT. */
 typedef enum {
   RESTKV_KERNEL_NONE = 0, RESTKV_KERNEL_PASS1 = 1, RESTKV_KERNEL_COMBINE = 2, RESTKV_KERNEL_PASS2 = 3,
   RESTKV_KERNEL_POOL = 4, RESTKV_KERNEL_SELECT = 5, RESTKV_KERNEL_COMPACT = 6

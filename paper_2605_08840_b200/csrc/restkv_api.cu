@@ -69,7 +69,6 @@ size_t plan_workspace(const Problem& p, int budget, int sm_count, bool adaptive,
   w.I_hat = (float*)take(BH * (size_t)p.n * sizeof(float));
   w.scores = (float*)take(BH * (size_t)p.n_kv * sizeof(float));
   w.pool = (int*)take(BH * 2 * sizeof(int));
-  w.sel_scratch = (unsigned int*)take(BH * kSelScratchWords * sizeof(unsigned int));
   w.dec_part = (float*)take(BH * (size_t)kDecodeMaxSplits * p.G * (d + 2) * sizeof(float));
   if (adaptive) {
     int Bp = budget - p.tail;

@@ -45,7 +45,6 @@ struct Workspace {
   float* I_hat;           // [BH, n]
   float* scores;          // [BH, n_kv] (used when the caller passes no scores buffer)
   int* pool;              // [BH, 2] (W, gamma)
-  unsigned int* sel_scratch;  // select scratch: [BH, kSelScratchWords]
   float* dec_part;        // decode partials
   float* I_raw;           // adaptive only: [batch, Hq, w, n]
   int32_t* adaptive_idx;  // adaptive only: [batch*Hq*w, B_p] per-query top-B_p indices
@@ -53,7 +52,6 @@ struct Workspace {
   size_t bytes;
 };
 
-constexpr int kSelScratchWords = 64;
 constexpr int kDecodeMaxSplits = 64;
 
 int pass1_splits(const Problem& p, int sm_count);

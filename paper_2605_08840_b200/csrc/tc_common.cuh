@@ -44,23 +44,24 @@ __device__ __forceinline__ void mma_tile_kk(uint32_t tmem_d, uint32_t a_smem, ui
   }
 }
 
+// Exact ||o - v||^2 for the rare entries whose attention weight is large (the expansion ||o||^2 + ||v||^2 - 2 o.v
+// cancels when o approaches v).  Computed by a whole warp: lane L takes elements 4L .. 4L+3, the partial sums meet by butterfly exchange (every
+// lane returns the full sum).
+__device__ __forceinline__ float exact_dist2_warp(const float* __restrict__ o_row, const __nv_bfloat16* __restrict__ v_row,
+                                                  int lane) {
+  const float4 o = *reinterpret_cast<const float4*>(o_row + lane * 4);
+  const uint2 vv = *reinterpret_cast<const uint2*>(v_row + lane * 4);
+  const float d0 = o.x - __uint_as_float(vv.x << 16), d1 = o.y - __uint_as_float(vv.x & 0xFFFF0000u);
+  const float d2 = o.z - __uint_as_float(vv.y << 16), d3 = o.w - __uint_as_float(vv.y & 0xFFFF0000u);
+  float ss = (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+  return ss;
+}
+
 constexpr uint32_t kAugBytes = kBoxBytes;     // [128 rows x 64 bf16], only K steps 0 (S') and 1 (C') are used
 constexpr uint32_t kOnesBytes = 1024;         // one 8-row group of ones, shared by all 16 groups (stride 0)
 constexpr float kHeavyA = 0.125f;             // attention weight above which ||o - v||^2 is recomputed exactly
-
-// Exact ||o - v||^2 for the rare entries whose attention weight is large (the expansion
-// ||o||^2 + ||v||^2 - 2 o.v cancels when o approaches v).
-__device__ __noinline__ float exact_dist2(const float* __restrict__ o_row, const __nv_bfloat16* __restrict__ v_row) {
-  float ss = 0.f;
-  for (int k = 0; k < kHeadDim; k += 2) {
-    const float2 o = *reinterpret_cast<const float2*>(o_row + k);
-    const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(v_row + k);
-    const float d0 = o.x - __low2float(v), d1 = o.y - __high2float(v);
-    ss = fmaf(d0, d0, ss);
-    ss = fmaf(d1, d1, ss);
-  }
-  return ss;
-}
 
 // ------------------------------------------------------------------------------------------------
 inline CUresult encode_tiles(TcState* st, CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims,

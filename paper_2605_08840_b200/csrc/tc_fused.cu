@@ -736,8 +736,16 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
           for (int u = 0; u < 8; ++u) {
             const float um = ex2_approx(sv[u] * neg_c2) - 1.f;
             float x = cv[u] + vnb;
-            if (sv[u] > heavy_thr && j < n)
-              x = exact_dist2(O_head + (cgp * 32 + c * 8 + u) * kHeadDim, V_head + (long long)j * a.vsn);
+            // the whole warp computes the exact distance of each of its lanes' heavy entries in turn
+            unsigned int todo = __ballot_sync(0xffffffffu, sv[u] > heavy_thr && j < n);
+            while (todo) {
+              const int src = __ffs(todo) - 1;
+              todo &= todo - 1;
+              const int js = __shfl_sync(0xffffffffu, j, src);
+              const float d2x = exact_dist2_warp(O_head + (cgp * 32 + c * 8 + u) * kHeadDim,
+                                                 V_head + (long long)js * a.vsn, lane);
+              if (lane == src) x = d2x;
+            }
             I[u] = x * rsqrt_approx(fmaf(x * um, um, 1e-36f));
           }
           if ((c * 8) % kRun == 0) I[0] *= seed_coef;
