@@ -460,12 +460,13 @@ __device__ void combine_rows(const FusedArgs& a, int bh, int group, int r, int s
   if (r >= 0) {
     const long long base = (long long)group * a.cpg * kRows + r;   // + p * kRows
     // running merge of this warp's partials (all loads of a batch are issued before any is used)
+    constexpr int kBatch = 10;   // loads in flight per lane
 #pragma unroll 1
-    for (int p0 = sub; p0 < a.cpg; p0 += 4 * wpr) {
-      float mp[4], lp[4];
-      float4 v[4];
+    for (int p0 = sub; p0 < a.cpg; p0 += kBatch * wpr) {
+      float mp[kBatch], lp[kBatch];
+      float4 v[kBatch];
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
+      for (int k = 0; k < kBatch; ++k) {
         const int p = p0 + k * wpr;
         const bool in = p < a.cpg;
         const long long pi = base + (long long)(in ? p : p0) * kRows;
@@ -474,7 +475,7 @@ __device__ void combine_rows(const FusedArgs& a, int bh, int group, int r, int s
         v[k] = *reinterpret_cast<const float4*>(a.part_O + pi * kHeadDim + lane * 4);
       }
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
+      for (int k = 0; k < kBatch; ++k) {
         const float m_new = fmaxf(m, mp[k]);
         const float s_old = (m == -INFINITY) ? 0.f : ex2_approx(m - m_new);
         const float s_p = (mp[k] == -INFINITY) ? 0.f : ex2_approx(mp[k] - m_new);   // an empty partial weighs 0
