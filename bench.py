@@ -70,9 +70,9 @@ def whole_job_value(tokens_per_rank_step, world, steps, total_ms):
 
 
 # DRAM bytes (read + write) per launch of the score kernel, from the ncu capture summarised in
-# profiles/tc_fused_select_compact_cfg4_ncu_full.md; valid for the kernel as it stood then (set to None when
+# profiles/tc_fused_select_cfg4_ncu_full.md; valid for the kernel as it stood then (set to None when
 # csrc/tc_fused.cu changes in more than comments).
-SCORE_KERNEL_TRAFFIC = {"cfg4": 1009.68e6 + 25.99e6}
+SCORE_KERNEL_TRAFFIC = {"cfg4": 1008.62e6 + 26.38e6}
 
 
 class ClockSampler:
