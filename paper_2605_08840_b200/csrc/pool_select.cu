@@ -81,6 +81,39 @@ __device__ __forceinline__ unsigned int block_inclusive_scan(unsigned int v, uns
   return v;
 }
 
+// Box means of one CTA's slice from its staged taps (staged[t - s_lo] = I_hat[t] for t in [s_lo, s_hi]), summed in
+// the same order as box_mean; writes the pooled scores and their keys.  kWidth = 0: width known only at run time.
+template <int kWidth>
+__device__ __forceinline__ void pool_staged(const float* __restrict__ staged, int s_lo, int s_hi, int n, int j0, int cnt,
+                                            int W, int gamma, float* __restrict__ srow, unsigned int* __restrict__ skeys) {
+  const int width = kWidth ? kWidth : W;
+  const int half = width / 2;
+  const float fw = (float)width;
+  for (int jj = threadIdx.x; jj < cnt; jj += kSelThreads) {
+    const int j = j0 + jj;
+    float out = INFINITY;
+    if (j < n) {
+      const long long a64 = (long long)j - half + gamma, b64 = (long long)j + half + gamma;
+      float acc = 0.f;
+      if (a64 >= s_lo && b64 <= s_hi) {   // the whole window is staged: fixed trip count
+        const float* p = staged + (int)(a64 - s_lo);
+        if (kWidth) {
+#pragma unroll
+          for (int k = 0; k < kWidth; ++k) acc += p[k];
+        } else {
+          for (int k = 0; k < width; ++k) acc += p[k];
+        }
+      } else {
+        const int a = a64 < s_lo ? s_lo : (int)(a64 <= s_hi ? a64 : s_hi + 1), b = b64 > s_hi ? s_hi : (int)(b64 >= s_lo ? b64 : s_lo - 1);
+        for (int t = a; t <= b; ++t) acc += staged[t - s_lo];
+      }
+      out = acc / fw;
+    }
+    srow[jj] = out;
+    skeys[jj] = float_key(out);
+  }
+}
+
 // One thread-block cluster per row; CTA `rank` of the cluster owns the contiguous slice [rank*per, (rank+1)*per)
 // of the row.  With I_hat non-null the kernel first applies the box mean of Eq. 13 and writes the pooled scores;
 // otherwise it reads `scores`.  The keys of the slice stay in shared memory (use_smem) or are re-read from
@@ -125,20 +158,29 @@ select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const 
       const int half = W / 2;
       const long long lo64 = j0 - half + gamma, hi64 = j0 + cnt - 1 + half + gamma;
       const int s_lo = lo64 < 0 ? 0 : (int)(lo64 < n ? lo64 : n), s_hi = hi64 > n - 1 ? n - 1 : (int)(hi64 > -1 ? hi64 : -1);
-      for (int t = s_lo + tid; t <= s_hi; t += kSelThreads) staged[t - s_lo] = src[t];
-      __syncthreads();
-      for (int jj = tid; jj < cnt; jj += kSelThreads) {
-        const int j = (int)(j0 + jj);
-        float out = INFINITY;
-        if (j < n) {
-          const long long a64 = (long long)j - half + gamma, b64 = (long long)j + half + gamma;
-          const int a = a64 < s_lo ? s_lo : (int)(a64 <= s_hi ? a64 : s_hi + 1), b = b64 > s_hi ? s_hi : (int)(b64 >= s_lo ? b64 : s_lo - 1);
-          float acc = 0.f;
-          for (int t = a; t <= b; ++t) acc += staged[t - s_lo];
-          out = acc / (float)W;
+      // several loads in flight per thread
+      for (int t0 = s_lo + tid; t0 <= s_hi; t0 += 8 * kSelThreads) {
+        float v[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int t = t0 + k * kSelThreads;
+          v[k] = t <= s_hi ? src[t] : 0.f;
         }
-        srow[j0 + jj] = out;
-        skeys[jj] = float_key(out);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int t = t0 + k * kSelThreads;
+          if (t <= s_hi) staged[t - s_lo] = v[k];
+        }
+      }
+      __syncthreads();
+      switch (W) {   // the common widths get a compile-time trip count
+        case 1: pool_staged<1>(staged, s_lo, s_hi, n, (int)j0, cnt, W, gamma, srow + j0, skeys); break;
+        case 3: pool_staged<3>(staged, s_lo, s_hi, n, (int)j0, cnt, W, gamma, srow + j0, skeys); break;
+        case 5: pool_staged<5>(staged, s_lo, s_hi, n, (int)j0, cnt, W, gamma, srow + j0, skeys); break;
+        case 7: pool_staged<7>(staged, s_lo, s_hi, n, (int)j0, cnt, W, gamma, srow + j0, skeys); break;
+        case 21: pool_staged<21>(staged, s_lo, s_hi, n, (int)j0, cnt, W, gamma, srow + j0, skeys); break;
+        case 31: pool_staged<31>(staged, s_lo, s_hi, n, (int)j0, cnt, W, gamma, srow + j0, skeys); break;
+        default: pool_staged<0>(staged, s_lo, s_hi, n, (int)j0, cnt, W, gamma, srow + j0, skeys); break;
       }
     } else {
       for (int jj = tid; jj < cnt; jj += kSelThreads) {
@@ -291,12 +333,13 @@ select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const 
   }
   __syncthreads();
   cluster.sync();
-  unsigned int run_gt = warp_a[wid], run_eq = warp_b[wid];
+  unsigned int g_before = 0, e_before = 0;   // totals of the lower ranks of the cluster
   for (unsigned int r = 0; r < rank; ++r) {
     const unsigned int* rc = cluster.map_shared_rank(cta_counts, r);
-    run_gt += rc[0];
-    run_eq += rc[1];
+    g_before += rc[0];
+    e_before += rc[1];
   }
+  unsigned int run_gt = warp_a[wid] + g_before, run_eq = warp_b[wid] + e_before;
   for (int base = wbeg; base < wend; base += 32) {
     const int jj = base + lane;
     const bool valid = jj < wend;
@@ -314,12 +357,6 @@ select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const 
   }
   if (ga.K) {
     // ---- gather the rows this CTA selected: its indices are the contiguous run dst[first, first + mine) ----
-    unsigned int g_before = 0, e_before = 0;
-    for (unsigned int r = 0; r < rank; ++r) {
-      const unsigned int* rc = cluster.map_shared_rank(cta_counts, r);
-      g_before += rc[0];
-      e_before += rc[1];
-    }
     const unsigned int first = g_before + min(e_before, need_eq);
     const unsigned int mine = cta_counts[0] + (min(e_before + cta_counts[1], need_eq) - min(e_before, need_eq));
     __syncthreads();   // the indices written above are visible to the whole CTA
@@ -328,15 +365,36 @@ select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const 
     const unsigned char* Vh = ga.V + ((long long)b * ga.vsb + (long long)h * ga.vsh) * ga.esize;
     const long long out_row0 = (long long)row * keep;
     const int rc2 = 2 * ga.row_chunks;
-    for (unsigned int e = tid; e < mine * (unsigned int)rc2; e += kSelThreads) {
-      const unsigned int r = e / rc2;
-      const int c = (int)(e - r * rc2);
-      const bool isV = c >= ga.row_chunks;
-      const int chunk = isV ? c - ga.row_chunks : c;
-      const long long j = dst[first + r];
-      const uint4* src = reinterpret_cast<const uint4*>((isV ? Vh + j * ga.vsn * ga.esize : Kh + j * ga.ksn * ga.esize)) + chunk;
-      uint4* out = reinterpret_cast<uint4*>((isV ? ga.V_out : ga.K_out) + (out_row0 + first + r) * ga.row_chunks * 16) + chunk;
-      *out = __ldg(src);
+    // four chunks per thread and round, the index loads first and then the row loads, so that they overlap
+    const unsigned int total = mine * (unsigned int)rc2;
+    for (unsigned int e0 = tid; e0 < total; e0 += 4 * kSelThreads) {
+      long long jj[4];
+      uint4 val[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const unsigned int e = e0 + k * kSelThreads;
+        jj[k] = e < total ? dst[first + e / rc2] : 0;
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const unsigned int e = e0 + k * kSelThreads;
+        const int c = (int)(e % rc2);
+        const bool isV = c >= ga.row_chunks;
+        const int chunk = isV ? c - ga.row_chunks : c;
+        const uint4* src = reinterpret_cast<const uint4*>((isV ? Vh + jj[k] * ga.vsn * ga.esize : Kh + jj[k] * ga.ksn * ga.esize)) + chunk;
+        if (e < total) val[k] = __ldg(src);
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const unsigned int e = e0 + k * kSelThreads;
+        if (e >= total) continue;
+        const unsigned int r = e / rc2;
+        const int c = (int)(e - r * rc2);
+        const bool isV = c >= ga.row_chunks;
+        const int chunk = isV ? c - ga.row_chunks : c;
+        uint4* out = reinterpret_cast<uint4*>((isV ? ga.V_out : ga.K_out) + (out_row0 + first + r) * ga.row_chunks * 16) + chunk;
+        *out = val[k];
+      }
     }
   }
   cluster.sync();   // shared memory stays alive until every peer has read cta_counts
