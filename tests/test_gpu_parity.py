@@ -128,6 +128,27 @@ def test_head_sequential_kernel_at_full_size(handle):
     np.testing.assert_allclose(got, ref, rtol=1e-3, atol=0)
 
 
+def test_config2_adaptive_window(handle):
+    """Eq. 10-12 on the 8B-shaped layer: D_front / D_rear from the per-query top-B, window width and shift."""
+    case = CONFIGS["cfg2"]
+    inp = make_inputs(case)
+    B = case.budget
+    probe = oracle_scores(inp, pool_mode=1, beta=1e9, base_width=1, budget=B)
+    delta = abs(probe.D[..., 0] - probe.D[..., 1]).min()
+    assert delta > 0
+    beta = float(delta / 1.5)                     # (D_front - D_rear) / beta = +-1.5 on the head with the smallest gap
+    ref = oracle_scores(inp, pool_mode=1, beta=beta, base_width=5, budget=B)
+    x = (ref.D[..., 0] - ref.D[..., 1]) / beta
+    keep = np.abs(x - np.round(x)) >= 0.05        # heads too close to a rounding boundary are not compared
+    run = GpuRun(handle, inp, adaptive_budget=B)
+    scores = run.score(pool=rk.adaptive_pool(beta, 5, B))
+    used = run.pool_used.cpu().numpy()
+    assert keep.any()
+    np.testing.assert_array_equal(used[keep], ref.pool[keep])
+    for b, h in zip(*np.nonzero(keep)):
+        assert_scores_close(scores[b, h], ref.scores[b, h], TOL[case.dtype])
+
+
 def test_config2_is_deterministic(handle):
     run = GpuRun(handle, make_inputs(CONFIGS["cfg2"]))
     a = run.evict()
