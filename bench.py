@@ -290,6 +290,8 @@ def main():
     # the tensor-core path runs pass 1, the merge and pass 2 in one launch; pooling and the gather run inside the
     # select kernel
     kernel_ids = {"score": rk.KERNEL_PASS2, "pool_select_compact": rk.KERNEL_SELECT}
+    if case.batch * case.n_kv_heads * 8 > 148:      # many rows: the gather runs as its own kernel
+        kernel_ids = {"score": rk.KERNEL_PASS2, "pool_select": rk.KERNEL_SELECT, "compact": rk.KERNEL_COMPACT}
     for _ in range(args.warmup):
         flush.zero_()
         step()

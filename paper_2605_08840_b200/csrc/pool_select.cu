@@ -356,10 +356,12 @@ select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const 
     run_eq += __popc(meq);
   }
   if (ga.K) {
-    // ---- gather the rows this CTA selected: its indices are the contiguous run dst[first, first + mine) ----
-    const unsigned int first = g_before + min(e_before, need_eq);
-    const unsigned int mine = cta_counts[0] + (min(e_before + cta_counts[1], need_eq) - min(e_before, need_eq));
-    __syncthreads();   // the indices written above are visible to the whole CTA
+    // ---- gather: every CTA of the cluster takes an equal share of the row's `keep` indices, whoever emitted them
+    //      (the selected rows may all lie in one CTA's slice) ----
+    cluster.sync();   // all indices of the row are written and visible to the cluster
+    const unsigned int share = ((unsigned int)keep + CS - 1) / CS;
+    const unsigned int first = min((unsigned int)keep, rank * share);
+    const unsigned int mine = min((unsigned int)keep, first + share) - first;
     const int b = row / ga.Hkv, h = row % ga.Hkv;
     const unsigned char* Kh = ga.K + ((long long)b * ga.ksb + (long long)h * ga.ksh) * ga.esize;
     const unsigned char* Vh = ga.V + ((long long)b * ga.vsb + (long long)h * ga.vsh) * ga.esize;

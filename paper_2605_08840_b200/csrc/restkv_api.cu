@@ -354,10 +354,19 @@ restkv_status restkv_evict(restkv_handle* h, const restkv_shape* shape, const vo
   Call c{h, (cudaStream_t)stream};
   float* scores = scores_out ? scores_out : ws.scores;
   if ((s = run_score(c, p, ws, Q_obs, K, V, ema_decay, pool, nullptr, nullptr)) != RESTKV_OK) return s;
-  // pooling (Eq. 13) and the gather (Eq. 14) run inside the select kernel, which also writes the pooled scores
+  // Pooling (Eq. 13) runs inside the select kernel, which also writes the pooled scores.  So does the gather
+  // (Eq. 14) while the select kernel's clusters fit the GPU in one wave; with more (batch, head) rows than that the
+  // stand-alone gather, which spreads over every SM, is the faster one.
+  const bool fuse_gather = p.BH * 8 <= h->sm_count;
   RESTKV_LAUNCH(c, RESTKV_KERNEL_SELECT,
                 launch_select(p.BH, p.n, p.n_kv, budget, ws.I_hat, adaptive ? ws.pool : nullptr, pool->width,
-                              pool->shift, scores, indices, nullptr, &p, K, V, K_out, V_out, c.st), 1);
+                              pool->shift, scores, indices, nullptr, fuse_gather ? &p : nullptr, K, V, K_out, V_out,
+                              c.st), 1);
+  if (!fuse_gather) {
+    const int n_sel = budget < p.n_kv ? budget : p.n_kv;
+    RESTKV_LAUNCH(c, RESTKV_KERNEL_COMPACT,
+                  launch_compact(p, K, V, indices, n_sel, K_out, V_out, h->dev_status, c.st), 1);
+  }
   return RESTKV_OK;
 }
 
