@@ -453,7 +453,15 @@ cudaError_t launch_select(int rows, int n, int n_kv, int budget, const float* I_
     ga.Hkv = gather->Hkv; ga.esize = gather->dtype == RESTKV_BF16 ? 2 : 4; ga.row_chunks = gather->d * ga.esize / 16;
   }
   const int keep = budget < n_kv ? budget : n_kv;
+  // CTAs per row: 8 for long rows, fewer when there are so many rows that all clusters would not be resident at
+  // once (two 1024-thread CTAs per SM) and the slices still fit in shared memory
   int CS = n_kv > 4096 ? 8 : 1;
+  int sms = 148;
+  {
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  }
+  while (CS > 1 && (long long)rows * CS > 2ll * sms && (n_kv + CS / 2 - 1) / (CS / 2) <= kSelMaxSmemKeys / 2) CS >>= 1;
   cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        kSelMaxSmemKeys * (int)sizeof(unsigned int));
   if (e != cudaSuccess) return e;
