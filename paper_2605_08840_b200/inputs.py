@@ -51,7 +51,7 @@ class Case:
         return replace(self, **kw)
 
 
-# The five workloads of the build contract (and the split of the first one).
+# The five workloads (tiny, 8B-shaped layer, 32-layer drift, 128k long context, batched sweep) and the split of the first one.
 CONFIGS: Dict[str, Case] = {
     # tiny single layer; "1a" keeps the K pre-scaling by 1/sqrt(64) literally, "1b" leaves K unscaled
     "cfg1a": Case("cfg1a", 1, 8, 2, 64, 1024, 32, 128, 7, 0, 0.9, "f32", 0, "normal_kscaled", 0),

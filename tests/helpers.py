@@ -1,5 +1,5 @@
 """Shared helpers of the GPU parity tests: run the CUDA library through its C ABI binding and
-compare with the CPU oracle by the acceptance rules of the build contract."""
+compare with the CPU oracle by the acceptance rules written out below."""
 from __future__ import annotations
 
 import numpy as np
