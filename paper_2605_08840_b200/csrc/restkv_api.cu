@@ -413,12 +413,7 @@ restkv_status restkv_decode(restkv_handle* h, const restkv_shape* shape, const v
   Problem p;
   restkv_status s = make_problem(shape, false, &p);
   if (s != RESTKV_OK) return s;
-  if (p.G != 1 && p.G != 2 && p.G != 4 && p.G != 8) return RESTKV_ERR_UNSUPPORTED;
-  const int chunks = p.d * (p.dtype == RESTKV_BF16 ? 2 : 4) / 16;
-  if (chunks != 2 && chunks != 4 && chunks != 8 && chunks != 16 && chunks != 32 && chunks != 64)
-    return RESTKV_ERR_UNSUPPORTED;
-  const size_t need = align256((size_t)p.BH * kDecodeMaxSplits * p.G * (p.d + 2) * sizeof(float));
-  if (!workspace || ((uintptr_t)workspace & 255u) != 0 || workspace_bytes < need) return RESTKV_ERR_WORKSPACE;
+  if (!workspace || ((uintptr_t)workspace & 255u) != 0) return RESTKV_ERR_WORKSPACE;
   Call c{h, (cudaStream_t)stream};
   // bf16, head_dim 128: the decode step is plain attention of up to 128 query rows per KV head, i.e. phases A and B
   // of the tensor-core score kernel with the group's queries padded to its 128 rows.  It needs about 10 MB of
@@ -439,6 +434,13 @@ restkv_status restkv_decode(restkv_handle* h, const restkv_shape* shape, const v
       return RESTKV_OK;
     }
   }
+  // SIMT kernels: 1, 2, 4 or 8 query heads per KV head, rows of 2 to 64 sixteen-byte chunks
+  if (p.G != 1 && p.G != 2 && p.G != 4 && p.G != 8) return RESTKV_ERR_UNSUPPORTED;
+  const int chunks = p.d * (p.dtype == RESTKV_BF16 ? 2 : 4) / 16;
+  if (chunks != 2 && chunks != 4 && chunks != 8 && chunks != 16 && chunks != 32 && chunks != 64)
+    return RESTKV_ERR_UNSUPPORTED;
+  const size_t need = align256((size_t)p.BH * kDecodeMaxSplits * p.G * (p.d + 2) * sizeof(float));
+  if (workspace_bytes < need) return RESTKV_ERR_WORKSPACE;
   int nl = 0;
   cudaError_t e = launch_decode(p, q, Kc, Vc, n_rows, out, lse, (float*)workspace,
                                 decode_splits(p, n_rows, h->sm_count), c.st, &nl);

@@ -357,7 +357,8 @@ def test_compact_bit_exact_and_bad_index_reported(handle):
 
 
 @pytest.mark.parametrize("spec", [("bf16", 32, 8, 128, 2048), ("bf16", 32, 8, 128, 131072), ("f32", 8, 2, 64, 777),
-                                  ("bf16", 4, 4, 64, 100), ("bf16", 16, 2, 256, 1500)])
+                                  ("bf16", 4, 4, 64, 100), ("bf16", 16, 2, 256, 1500), ("bf16", 16, 1, 128, 1000),
+                                  ("bf16", 3, 3, 128, 129), ("bf16", 8, 8, 128, 2)])
 def test_decode_matches_oracle(handle, spec):
     import torch
     dtype, Hq, Hkv, d, rows = spec
