@@ -20,10 +20,19 @@
  *    window query sees every row.  causal_tail = w: the last w rows of K,V are the window tokens'
  *    own pairs; window query i sees trailing row j' only if j' <= i, and those rows receive
  *    the score +inf (the paper's Omega, Eq. 8) so they are always kept.
- *  - Errors are return codes.  A call that returns anything but RESTKV_OK has enqueued nothing.
- *    Conditions detected on the device (a bounded wait that ran out) set a sticky status word
- *    that restkv_poll_status() reads; kernels never trap.
- *  - Calls on one handle must not overlap on the GPU if they share a workspace.
+ *  - Errors are return codes.  A call refused for its arguments, shape, pool parameters or
+ *    workspace (INVALID_ARG, UNSUPPORTED, WORKSPACE) has enqueued nothing; RESTKV_ERR_CUDA may
+ *    come from the middle of a call's launch sequence.  Conditions detected on the device (a
+ *    bounded wait that ran out) set a sticky status word that restkv_poll_status() reads;
+ *    kernels never trap.  Check restkv_poll_status() before using the outputs of a call.
+ *  - Calls must not overlap on the GPU if they share a workspace.
+ *  - The tensor-core kernels behind restkv_score, restkv_evict and restkv_decode (bf16, head_dim 128)
+ *    are persistent: their thread blocks wait for one another inside one launch, so each launch
+ *    needs every SM of the device for itself.  Do not let two such calls, or one of them and any
+ *    other kernel that occupies SMs, run at the same time (two streams without ordering): order
+ *    them on one stream or with events.  If SMs are held by something else the waits are bounded:
+ *    the kernel gives up after about a second, the outputs of that call are undefined, and
+ *    restkv_poll_status() returns RESTKV_ERR_TIMEOUT.
  */
 #ifndef RESTKV_H_
 #define RESTKV_H_
@@ -181,12 +190,17 @@ restkv_status restkv_decode(restkv_handle* h, const restkv_shape* shape, const v
  *    splits as fit (at most 64), so very wide batches run with fewer splits than restkv_decode would use.
  *  - Every GPU that loads the library carries the 2 MiB until the process exits.
  *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that
- *    device current) and remembers it; make that first call outside any stream capture.
+ *    device current) and remembers it; make that first call outside any stream capture.  With CUDA's lazy
+ *    module loading that first call is also the moment the driver places the module, array included, in
+ *    device memory: a host that hands all device memory to its own pool must make one call (any small
+ *    shape) BEFORE it does so, or the first call can fail with RESTKV_ERR_CUDA (out of memory);
+ *    restkv_decode_static_last_cuda_error() then returns the cudaError_t.
  *  - All calls on a device share the one array.  A call overwrites every slot it later reads, so nothing from
  *    an earlier call leaks into a result; but two calls whose kernels overlap on the GPU (different streams,
  *    no ordering between them) race on it.  Order them on one stream or with events.
  *  - There is no device status word on this path and no launch counter; errors are the return code only.
  */
+int restkv_decode_static_last_cuda_error(void);   /* cudaError_t of the last failed CUDA call of the entry below, 0 if none */
 restkv_status restkv_decode_static(const restkv_shape* shape, const void* q, const void* Kc, const void* Vc,
                                    int n_rows, float* out, float* lse, restkv_stream stream);
 

@@ -22,6 +22,7 @@ PATH_AUTO, PATH_SIMT, PATH_TENSOR_CORE, PATH_HEAD_SEQUENTIAL = 0, 1, 2, 3
 EXPORTS = [
     "restkv_create", "restkv_destroy", "restkv_workspace_bytes", "restkv_workspace_bytes_adaptive",
     "restkv_score", "restkv_select", "restkv_compact", "restkv_evict", "restkv_evict_host", "restkv_decode", "restkv_decode_static",
+    "restkv_decode_static_last_cuda_error",
     "restkv_poll_status", "restkv_launch_count", "restkv_last_cuda_error", "restkv_error_string",
     "restkv_set_kernel_path", "restkv_set_profile_events",
 ]
@@ -131,7 +132,7 @@ def decode_static(shape, q, Kc, Vc, n_rows, out, lse=None, stream=None) -> None:
     st = lib.restkv_decode_static(ctypes.byref(shape), _ptr(q), _ptr(Kc), _ptr(Vc), int(n_rows), _ptr(out), _ptr(lse),
                                   _stream_ptr(stream))
     if st != RESTKV_OK:
-        raise RestKVError(st, "restkv_decode_static")
+        raise RestKVError(st, "restkv_decode_static", lib.restkv_decode_static_last_cuda_error())
 
 
 class Handle:

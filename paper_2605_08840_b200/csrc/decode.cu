@@ -297,6 +297,7 @@ constexpr int kMaxDevices = 64;
 std::mutex g_static_mutex;
 float* g_static_scratch_addr[kMaxDevices];   // device address of the array, per device ordinal (null: not looked up yet)
 int g_static_sm_count[kMaxDevices];
+int g_static_last_cuda_error = 0;
 
 // In host code `g_static_decode_scratch` only names the symbol; the address a kernel can use comes from the
 // runtime, for the device that is current.
@@ -348,7 +349,10 @@ extern "C" restkv_status restkv_decode_static(const restkv_shape* shape, const v
   if (per_split > kStaticScratchFloats) return RESTKV_ERR_WORKSPACE;
   float* scratch = nullptr;
   int sm_count = 0;
-  if (static_scratch_for_current_device(&scratch, &sm_count) != cudaSuccess) return RESTKV_ERR_CUDA;
+  if (const cudaError_t es = static_scratch_for_current_device(&scratch, &sm_count); es != cudaSuccess) {
+    g_static_last_cuda_error = (int)es;
+    return RESTKV_ERR_CUDA;
+  }
   int splits = (2 * sm_count + p.BH - 1) / p.BH;
   const int by_rows = (n_rows + 255) / 256;
   if (splits > by_rows) splits = by_rows;
@@ -360,5 +364,8 @@ extern "C" restkv_status restkv_decode_static(const restkv_shape* shape, const v
   // nothing left in the array by an earlier call is ever read and nothing has to be cleared first.
   const cudaError_t e = launch_decode(p, q, Kc, Vc, n_rows, out, lse, scratch, splits, (cudaStream_t)stream,
                                       &n_launches);
+  if (e != cudaSuccess) g_static_last_cuda_error = (int)e;
   return e == cudaSuccess ? RESTKV_OK : RESTKV_ERR_CUDA;
 }
+
+extern "C" int restkv_decode_static_last_cuda_error(void) { return restkv::g_static_last_cuda_error; }

@@ -383,6 +383,18 @@ restkv_status restkv_evict_host(restkv_handle* h, const restkv_shape* shape, con
   if (shape->k_stride_b || shape->k_stride_h || shape->k_stride_n || shape->v_stride_b || shape->v_stride_h ||
       shape->v_stride_n)
     return RESTKV_ERR_INVALID_ARG;
+  // everything restkv_evict would refuse is refused here, before the first copy is enqueued
+  if (budget < 1 || !(ema_decay >= 0.f && ema_decay <= 1.f)) return RESTKV_ERR_INVALID_ARG;
+  if (!aligned16(d_Q) || !aligned16(d_K) || !aligned16(d_V) || !aligned16(d_K_out) || !aligned16(d_V_out))
+    return RESTKV_ERR_INVALID_ARG;
+  if ((s = check_pool(pool, p)) != RESTKV_OK) return s;
+  {
+    Workspace ws_check;
+    const bool adaptive = pool->mode == RESTKV_POOL_ADAPTIVE;
+    const int ws_budget = adaptive ? (pool->budget > budget ? pool->budget : budget) : budget;
+    if ((s = check_ws(p, ws_budget, h->sm_count, adaptive, workspace, workspace_bytes, &ws_check)) != RESTKV_OK)
+      return s;
+  }
   const size_t es = p.dtype == RESTKV_BF16 ? 2 : 4;
   const size_t q_bytes = (size_t)p.batch * p.Hq * p.w * p.d * es;
   const size_t kv_bytes = (size_t)p.BH * p.n_kv * p.d * es;
@@ -418,6 +430,7 @@ restkv_status restkv_decode(restkv_handle* h, const restkv_shape* shape, const v
   // bf16, head_dim 128: the decode step is plain attention of up to 128 query rows per KV head, i.e. phases A and B
   // of the tensor-core score kernel with the group's queries padded to its 128 rows.  It needs about 10 MB of
   // workspace (any restkv_workspace_bytes result has that); with less, or for other shapes, the SIMT kernels run.
+  bool tc_ws_too_small = false;
   if (h->tc_state && h->kernel_path != 1 && p.dtype == RESTKV_BF16 && p.d == 128 && p.G <= 128 && n_rows > 1) {
     Problem pd = p;
     pd.G = 128; pd.Hq = p.Hkv * 128; pd.w = 1; pd.R = 128; pd.tail = 0; pd.n = pd.n_kv = n_rows;
@@ -433,9 +446,11 @@ restkv_status restkv_decode(restkv_handle* h, const restkv_shape* shape, const v
       RESTKV_LAUNCH(c, RESTKV_KERNEL_NONE, launch_decode_extract(p, ws.O_f32, ws.row_M2, out, lse, c.st), 1);
       return RESTKV_OK;
     }
+    tc_ws_too_small = true;
   }
   // SIMT kernels: 1, 2, 4 or 8 query heads per KV head, rows of 2 to 64 sixteen-byte chunks
-  if (p.G != 1 && p.G != 2 && p.G != 4 && p.G != 8) return RESTKV_ERR_UNSUPPORTED;
+  if (p.G != 1 && p.G != 2 && p.G != 4 && p.G != 8)
+    return tc_ws_too_small ? RESTKV_ERR_WORKSPACE : RESTKV_ERR_UNSUPPORTED;
   const int chunks = p.d * (p.dtype == RESTKV_BF16 ? 2 : 4) / 16;
   if (chunks != 2 && chunks != 4 && chunks != 8 && chunks != 16 && chunks != 32 && chunks != 64)
     return RESTKV_ERR_UNSUPPORTED;

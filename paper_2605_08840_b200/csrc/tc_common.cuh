@@ -18,7 +18,6 @@ constexpr uint32_t kBoxBytes = 128 * 64 * 2;     // one [128 rows x 64 bf16] TMA
 constexpr uint32_t kTileBytes = 2 * kBoxBytes;   // a [128 x 128] bf16 operand tile
 constexpr uint32_t kStageBytes = 2 * kTileBytes; // K tile + V tile
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;        // log2 units the running maximum may exceed the reference by
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
