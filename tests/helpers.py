@@ -17,9 +17,9 @@ DECODE_TOL = {"f32": 2e-5}
 def decode_error_bound(q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: float | None = None) -> np.ndarray:
     """Worst-case error of every decode output element on the bf16 path, from the exact softmax weights.
 
-    The tensor-core kernel rounds each unnormalised softmax weight to bf16 (round to nearest: relative error
-    at most 2^-9) before the P V product and divides by the sum of the unrounded weights, so
-    |out_k - exact_k| <= 2^-9 * sum_j A_j |v_jk|.  On top of that come the fp32 rounding of the logits (a few 1e-6
+    The tensor-core kernel rounds each unnormalised softmax weight to bf16 (8 significant bits, round to nearest:
+    relative error at most 2^-8) before the P V product and divides by the sum of the unrounded weights, so
+    |out_k - exact_k| <= 2^-8 * sum_j A_j |v_jk|.  On top of that come the fp32 rounding of the logits (a few 1e-6
     of a weight after exponentiation), exp2 in hardware (2^-22 relative per weight) and fp32 accumulation
     (tensor-core accumulators, the split merge): a further 2^-15 of the same sum is allowed for those.  q [b,Hq,d], K,V [b,Hkv,rows,d] as float32 arrays holding the exact input values."""
     from scipy.special import softmax
@@ -34,7 +34,7 @@ def decode_error_bound(q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: float
             Kh, Vh = K[bi, h].astype(np.float64), np.abs(V[bi, h].astype(np.float64))
             A = softmax(scale * (q[bi, h * G:(h + 1) * G].astype(np.float64) @ Kh.T), axis=-1)
             bound[bi, h * G:(h + 1) * G] = A @ Vh
-    return bound * (2.0 ** -9 + 2.0 ** -15)
+    return bound * (2.0 ** -8 + 2.0 ** -15)
 
 
 def assert_decode_close(out: np.ndarray, ref: np.ndarray, q, K, V, dtype: str):
