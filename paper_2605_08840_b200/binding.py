@@ -17,14 +17,14 @@ RESTKV_OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 1, 2, 3, 4, 5
 BF16, F32 = 0, 1
 POOL_FIXED, POOL_ADAPTIVE = 0, 1
-PATH_AUTO, PATH_SIMT, PATH_TENSOR_CORE, PATH_HEAD_SEQUENTIAL = 0, 1, 2, 3
+PATH_AUTO, PATH_SIMT, PATH_TENSOR_CORE, PATH_HEAD_SEQUENTIAL, PATH_ALL_HEADS = 0, 1, 2, 3, 4
 
 EXPORTS = [
     "restkv_create", "restkv_destroy", "restkv_workspace_bytes", "restkv_workspace_bytes_adaptive",
     "restkv_score", "restkv_select", "restkv_compact", "restkv_evict", "restkv_evict_host", "restkv_decode", "restkv_decode_static",
     "restkv_decode_static_last_cuda_error",
     "restkv_poll_status", "restkv_launch_count", "restkv_last_cuda_error", "restkv_error_string",
-    "restkv_set_kernel_path", "restkv_set_profile_events",
+    "restkv_set_kernel_path", "restkv_set_profile_events", "restkv_set_wait_limit",
 ]
 KERNEL_NONE, KERNEL_PASS1, KERNEL_COMBINE, KERNEL_PASS2, KERNEL_POOL, KERNEL_SELECT, KERNEL_COMPACT = range(7)
 
@@ -87,6 +87,7 @@ def load_library() -> ctypes.CDLL:
     lib.restkv_error_string.restype = ctypes.c_char_p
     lib.restkv_set_kernel_path.argtypes = [vp, ci]
     lib.restkv_set_profile_events.argtypes = [vp, ci, vp, vp]
+    lib.restkv_set_wait_limit.argtypes = [vp, ctypes.c_longlong]
     _lib = lib
     return lib
 
@@ -211,6 +212,9 @@ class Handle:
 
     def set_kernel_path(self, path: int):
         self._check(self._lib.restkv_set_kernel_path(self._h, int(path)), "restkv_set_kernel_path")
+
+    def set_wait_limit(self, sm_clocks: int):
+        self._check(self._lib.restkv_set_wait_limit(self._h, int(sm_clocks)), "restkv_set_wait_limit")
 
     def set_profile_events(self, which: int, start=None, stop=None):
         """start/stop: torch.cuda.Event(enable_timing=True) that have been recorded once, or None to clear."""
