@@ -227,12 +227,11 @@ typedef enum {
 } restkv_kernel_id;
 restkv_status restkv_set_profile_events(restkv_handle* h, int which, void* start, void* stop);
 
-/* Kernel choice: 0 = automatic, 1 = force the fp32 SIMT kernels, 2 = require the tensor-core kernel that 0 picks
- * when the shape qualifies (bf16, head_dim 128, w * group = 128, fixed pooling window): one persistent launch in
- * which the heads follow one another and pass 2 of a head (Eq. 7-9, fed from L2) runs under pass 1 of the next
- * (Eq. 3, fed from DRAM), so K and V are read from DRAM once.  3 and 4 select the earlier tensor-core kernel, whose
- * passes do not overlap: 3 with only as many heads in flight as fit in L2, 4 with every head in flight (K and V
- * read twice). */
+/* Kernel choice: 0 = automatic, 1 = force the fp32 SIMT kernels, 2 = require the tensor-core kernel (one persistent
+ * launch that runs pass 1, the merge of the partial softmax results and pass 2 with every head in flight; what 0
+ * picks when the shape qualifies), 3 = require the tensor-core kernel in its head-sequential form: only as many
+ * heads in flight as fit in L2, so that pass 2 re-reads K and V from there (half the DRAM reads, but two grid
+ * barriers per head; the slower of the two on today's shapes). */
 restkv_status restkv_set_kernel_path(restkv_handle* h, int path);
 
 /* Bound of every device-side wait of the persistent kernels, in SM clocks (default 2e9, about a second).  A wait

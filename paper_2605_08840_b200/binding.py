@@ -17,7 +17,7 @@ RESTKV_OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 1, 2, 3, 4, 5
 BF16, F32 = 0, 1
 POOL_FIXED, POOL_ADAPTIVE = 0, 1
-PATH_AUTO, PATH_SIMT, PATH_TENSOR_CORE, PATH_HEAD_SEQUENTIAL, PATH_ALL_HEADS = 0, 1, 2, 3, 4
+PATH_AUTO, PATH_SIMT, PATH_TENSOR_CORE, PATH_HEAD_SEQUENTIAL = 0, 1, 2, 3
 
 EXPORTS = [
     "restkv_create", "restkv_destroy", "restkv_workspace_bytes", "restkv_workspace_bytes_adaptive",

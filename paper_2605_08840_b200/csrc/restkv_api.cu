@@ -13,8 +13,7 @@ struct restkv_handle {
   void* tc_state;
   long long launches;
   int last_cuda_error;
-  int kernel_path;            // 0 auto, 1 SIMT, 2 tensor core required, 3 / 4 the older tensor-core kernel
-  bool pipe_ok;               // the head-pipelined kernel can be launched
+  int kernel_path;            // 0 auto, 1 SIMT, 2 tensor core required, 3 tensor core in its head-sequential form
   long long wait_limit;       // SM clocks a device-side wait may last
   cudaEvent_t prof_start[7], prof_stop[7];   // per restkv_kernel_id, null = not timed
 };
@@ -52,20 +51,17 @@ size_t plan_workspace(const Problem& p, int budget, int sm_count, bool adaptive,
   w.splits = pass1_splits(p, sm_count);
   // at least the tensor-core kernel's 128 query rows, so that restkv_decode can use it whatever w * group is
   const size_t BH = (size_t)p.BH, R = (size_t)(p.R > 128 ? p.R : 128), d = (size_t)p.d;
-  // partial slots: one per (head, split) on the SIMT path, one per CTA in the persistent tensor-core kernels (two
-  // per CTA in the head-pipelined one, used in turn)
+  // partial slots: one per (head, split) on the SIMT path, one per CTA in the persistent tensor-core kernel
   size_t slots = BH * w.splits;
-  if (slots < 2 * (size_t)sm_count) slots = 2 * (size_t)sm_count;
+  if (slots < (size_t)sm_count) slots = (size_t)sm_count;
   w.part_m = (float*)take(slots * R * sizeof(float));
   w.part_l = (float*)take(slots * R * sizeof(float));
   w.part_O = (float*)take(slots * R * d * sizeof(float));
   w.counters = (unsigned int*)take(1024);
-  w.pipe_counters = (unsigned int*)take(kPipeCounterBytes);
-  w.tile_max = (float*)take(BH * (size_t)((p.n_kv + 63) / 64) * 128 * sizeof(float));
+  w.tile_max = (float*)take(BH * (size_t)((p.n_kv + 127) / 128) * 128 * sizeof(float));
   w.row_M2 = (float*)take(BH * 128 * sizeof(float));
   w.q_pad = (__nv_bfloat16*)take(BH * 128 * 128 * sizeof(__nv_bfloat16));
-  w.vn_stride = (p.n_kv + 127) / 128 * 128;
-  w.vnorm = (float*)take(BH * (size_t)w.vn_stride * sizeof(float));
+  w.vnorm = (float*)take(BH * (size_t)p.n_kv * sizeof(float));
   w.fin_m = (float*)take(BH * R * sizeof(float));
   w.fin_l = (float*)take(BH * R * sizeof(float));
   w.O_f32 = (float*)take(BH * R * d * sizeof(float));
@@ -195,10 +191,6 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
   const bool adaptive = pool->mode == RESTKV_POOL_ADAPTIVE;
   // the tensor-core pass 2 seeds its EMA chain with 1/alpha, so ema_decay = 1 (alpha = 0) runs on the SIMT kernels
   bool use_tc = tc_supported(p) && c.h->tc_state != nullptr && !adaptive && ema_decay < 1.f;
-  // the head-pipelined kernel (the default) takes its temporal weights per query row, so any decay works
-  const bool use_pipe = tc_pipe_supported(p) && c.h->tc_state != nullptr && c.h->pipe_ok && !adaptive &&
-                        (c.h->kernel_path == 0 || c.h->kernel_path == 2);
-  if (use_pipe) use_tc = true;
   if (c.h->kernel_path == 1) use_tc = false;
   if (c.h->kernel_path >= 2 && !use_tc) return RESTKV_ERR_UNSUPPORTED;
   if (!use_tc && !simt_supported(p)) return RESTKV_ERR_UNSUPPORTED;
@@ -209,17 +201,12 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
     if (e == cudaSuccess && adaptive)
       e = cudaMemsetAsync(ws.I_raw, 0, (size_t)p.batch * p.Hq * p.w * p.n * sizeof(float), c.st);
     if (e != cudaSuccess) return c.fail(e);
-  } else if (use_pipe) {
-    // every head in one persistent launch, pass 2 of a head under pass 1 of the next (timed as "pass 2")
-    RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2,
-                  launch_tc_pipe(c.h->tc_state, p, ws, Q, K, V, ema_decay, c.h->sm_count, c.h->wait_limit,
-                                 c.h->dev_status, c.st), 1);
   } else if (use_tc) {
     // pass 1, merge and pass 2 in one persistent launch (timed as "pass 2"); path 3 keeps only as many heads in
     // flight as fit in L2 so that pass 2 re-reads K and V from there
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2,
                   launch_tc_fused(c.h->tc_state, p, ws, Q, K, V, ema_decay, c.h->sm_count, c.h->kernel_path == 3,
-                                  false, c.h->dev_status, c.st), 1);
+                                  false, c.h->wait_limit, c.h->dev_status, c.st), 1);
   } else {
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS1, launch_simt_pass1(p, ws, Q, K, V, c.st), 1);
     RESTKV_LAUNCH(c, RESTKV_KERNEL_COMBINE, launch_combine(p, ws, c.st), 1);
@@ -266,7 +253,6 @@ restkv_status restkv_create(restkv_handle** out) {
   if (e != cudaSuccess) { delete h; return RESTKV_ERR_CUDA; }
   h->tc_state = nullptr;
   if (tc_init(&h->tc_state) != cudaSuccess || tc_fused_init() != cudaSuccess) h->tc_state = nullptr;
-  h->pipe_ok = h->tc_state != nullptr && tc_pipe_init() == cudaSuccess;
   h->wait_limit = 2000000000ll;
   h->launches = 0;
   h->last_cuda_error = 0;
@@ -457,8 +443,8 @@ restkv_status restkv_decode(restkv_handle* h, const restkv_shape* shape, const v
     if (plan_decode_tc(pd.BH, h->sm_count, workspace, &ws) <= workspace_bytes) {
       RESTKV_LAUNCH(c, RESTKV_KERNEL_NONE, launch_decode_pad(p, q, ws.q_pad, c.st), 1);
       RESTKV_LAUNCH(c, RESTKV_KERNEL_NONE,
-                    launch_tc_fused(h->tc_state, pd, ws, ws.q_pad, Kc, Vc, 0.f, h->sm_count, false, true, h->dev_status,
-                                    c.st), 1);
+                    launch_tc_fused(h->tc_state, pd, ws, ws.q_pad, Kc, Vc, 0.f, h->sm_count, false, true, h->wait_limit,
+                                    h->dev_status, c.st), 1);
       RESTKV_LAUNCH(c, RESTKV_KERNEL_NONE, launch_decode_extract(p, ws.O_f32, ws.row_M2, out, lse, c.st), 1);
       return RESTKV_OK;
     }
@@ -523,7 +509,7 @@ restkv_status restkv_set_wait_limit(restkv_handle* h, long long sm_clocks) {
 }
 
 restkv_status restkv_set_kernel_path(restkv_handle* h, int path) {
-  if (!h || path < 0 || path > 4) return RESTKV_ERR_INVALID_ARG;
+  if (!h || path < 0 || path > 3) return RESTKV_ERR_INVALID_ARG;
   h->kernel_path = path;
   return RESTKV_OK;
 }

@@ -32,11 +32,9 @@ struct Workspace {
   float* part_m;          // [slots, R]     partial softmax results: one slot per (head, split) on the SIMT path,
   float* part_l;          // [slots, R]      one per CTA in the persistent tensor-core kernel
   float* part_O;          // [slots, R, d]
-  float* vnorm;           // [BH, vn_stride]  ||v_j||^2 (tensor-core path)
-  int vn_stride;          // n_kv rounded up to a multiple of 128
-  unsigned int* counters; // [256] group barrier counters of the head-sequential kernel
-  unsigned int* pipe_counters;   // [128 groups, 64] counters of the head-pipelined kernel
-  float* tile_max;        // [BH, sub-tiles of 64, 128] row maxima per sub-tile (per tile of 128 in the older kernel)
+  float* vnorm;           // [BH, n_kv]  ||v_j||^2 (tensor-core path)
+  unsigned int* counters; // [256] group barrier counters of the persistent score kernel
+  float* tile_max;        // [BH, tiles, 128] per-tile row maxima of the persistent score kernel
   float* row_M2;          // [BH, 128] log2 normaliser of each query row
   __nv_bfloat16* q_pad;   // [BH, 128, 128] decode queries padded to the kernel's 128 rows
   float* fin_m;           // [BH, R]    row max of the scaled logits (natural units)
@@ -55,7 +53,6 @@ struct Workspace {
 };
 
 constexpr int kDecodeMaxSplits = 64;
-constexpr size_t kPipeCounterBytes = 128 * 64 * sizeof(unsigned int);
 
 int pass1_splits(const Problem& p, int sm_count);
 size_t plan_workspace(const Problem& p, int budget, int sm_count, bool adaptive, void* base, Workspace* ws);
@@ -84,12 +81,7 @@ cudaError_t tc_init(void** state);   // resolves the driver entry point for tens
 cudaError_t tc_fused_init();
 cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
                             const void* V, float ema_decay, int sm_count, bool reuse_l2, bool attention_only,
-                            unsigned int* dev_status, cudaStream_t st);
-bool tc_pipe_supported(const Problem& p);
-cudaError_t tc_pipe_init();
-cudaError_t launch_tc_pipe(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
-                           const void* V, float ema_decay, int sm_count, long long wait_limit,
-                           unsigned int* dev_status, cudaStream_t st);
+                            long long wait_limit, unsigned int* dev_status, cudaStream_t st);
 cudaError_t launch_decode_pad(const Problem& p, const void* q, __nv_bfloat16* q_pad, cudaStream_t st);
 cudaError_t launch_decode_extract(const Problem& p, const float* O_f32, const float* row_M2, float* out, float* lse,
                                   cudaStream_t st);

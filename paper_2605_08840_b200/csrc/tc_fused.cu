@@ -49,6 +49,7 @@ struct FusedArgs {
   long long vsb, vsh, vsn;
   unsigned int* counters;            // [groups] (at most 256), zero at launch
   unsigned int* dev_status;
+  long long wait_limit;              // SM clocks a wait may last
 };
 
 struct FusedBars {
@@ -56,6 +57,7 @@ struct FusedBars {
   uint64_t q_full, k_full[2], k_empty[2], v_full[kFVSlots], v_empty[kFVSlots], s_full[2], p_full[2], pv_done[2];
   // phase C
   uint64_t const_full, kv_full[2], kv_empty[2], acc_full[2], acc_empty[2], red_full[4];
+  uint64_t drain;   // only after a failed wait: completion of the MMAs issued so far
 };
 
 __device__ __forceinline__ void mbar_inval(uint64_t* bar) {
@@ -69,6 +71,14 @@ __device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p) {
   unsigned int v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
+}
+
+// After a wait has failed: wait (bounded, whatever the abort flag says) for a bulk copy or an MMA that this thread
+// itself set in motion, so that nothing is still writing this CTA's shared or tensor memory when it returns.
+__device__ __forceinline__ void wait_issued(uint64_t* bar, uint32_t parity) {
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity & 1u))
+    if (clock64() - t0 > 4000000000ll) return;
 }
 
 // (Re)initialises every mbarrier of the CTA for one phase.  Called by one thread between two __syncthreads.
@@ -94,6 +104,7 @@ __device__ void init_bars(FusedBars* B, bool first) {
     mbar_init(&B->v_empty[i], 1 + 1);   // MMA commit + the warp that reduces ||v||^2
   }
   mbar_init(&B->const_full, 1);
+  mbar_init(&B->drain, 1);
   for (int i = 0; i < 4; ++i) mbar_init(&B->red_full[i], kFWorkerWarps);
   fence_mbar_init();
 }
@@ -102,7 +113,7 @@ __device__ void init_bars(FusedBars* B, bool first) {
 // counter; every other thread calls group_barrier_follow at the same point.  Both return the same verdict (one
 // shared word written between the two synchronisations): false once any wait of the CTA has run out.
 __device__ bool group_barrier(unsigned int* counter, unsigned int target, volatile int* abort_flag, volatile int* go,
-                              unsigned int* dev_status) {
+                              unsigned int* dev_status, long long wait_limit) {
   __syncthreads();
   if (threadIdx.x == 0) {
     // release: everything the CTA wrote before the __syncthreads is visible to whoever acquires the count
@@ -110,7 +121,7 @@ __device__ bool group_barrier(unsigned int* counter, unsigned int target, volati
     const long long t0 = clock64();
     while (ld_acquire_gpu(counter) < target) {
       if (*abort_flag) break;
-      if (clock64() - t0 > 2000000000ll) {
+      if (clock64() - t0 > wait_limit) {
         *abort_flag = 1;
         atomicOr(dev_status, kDevTimeout);
         break;
@@ -162,31 +173,40 @@ __device__ void phase_a_control(const Ctx& cx, const FusedArgs& a, const CUtenso
       mbar_arrive_expect_tx(&B->q_full, kTileBytes);
       tma_load_3d(cx.gen_base + kOffQ, tmQ, &B->q_full, 0, 0, bh);
       tma_load_3d(cx.gen_base + kOffQ + kBoxBytes, tmQ, &B->q_full, 64, 0, bh);
+      int nK = 0, nV = 0;   // K and V tiles requested so far
       for (int it = 0; it < T; ++it) {
         const int ks = it & 1, vs = it % kFVSlots;
         const int j0 = (tile0 + it) * kTile;
-        if (it >= 2 && !mbar_wait(&B->k_empty[ks], ((it >> 1) - 1) & 1, abort_flag, dev_status, kDevTimeout)) break;
+        if (it >= 2 && !mbar_wait(&B->k_empty[ks], ((it >> 1) - 1) & 1, abort_flag, dev_status, kDevTimeout, a.wait_limit)) break;
         uint8_t* dK = cx.gen_base + k_slot_off(ks);
         mbar_arrive_expect_tx(&B->k_full[ks], kTileBytes);
         tma_load_4d(dK, tmK, &B->k_full[ks], 0, j0, h, b);
         tma_load_4d(dK + kBoxBytes, tmK, &B->k_full[ks], 64, j0, h, b);
+        ++nK;
         if (it >= kFVSlots &&
-            !mbar_wait(&B->v_empty[vs], (it / kFVSlots - 1) & 1, abort_flag, dev_status, kDevTimeout))
+            !mbar_wait(&B->v_empty[vs], (it / kFVSlots - 1) & 1, abort_flag, dev_status, kDevTimeout, a.wait_limit))
           break;
         uint8_t* dV = cx.gen_base + v_slot_off(vs);
         mbar_arrive_expect_tx(&B->v_full[vs], kTileBytes);
         tma_load_4d(dV, tmV, &B->v_full[vs], 0, j0, h, b);
         tma_load_4d(dV + kBoxBytes, tmV, &B->v_full[vs], 64, j0, h, b);
+        ++nV;
+      }
+      if (*(volatile int*)abort_flag) {
+        // a wait of this CTA has failed: the tiles requested last may still be on their way into shared memory
+        wait_issued(&B->q_full, 0);
+        for (int i = max(0, nK - 2); i < nK; ++i) wait_issued(&B->k_full[i & 1], (uint32_t)(i >> 1));
+        for (int i = max(0, nV - kFVSlots); i < nV; ++i) wait_issued(&B->v_full[i % kFVSlots], (uint32_t)(i / kFVSlots));
       }
     }
   } else if (warp == 1) {
     // S(it), then O += P V of tile it - 1
     if (lane == 0 && T > 0) {
-      bool ok = mbar_wait(&B->q_full, 0, abort_flag, dev_status, kDevTimeout);
+      bool ok = mbar_wait(&B->q_full, 0, abort_flag, dev_status, kDevTimeout, a.wait_limit);
       for (int it = 0; ok && it <= T; ++it) {
         if (it < T) {
           const int ks = it & 1, g = it & 1;
-          if (!mbar_wait(&B->k_full[ks], (it >> 1) & 1, abort_flag, dev_status, kDevTimeout)) break;
+          if (!mbar_wait(&B->k_full[ks], (it >> 1) & 1, abort_flag, dev_status, kDevTimeout, a.wait_limit)) break;
           tc_fence_after();
           // S_g may be overwritten: O += P V of tile it - 2 (which read P_g) was issued earlier and MMAs run in order
           mma_tile_kk(tmem + (uint32_t)g * 128u, cx.smem_base + kOffQ, cx.smem_base + k_slot_off(ks), false);
@@ -195,8 +215,8 @@ __device__ void phase_a_control(const Ctx& cx, const FusedArgs& a, const CUtenso
         }
         if (it >= 1) {
           const int pt = it - 1, g = pt & 1, vs = pt % kFVSlots;
-          if (!mbar_wait(&B->p_full[g], (pt >> 1) & 1, abort_flag, dev_status, kDevTimeout)) break;
-          if (!mbar_wait(&B->v_full[vs], (pt / kFVSlots) & 1, abort_flag, dev_status, kDevTimeout)) break;
+          if (!mbar_wait(&B->p_full[g], (pt >> 1) & 1, abort_flag, dev_status, kDevTimeout, a.wait_limit)) break;
+          if (!mbar_wait(&B->v_full[vs], (pt / kFVSlots) & 1, abort_flag, dev_status, kDevTimeout, a.wait_limit)) break;
           tc_fence_after();
           // A = P_g in TMEM (16 tokens = 8 packed columns per K step), B = V tile, MN-major
           const uint32_t vaddr = cx.smem_base + v_slot_off(vs);
@@ -212,6 +232,10 @@ __device__ void phase_a_control(const Ctx& cx, const FusedArgs& a, const CUtenso
           umma_commit(&B->v_empty[vs]);
         }
       }
+      if (*(volatile int*)abort_flag) {   // let the MMAs already issued finish before the CTA goes on to return
+        umma_commit(&B->drain);
+        wait_issued(&B->drain, 0);
+      }
     }
   } else if (warp < kFFirstWorker) {
     // ---------------- ||v||^2: one warp takes the even tiles, the other the odd ones; lane = 4 tokens ----------------
@@ -220,7 +244,7 @@ __device__ void phase_a_control(const Ctx& cx, const FusedArgs& a, const CUtenso
     for (int it = 0; it < T && ok; ++it) {
       const int vs = it % kFVSlots;
       // both warps wait for every tile so that neither falls a whole phase behind a slot's barrier
-      ok = mbar_wait(&B->v_full[vs], (it / kFVSlots) & 1, abort_flag, dev_status, kDevTimeout);
+      ok = mbar_wait(&B->v_full[vs], (it / kFVSlots) & 1, abort_flag, dev_status, kDevTimeout, a.wait_limit);
       if (!ok || (it & 1) != vg) continue;
       const uint8_t* vt = cx.gen_base + v_slot_off(vs);
       float vn[4];
@@ -289,7 +313,7 @@ __device__ void phase_a_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
   bool ok = true;
   int uses = 0;                             // tiles this warpgroup has processed
   for (int it = g; it < T; it += 2, ++uses) {
-    ok = ok && mbar_wait(&B->s_full[g], (uint32_t)uses & 1u, abort_flag, dev_status, kDevTimeout);
+    ok = ok && mbar_wait(&B->s_full[g], (uint32_t)uses & 1u, abort_flag, dev_status, kDevTimeout, a.wait_limit);
     if (ok) tc_fence_after();
     const int j0 = (tile0 + it) * kTile + hf * 64;
     const bool ragged = j0 + 64 > n;   // rows past the scored prefix: window rows (causal) or padding
@@ -373,7 +397,7 @@ __device__ void phase_a_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
     tc_fence_before();
     mbar_arrive(&B->p_full[g]);
   }
-  if (uses > 0 && ok) ok = mbar_wait(&B->pv_done[g], (uint32_t)(uses - 1) & 1u, abort_flag, dev_status, kDevTimeout);
+  if (uses > 0 && ok) ok = mbar_wait(&B->pv_done[g], (uint32_t)(uses - 1) & 1u, abort_flag, dev_status, kDevTimeout, a.wait_limit);
   if (ok && uses > 0) tc_fence_after();
   const bool have = ok && uses > 0;
   const float m_mine = have ? m_ref : -INFINITY, l_mine = have ? l2.x + l2.y : 0.f;
@@ -576,22 +600,28 @@ __device__ void phase_c_control(const Ctx& cx, const FusedArgs& a, const CUtenso
       tma_load_3d(cx.gen_base + kOffO, tmO, &B->const_full, 0, 0, bh);
       tma_load_3d(cx.gen_base + kOffO + kBoxBytes, tmO, &B->const_full, 64, 0, bh);
       tma_load_3d(cx.gen_base + kOffAug, tmAug, &B->const_full, 0, 0, bh);
+      int nS = pre;   // stages requested so far
       for (int it = pre; it < T; ++it) {   // the first `pre` tiles were requested before the group barriers
         const int s = it & 1;
-        if (it >= 2 && !mbar_wait(&B->kv_empty[s], ((it >> 1) - 1) & 1, abort_flag, dev_status, kDevTimeout)) break;
+        if (it >= 2 && !mbar_wait(&B->kv_empty[s], ((it >> 1) - 1) & 1, abort_flag, dev_status, kDevTimeout, a.wait_limit)) break;
         load_stage_c(cx, tmK, tmV, b, h, (tile0 + T - 1 - it) * kTile, s);
+        ++nS;
+      }
+      if (*(volatile int*)abort_flag) {
+        wait_issued(&B->const_full, 0);
+        for (int i = max(0, nS - 2); i < nS; ++i) wait_issued(&B->kv_full[i & 1], (uint32_t)(i >> 1));
       }
     }
   } else if (warp == 1) {
     if (lane == 0 && T > 0) {
-      bool ok = mbar_wait(&B->const_full, 0, abort_flag, dev_status, kDevTimeout);
+      bool ok = mbar_wait(&B->const_full, 0, abort_flag, dev_status, kDevTimeout, a.wait_limit);
       const uint32_t sQ = cx.smem_base + kOffQ, sO = cx.smem_base + kOffO, sAug = cx.smem_base + kOffAug;
       const uint64_t ones_desc = make_smem_desc(cx.smem_base + kOffOnes, 16, 0);   // every 8-row group reads the same block
       const uint64_t aug_s = kmajor_desc(sAug), aug_c = kmajor_desc(sAug + 32u);
       for (int it = 0; ok && it < T; ++it) {
         const int s = it & 1;
-        if (!mbar_wait(&B->kv_full[s], (it >> 1) & 1, abort_flag, dev_status, kDevTimeout)) break;
-        if (it >= 2 && !mbar_wait(&B->acc_empty[s], ((it >> 1) - 1) & 1, abort_flag, dev_status, kDevTimeout)) break;
+        if (!mbar_wait(&B->kv_full[s], (it >> 1) & 1, abort_flag, dev_status, kDevTimeout, a.wait_limit)) break;
+        if (it >= 2 && !mbar_wait(&B->acc_empty[s], ((it >> 1) - 1) & 1, abort_flag, dev_status, kDevTimeout, a.wait_limit)) break;
         tc_fence_after();
         const uint32_t sK = cx.smem_base + k_slot_off(2 * s), sV = sK + kTileBytes;
         const uint32_t tS = tmem + (uint32_t)s * 256u, tC = tS + 128u;
@@ -601,6 +631,10 @@ __device__ void phase_c_control(const Ctx& cx, const FusedArgs& a, const CUtenso
         umma_ss(tC, ones_desc, aug_c, kIdescKK, true);        //   + ||o||^2
         umma_commit(&B->acc_full[s]);
         umma_commit(&B->kv_empty[s]);
+      }
+      if (*(volatile int*)abort_flag) {
+        umma_commit(&B->drain);
+        wait_issued(&B->drain, 0);
       }
     }
   }
@@ -677,11 +711,11 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
     // allow after every warp has moved past this point.
     if (it > 0 && cgp == 0) {
       const int rs = (it - 1) & 3;
-      ok = ok && mbar_wait(&B->red_full[rs], (uint32_t)((it - 1) >> 2) & 1u, abort_flag, dev_status, kDevTimeout);
+      ok = ok && mbar_wait(&B->red_full[rs], (uint32_t)((it - 1) >> 2) & 1u, abort_flag, dev_status, kDevTimeout, a.wait_limit);
       const int jp = (tile0 + T - it) * kTile + t;
       if (ok && jp < n) I_head[jp] = (red[rs][0][t] + red[rs][1][t]) + (red[rs][2][t] + red[rs][3][t]);
     }
-    ok = ok && mbar_wait(&B->acc_full[s], par, abort_flag, dev_status, kDevTimeout);
+    ok = ok && mbar_wait(&B->acc_full[s], par, abort_flag, dev_status, kDevTimeout, a.wait_limit);
     float tot = 0.f;
     if (ok) {
       tc_fence_after();
@@ -771,7 +805,7 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
   }
   if (T > 0 && cgp == 0) {
     const int rs = (T - 1) & 3;
-    ok = ok && mbar_wait(&B->red_full[rs], (uint32_t)((T - 1) >> 2) & 1u, abort_flag, dev_status, kDevTimeout);
+    ok = ok && mbar_wait(&B->red_full[rs], (uint32_t)((T - 1) >> 2) & 1u, abort_flag, dev_status, kDevTimeout, a.wait_limit);
     const int jl = tile0 * kTile + t;   // the last tile processed is the first of the share
     if (ok && jl < n) I_head[jl] = (red[rs][0][t] + red[rs][1][t]) + (red[rs][2][t] + red[rs][3][t]);
   }
@@ -806,9 +840,15 @@ __device__ void control_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, 
     if (threadIdx.x == 0)
       for (int it = 0; it < pre; ++it)
         load_stage_c(cx, tmK, tmV, bh / a.Hkv, bh % a.Hkv, (pl.tile0 + pl.T2 - 1 - it) * kTile, it);
-    if (!group_barrier(counter, (++epoch) * (unsigned int)a.cpg, abort_flag, go, a.dev_status)) break;
+    bool through = group_barrier(counter, (++epoch) * (unsigned int)a.cpg, abort_flag, go, a.dev_status, a.wait_limit);
     // phase B belongs to the worker warps
-    if (!group_barrier(counter, (++epoch) * (unsigned int)a.cpg, abort_flag, go, a.dev_status)) break;
+    through = through && group_barrier(counter, (++epoch) * (unsigned int)a.cpg, abort_flag, go, a.dev_status, a.wait_limit);
+    if (!through) {
+      // a barrier gave up: the stages requested above must have landed before this CTA may return
+      if (threadIdx.x == 0)
+        for (int it = 0; it < pre; ++it) wait_issued(&bars->kv_full[it], 0);
+      break;
+    }
     tc_fence_after();
     phase_c_control<kW>(cx, a, tmO, tmAug, tmK, tmV, bh, pl.tile0, pl.T2, pre);
     tc_fence_before();
@@ -995,7 +1035,7 @@ cudaError_t tc_fused_init() {
 // with the timeout status instead of hanging.  (A cooperative launch would guarantee residency but costs ~25 us.)
 cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
                             const void* V, float ema_decay, int sm_count, bool reuse_l2, bool attention_only,
-                            unsigned int* dev_status, cudaStream_t st) {
+                            long long wait_limit, unsigned int* dev_status, cudaStream_t st) {
   TcState* ts = (TcState*)state;
   CUtensorMap tmQ, tmK, tmV, tmO, tmAug;
   if (!make_rows_map(ts, &tmQ, Q, p.BH) || !make_rows_map(ts, &tmO, ws.O_m2, p.BH) ||
@@ -1011,6 +1051,7 @@ cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, 
   a.O_f32 = ws.O_f32; a.O_m2 = ws.O_m2; a.aug = ws.aug; a.vnorm = ws.vnorm; a.I_hat = ws.I_hat;
   a.V = (const __nv_bfloat16*)V; a.vsb = p.vsb; a.vsh = p.vsh; a.vsn = p.vsn;
   a.counters = ws.counters; a.tile_max = ws.tile_max; a.row_M2 = ws.row_M2; a.dev_status = dev_status;
+  a.wait_limit = wait_limit;
   cudaError_t e = cudaMemsetAsync(ws.counters, 0, 1024, st);
   if (e != cudaSuccess) return e;
   const dim3 grid(a.groups * a.cpg), block(kFThreads);

@@ -429,6 +429,29 @@ def test_decode_over_compacted_cache_of_config2(handle):
     assert_decode_close(out.cpu().numpy(), ref, q, Kc, Vc, "bf16")
 
 
+# ------------------------------------------------------------------ a device-side wait that runs out
+def test_wait_limit_runs_out_and_the_handle_recovers(handle):
+    """With a wait limit of one SM clock the first CTA to reach a group barrier of the persistent score kernel gives
+    up at once (its peers have not arrived yet): the kernel must stop issuing work, let what it already issued land,
+    return by itself and leave RESTKV_ERR_TIMEOUT in the sticky status; with the default limit restored the same
+    handle and workspace then give the oracle's scores."""
+    case = Case("timeout", 1, 4, 1, 128, 2000, 32, 100, 5, 0, 0.9, "bf16", 0, "normal", 123)
+    inp = make_inputs(case)
+    run = GpuRun(handle, inp)
+    handle.set_kernel_path(rk.PATH_TENSOR_CORE)
+    try:
+        handle.set_wait_limit(1)
+        handle.evict(run.shape, run.Q, run.K, run.V, case.ema_decay, run.pool(), run.budget, run.indices, run.K_out,
+                     run.V_out, run.ws, scores_out=run.scores)
+        run.torch.cuda.synchronize()
+        assert handle.poll_status() == rk.ERR_TIMEOUT
+        assert handle.poll_status() == rk.RESTKV_OK          # the sticky word is cleared by the poll
+    finally:
+        handle.set_wait_limit(2_000_000_000)
+        handle.set_kernel_path(rk.PATH_AUTO)
+    full_check(handle, inp)
+
+
 # ------------------------------------------------------------------ API misuse: error codes, never a fault
 def test_api_rejects_bad_arguments(handle):
     import torch
