@@ -234,6 +234,12 @@ restkv_status restkv_set_profile_events(restkv_handle* h, int which, void* start
  * barriers per head; the slower of the two on today's shapes). */
 restkv_status restkv_set_kernel_path(restkv_handle* h, int path);
 
+/* restkv_evict on the tensor-core path with a fixed window lets the score kernel itself pool (Eq. 13), select and
+ * gather (Eq. 14) each head, with the head's own thread blocks, as soon as the head's scores are complete (default:
+ * on).  With 0 the pooling, selection and gather always run as the separate kernel that other paths use; the results
+ * are the same.  Meant for timing the two against each other. */
+restkv_status restkv_set_fused_select(restkv_handle* h, int on);
+
 /* Bound of every device-side wait of the persistent kernels, in SM clocks (default 2e9, about a second).  A wait
  * that runs out sets the sticky status (RESTKV_ERR_TIMEOUT from restkv_poll_status), the kernel stops issuing
  * work, waits for what it already issued and returns; the call's outputs are then undefined.  Meant for tests of

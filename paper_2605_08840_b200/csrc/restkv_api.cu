@@ -14,6 +14,7 @@ struct restkv_handle {
   long long launches;
   int last_cuda_error;
   int kernel_path;            // 0 auto, 1 SIMT, 2 tensor core required, 3 tensor core in its head-sequential form
+  bool fused_select;          // restkv_evict lets the tensor-core score kernel pool, select and gather when it can
   long long wait_limit;       // SM clocks a device-side wait may last
   cudaEvent_t prof_start[7], prof_stop[7];   // per restkv_kernel_id, null = not timed
 };
@@ -60,6 +61,8 @@ size_t plan_workspace(const Problem& p, int budget, int sm_count, bool adaptive,
   w.counters = (unsigned int*)take(1024);
   w.tile_max = (float*)take(BH * (size_t)((p.n_kv + 127) / 128) * 128 * sizeof(float));
   w.row_M2 = (float*)take(BH * 128 * sizeof(float));
+  w.sel_hist = (unsigned int*)take(tc_fused_select_hist_words(p.BH) * sizeof(unsigned int));
+  w.sel_sfx = (unsigned int*)take(tc_fused_select_sfx_words(p.BH, sm_count) * sizeof(unsigned int));
   w.q_pad = (__nv_bfloat16*)take(BH * 128 * 128 * sizeof(__nv_bfloat16));
   w.vnorm = (float*)take(BH * (size_t)p.n_kv * sizeof(float));
   w.fin_m = (float*)take(BH * R * sizeof(float));
@@ -187,7 +190,7 @@ struct Call {
 // null the caller pools (the fused path does it inside the select kernel).
 static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, const void* Q, const void* K,
                                const void* V, float ema_decay, const restkv_pool_params* pool, float* scores,
-                               int32_t* pool_used) {
+                               int32_t* pool_used, const FusedSelect* sel = nullptr, bool* sel_done = nullptr) {
   const bool adaptive = pool->mode == RESTKV_POOL_ADAPTIVE;
   // the tensor-core pass 2 seeds its EMA chain with 1/alpha, so ema_decay = 1 (alpha = 0) runs on the SIMT kernels
   bool use_tc = tc_supported(p) && c.h->tc_state != nullptr && !adaptive && ema_decay < 1.f;
@@ -204,9 +207,13 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
   } else if (use_tc) {
     // pass 1, merge and pass 2 in one persistent launch (timed as "pass 2"); path 3 keeps only as many heads in
     // flight as fit in L2 so that pass 2 re-reads K and V from there
+    const bool reuse_l2 = c.h->kernel_path == 3;
+    const bool with_sel = sel && c.h->fused_select &&
+                          tc_fused_select_supported(p, c.h->sm_count, reuse_l2, sel->keep, sel->W, sel->gamma);
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2,
-                  launch_tc_fused(c.h->tc_state, p, ws, Q, K, V, ema_decay, c.h->sm_count, c.h->kernel_path == 3,
-                                  false, c.h->wait_limit, c.h->dev_status, c.st), 1);
+                  launch_tc_fused(c.h->tc_state, p, ws, Q, K, V, ema_decay, c.h->sm_count, reuse_l2, false,
+                                  c.h->wait_limit, with_sel ? sel : nullptr, c.h->dev_status, c.st), 1);
+    if (sel_done) *sel_done = with_sel;
   } else {
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS1, launch_simt_pass1(p, ws, Q, K, V, c.st), 1);
     RESTKV_LAUNCH(c, RESTKV_KERNEL_COMBINE, launch_combine(p, ws, c.st), 1);
@@ -254,6 +261,7 @@ restkv_status restkv_create(restkv_handle** out) {
   h->tc_state = nullptr;
   if (tc_init(&h->tc_state) != cudaSuccess || tc_fused_init() != cudaSuccess) h->tc_state = nullptr;
   h->wait_limit = 2000000000ll;
+  h->fused_select = true;
   h->launches = 0;
   h->last_cuda_error = 0;
   h->kernel_path = 0;
@@ -355,7 +363,15 @@ restkv_status restkv_evict(restkv_handle* h, const restkv_shape* shape, const vo
   if ((s = check_ws(p, ws_budget, h->sm_count, adaptive, workspace, workspace_bytes, &ws)) != RESTKV_OK) return s;
   Call c{h, (cudaStream_t)stream};
   float* scores = scores_out ? scores_out : ws.scores;
-  if ((s = run_score(c, p, ws, Q_obs, K, V, ema_decay, pool, nullptr, nullptr)) != RESTKV_OK) return s;
+  // With a fixed window the tensor-core score kernel pools, selects and gathers each head itself, right after the
+  // head's scores are complete and with the head's own CTAs; otherwise the kernels below do.
+  const int keep_rows = budget < p.n_kv ? budget : p.n_kv;
+  FusedSelect sel{keep_rows, pool->width, pool->shift, scores, indices, K_out, V_out};
+  bool sel_done = false;
+  if ((s = run_score(c, p, ws, Q_obs, K, V, ema_decay, pool, nullptr, nullptr, adaptive ? nullptr : &sel, &sel_done)) !=
+      RESTKV_OK)
+    return s;
+  if (sel_done) return RESTKV_OK;
   // Pooling (Eq. 13) runs inside the select kernel, which also writes the pooled scores.  So does the gather
   // (Eq. 14) while the select kernel's clusters fit the GPU in one wave; with more (batch, head) rows than that the
   // stand-alone gather, which spreads over every SM, is the faster one.
@@ -444,7 +460,7 @@ restkv_status restkv_decode(restkv_handle* h, const restkv_shape* shape, const v
       RESTKV_LAUNCH(c, RESTKV_KERNEL_NONE, launch_decode_pad(p, q, ws.q_pad, c.st), 1);
       RESTKV_LAUNCH(c, RESTKV_KERNEL_NONE,
                     launch_tc_fused(h->tc_state, pd, ws, ws.q_pad, Kc, Vc, 0.f, h->sm_count, false, true, h->wait_limit,
-                                    h->dev_status, c.st), 1);
+                                    nullptr, h->dev_status, c.st), 1);
       RESTKV_LAUNCH(c, RESTKV_KERNEL_NONE, launch_decode_extract(p, ws.O_f32, ws.row_M2, out, lse, c.st), 1);
       return RESTKV_OK;
     }
@@ -499,6 +515,12 @@ restkv_status restkv_set_profile_events(restkv_handle* h, int which, void* start
   if ((start == nullptr) != (stop == nullptr)) return RESTKV_ERR_INVALID_ARG;
   h->prof_start[which] = (cudaEvent_t)start;
   h->prof_stop[which] = (cudaEvent_t)stop;
+  return RESTKV_OK;
+}
+
+restkv_status restkv_set_fused_select(restkv_handle* h, int on) {
+  if (!h) return RESTKV_ERR_INVALID_ARG;
+  h->fused_select = on != 0;
   return RESTKV_OK;
 }
 

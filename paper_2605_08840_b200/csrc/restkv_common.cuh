@@ -36,6 +36,8 @@ struct Workspace {
   unsigned int* counters; // [256] group barrier counters of the persistent score kernel
   float* tile_max;        // [BH, tiles, 128] per-tile row maxima of the persistent score kernel
   float* row_M2;          // [BH, 128] log2 normaliser of each query row
+  unsigned int* sel_hist; // [BH, 4, 256] digit histograms of the selection inside the score kernel
+  unsigned int* sel_sfx;  // [BH, SMs, 4, 260] per-CTA suffix sums of those histograms
   __nv_bfloat16* q_pad;   // [BH, 128, 128] decode queries padded to the kernel's 128 rows
   float* fin_m;           // [BH, R]    row max of the scaled logits (natural units)
   float* fin_l;           // [BH, R]    sum of exp(s - m)
@@ -53,6 +55,15 @@ struct Workspace {
 };
 
 constexpr int kDecodeMaxSplits = 64;
+
+// Pooling window, budget and outputs of the selection that the tensor-core score kernel can run itself.
+struct FusedSelect {
+  int keep, W, gamma;
+  float* scores;          // [BH, n_kv] pooled scores
+  int32_t* indices;       // [BH, keep]
+  void* K_out;            // [BH, keep, d]
+  void* V_out;
+};
 
 int pass1_splits(const Problem& p, int sm_count);
 size_t plan_workspace(const Problem& p, int budget, int sm_count, bool adaptive, void* base, Workspace* ws);
@@ -81,7 +92,10 @@ cudaError_t tc_init(void** state);   // resolves the driver entry point for tens
 cudaError_t tc_fused_init();
 cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
                             const void* V, float ema_decay, int sm_count, bool reuse_l2, bool attention_only,
-                            long long wait_limit, unsigned int* dev_status, cudaStream_t st);
+                            long long wait_limit, const FusedSelect* sel, unsigned int* dev_status, cudaStream_t st);
+bool tc_fused_select_supported(const Problem& p, int sm_count, bool reuse_l2, int keep, int W, int gamma);
+size_t tc_fused_select_sfx_words(int BH, int sm_count);
+size_t tc_fused_select_hist_words(int BH);
 cudaError_t launch_decode_pad(const Problem& p, const void* q, __nv_bfloat16* q_pad, cudaStream_t st);
 cudaError_t launch_decode_extract(const Problem& p, const float* O_f32, const float* row_M2, float* out, float* lse,
                                   cudaStream_t st);

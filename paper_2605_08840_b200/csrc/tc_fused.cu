@@ -50,7 +50,24 @@ struct FusedArgs {
   unsigned int* counters;            // [groups] (at most 256), zero at launch
   unsigned int* dev_status;
   long long wait_limit;              // SM clocks a wait may last
+  // Pooling (Eq. 13), top-B selection and row gather (Eq. 14) of every head right after its phase C, by the head's own
+  // group of CTAs (sel_keep = 0: not done here).
+  int sel_keep, sel_W, sel_gamma;
+  float* sel_scores;                 // [BH, n_kv] pooled scores
+  int32_t* sel_indices;              // [BH, keep]
+  unsigned int* sel_hist;            // [BH, 4, 256] digit histograms of the group, zero at launch
+  unsigned int* sel_sfx;             // [BH, cpg, 4, kSfxStride] per CTA: suffix sums of its own digit histograms
+  const __nv_bfloat16* K;
+  long long ksb, ksh, ksn;
+  __nv_bfloat16* K_out;              // [BH, keep, 128]
+  __nv_bfloat16* V_out;
 };
+
+constexpr int kSelPasses = 4;                     // 8-bit digits of the 32-bit keys, from the top
+constexpr int kSfxStride = 260;                   // 257 suffix sums per (CTA, pass), padded
+constexpr int kSelMaxKeys = 20480;                // scores of one CTA's share of a head kept in shared memory
+constexpr int kSelHalo = 64;                      // widest reach of the pooling window beyond the share
+constexpr int kSelBarriers = 2 + kSelPasses;      // group barriers of the selection phase
 
 struct FusedBars {
   // phase A
@@ -816,6 +833,245 @@ struct Plan {
   int group, rank, tile0, T1, T2;
 };
 
+// Scores map to unsigned keys whose order matches the float order.
+__device__ __forceinline__ unsigned int sel_key(float x) {
+  const unsigned int u = __float_as_uint(x);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Pooling, selection and gather of one head by its group of CTAs, run by the sixteen worker warps right after the
+// head's phase C (the control warps run the matching group barriers).  CTA `rank` owns the tokens of its tiles, a
+// contiguous run [j_first, j_first + cnt) of the head; lower ranks own lower tokens.
+//   1. after a group barrier (every I_hat of the head is written): box mean of Eq. 13 over the own run (taps staged
+//      in shared memory, summed in ascending order), pooled scores to global memory, their keys kept in shared memory;
+//   2. four radix passes over 8-bit digits from the top: per-warp histograms of the keys that match the digits
+//      chosen so far, summed per CTA, added to the group's histogram in global memory; the CTA also publishes the
+//      suffix sums of its own histogram.  After the pass's group barrier every CTA finds the digit that holds the
+//      keep-th largest key and adds up, from the suffix sums of the lower ranks, how many keys above it they hold;
+//   3. ordered emit: indices ascending, every key above the threshold key T plus the first ones equal to it (the
+//      lower index wins ties), at positions that continue the lower ranks' counts;
+//   4. after a last group barrier the rows of the head's `keep` indices are copied, an equal share per CTA.
+// Returns false once a wait of the CTA has run out.
+__device__ bool select_worker(const Ctx& cx, const FusedArgs& a, const Plan& pl, int bh, volatile int* go) {
+  const int tid = (int)threadIdx.x - kFFirstWorker * 32, lane = cx.lane, wq = cx.warp - kFFirstWorker;
+  constexpr int kT = kFWorkerWarps * 32;
+  const int n = a.n, n_kv = a.n_kv, keep = a.sel_keep;
+  const int j_first = pl.tile0 * kTile;
+  const int cnt = max(0, min(n_kv, (pl.tile0 + pl.T1) * kTile) - j_first);
+  unsigned int* wh = reinterpret_cast<unsigned int*>(cx.gen_base + kOffQ);   // [16 warps][256]
+  unsigned int* hist_s = wh + kFWorkerWarps * 256;                            // [256]
+  unsigned int* misc = hist_s + 256;                                          // digit, remaining, gt/eq of lower ranks, warp sums
+  unsigned int* keys = misc + 64;                                             // [kSelMaxKeys]
+  float* staged = reinterpret_cast<float*>(keys + kSelMaxKeys);               // [kSelMaxKeys + 2 * kSelHalo]
+  static_assert((kFWorkerWarps * 256 + 256 + 64 + 2 * kSelMaxKeys + 2 * kSelHalo) * 4 <= kOffRing + kFRing * kTileBytes,
+                "the selection's buffers must fit the operand tiles and the ring");
+
+  if (!group_barrier_follow(go)) return false;   // every CTA of the group has written its I_hat of this head
+  // ---- 1. pooling ----
+  {
+    const int W = a.sel_W, gamma = a.sel_gamma, half = W / 2;
+    const float* src = a.I_hat + (long long)bh * n;
+    const long long lo64 = (long long)j_first - half + gamma, hi64 = (long long)j_first + cnt - 1 + half + gamma;
+    const int s_lo = lo64 < 0 ? 0 : (int)(lo64 < n ? lo64 : n), s_hi = hi64 > n - 1 ? n - 1 : (int)(hi64 > -1 ? hi64 : -1);
+    for (int t0 = s_lo + tid; t0 <= s_hi; t0 += 8 * kT) {   // several loads in flight per thread
+      float v[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int t = t0 + k * kT;
+        v[k] = t <= s_hi ? __ldcg(src + t) : 0.f;
+      }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int t = t0 + k * kT;
+        if (t <= s_hi) staged[t - s_lo] = v[k];
+      }
+    }
+    named_barrier_sync(1, kT);
+    float* srow = a.sel_scores + (long long)bh * n_kv + j_first;
+    const float fw = (float)W;
+    for (int jj = tid; jj < cnt; jj += kT) {
+      const int j = j_first + jj;
+      float out = INFINITY;
+      if (j < n) {
+        const long long a64 = (long long)j - half + gamma, b64 = (long long)j + half + gamma;
+        const int ta = a64 < s_lo ? s_lo : (int)(a64 <= s_hi ? a64 : s_hi + 1), tb = b64 > s_hi ? s_hi : (int)(b64 >= s_lo ? b64 : s_lo - 1);
+        float acc = 0.f;
+        for (int t = ta; t <= tb; ++t) acc += staged[t - s_lo];
+        out = acc / fw;
+      }
+      srow[jj] = out;
+      keys[jj] = sel_key(out);
+    }
+    if (tid < 4) misc[2 + tid] = 0u;
+    named_barrier_sync(1, kT);
+  }
+  // ---- 2. radix passes ----
+  unsigned int prefix = 0, remaining = (unsigned int)keep;
+  unsigned int* sfx_mine = a.sel_sfx + ((long long)bh * a.cpg + pl.rank) * kSelPasses * kSfxStride;
+#pragma unroll 1
+  for (int p = 0; p < kSelPasses; ++p) {
+    const int lo = 24 - 8 * p;
+    for (int b = tid; b < kFWorkerWarps * 256; b += kT) wh[b] = 0u;
+    named_barrier_sync(1, kT);
+    for (int jj = tid; jj < cnt; jj += kT) {
+      const unsigned int key = keys[jj];
+      if (p == 0 || ((key ^ prefix) >> (lo + 8)) == 0u) atomicAdd(&wh[wq * 256 + ((key >> lo) & 255u)], 1u);
+    }
+    named_barrier_sync(1, kT);
+    if (tid < 256) {
+      unsigned int h = 0;
+#pragma unroll 4
+      for (int w = 0; w < kFWorkerWarps; ++w) h += wh[w * 256 + tid];
+      hist_s[tid] = h;
+      if (h) atomicAdd(a.sel_hist + ((long long)bh * kSelPasses + p) * 256 + tid, h);
+    }
+    named_barrier_sync(1, kT);
+    if (wq == 0) {
+      // suffix sums of the CTA's histogram: sfx[b] = keys of this CTA, matching the digits so far, with digit >= b
+      unsigned int mine[8], sum = 0;
+#pragma unroll
+      for (int k = 7; k >= 0; --k) { sum += hist_s[8 * lane + k]; mine[k] = sum; }   // within the lane's eight bins
+      unsigned int above = sum;                                                      // inclusive over lanes >= this one
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const unsigned int t = __shfl_down_sync(0xffffffffu, above, off);
+        if (lane + off < 32) above += t;
+      }
+      above -= sum;                                                                  // lanes above this one
+      unsigned int* dst = sfx_mine + p * kSfxStride + 8 * lane;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) dst[k] = mine[k] + above;
+      if (lane == 31) dst[8] = 0u;   // sfx[256]
+    }
+    if (!group_barrier_follow(go)) return false;
+    if (wq == 0) {
+      // lane L owns bins 255-8L .. 248-8L of the group's histogram, so that the lanes walk the bins from the top
+      const unsigned int* gh = a.sel_hist + ((long long)bh * kSelPasses + p) * 256;
+      unsigned int mine[8], sum = 0;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) { mine[k] = __ldcg(gh + 255 - 8 * lane - k); sum += mine[k]; }
+      unsigned int incl = sum;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const unsigned int t = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += t;
+      }
+      unsigned int acc = incl - sum;
+      if (acc < remaining && remaining <= incl) {   // exactly one lane
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          if (acc < remaining && remaining <= acc + mine[k]) {
+            misc[0] = (unsigned int)(255 - 8 * lane - k);
+            misc[1] = remaining - acc;
+          }
+          acc += mine[k];
+        }
+      }
+    }
+    named_barrier_sync(1, kT);
+    const unsigned int d = misc[0];
+    remaining = misc[1];
+    prefix |= d << lo;
+    if (wq == 1) {
+      // keys of the lower ranks above the chosen digit (and, in the last pass, equal to the threshold key)
+      unsigned int g = 0, e = 0;
+      for (int r = lane; r < pl.rank; r += 32) {
+        const unsigned int* sr = a.sel_sfx + (((long long)bh * a.cpg + r) * kSelPasses + p) * kSfxStride;
+        const unsigned int above = __ldcg(sr + d + 1);
+        g += above;
+        if (p == kSelPasses - 1) e += __ldcg(sr + d) - above;
+      }
+      g = __reduce_add_sync(0xffffffffu, g);
+      e = __reduce_add_sync(0xffffffffu, e);
+      if (lane == 0) { misc[2] += g; misc[3] += e; }
+    }
+    named_barrier_sync(1, kT);   // misc[0..1] may be rewritten, misc[2..3] are final after the last pass
+  }
+  const unsigned int T = prefix, need_eq = remaining;
+  // ---- 3. ordered emit: warp wq owns a contiguous run of the CTA's tokens ----
+  {
+    int32_t* dst = a.sel_indices + (long long)bh * keep;
+    unsigned int* warp_a = misc + 8;
+    unsigned int* warp_b = misc + 8 + kFWorkerWarps;
+    const int cw = (((cnt + kFWorkerWarps - 1) / kFWorkerWarps) + 31) & ~31;
+    const int wbeg = min(cnt, wq * cw), wend = min(cnt, wbeg + cw);
+    const unsigned int lt_mask = (1u << lane) - 1u;
+    unsigned int cgt = 0, ceq = 0;
+    for (int base = wbeg; base < wend; base += 32) {
+      const int jj = base + lane;
+      const bool valid = jj < wend;
+      const unsigned int key = valid ? keys[jj] : 0u;
+      cgt += __popc(__ballot_sync(0xffffffffu, valid && key > T));
+      ceq += __popc(__ballot_sync(0xffffffffu, valid && key == T));
+    }
+    if (lane == 0) { warp_a[wq] = cgt; warp_b[wq] = ceq; }
+    named_barrier_sync(1, kT);
+    unsigned int run_gt = misc[2], run_eq = misc[3];
+    for (int w = 0; w < wq; ++w) { run_gt += warp_a[w]; run_eq += warp_b[w]; }
+    for (int base = wbeg; base < wend; base += 32) {
+      const int jj = base + lane;
+      const bool valid = jj < wend;
+      const unsigned int key = valid ? keys[jj] : 0u;
+      const bool gt = valid && key > T, eq = valid && key == T;
+      const unsigned int mgt = __ballot_sync(0xffffffffu, gt), meq = __ballot_sync(0xffffffffu, eq);
+      const unsigned int gt_before = run_gt + __popc(mgt & lt_mask);
+      const unsigned int eq_before = run_eq + __popc(meq & lt_mask);
+      if (gt || (eq && eq_before < need_eq)) {
+        const unsigned int pos = gt_before + min(eq_before, need_eq);
+        if (pos < (unsigned int)keep) dst[pos] = (int32_t)(j_first + jj);
+      }
+      run_gt += __popc(mgt);
+      run_eq += __popc(meq);
+    }
+  }
+  if (!group_barrier_follow(go)) return false;   // all indices of the head are written
+  // ---- 4. gather: an equal share of the head's rows per CTA, eight 16-byte chunks in flight per thread ----
+  {
+    const int b = bh / a.Hkv, h = bh % a.Hkv;
+    const int share = (keep + a.cpg - 1) / a.cpg;
+    const int first = min(keep, pl.rank * share), mine = min(keep, first + share) - first;
+    const int32_t* idx = a.sel_indices + (long long)bh * keep + first;
+    const __nv_bfloat16* Kh = a.K + (long long)b * a.ksb + (long long)h * a.ksh;
+    const __nv_bfloat16* Vh = a.V + (long long)b * a.vsb + (long long)h * a.vsh;
+    constexpr int kRC = kHeadDim * 2 / 16;   // 16-byte chunks per row
+    const int total = mine * 2 * kRC;
+    for (int e0 = tid; e0 < total; e0 += 8 * kT) {
+      long long jj[8];
+      uint4 val[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int e = e0 + k * kT;
+        jj[k] = e < total ? __ldcg(idx + e / (2 * kRC)) : 0;
+      }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int e = e0 + k * kT;
+        const int c = e % (2 * kRC);
+        const bool isV = c >= kRC;
+        const uint4* srcp = reinterpret_cast<const uint4*>(isV ? Vh + jj[k] * a.vsn : Kh + jj[k] * a.ksn) + (isV ? c - kRC : c);
+        if (e < total) val[k] = __ldg(srcp);
+      }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int e = e0 + k * kT;
+        if (e >= total) continue;
+        const int r = e / (2 * kRC), c = e % (2 * kRC);
+        const bool isV = c >= kRC;
+        uint4* outp = reinterpret_cast<uint4*>((isV ? a.V_out : a.K_out) + ((long long)bh * keep + first + r) * kHeadDim) + (isV ? c - kRC : c);
+        *outp = val[k];
+      }
+    }
+  }
+  // the buffers lie where the operand tiles of the next head land, and they covered the block of ones
+  named_barrier_sync(1, kT);
+  if (tid < (int)(kOnesBytes / 4)) reinterpret_cast<uint32_t*>(cx.gen_base + kOffOnes)[tid] = 0x3F803F80u;
+  fence_proxy_async_smem();
+  return true;
+}
+
+
+
 // The two role loops below run through the same sequence of CTA-wide synchronisations: per head a barrier
 // re-initialisation (from the second head on), phase A, the prefetch point, group barrier, phase B, group
 // barrier, phase C, and a closing __syncthreads.
@@ -854,6 +1110,13 @@ __device__ void control_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, 
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    if (a.sel_keep > 0) {   // the worker warps pool, select and gather; this side runs the group barriers
+      bool sel_ok = true;
+      for (int i = 0; i < kSelBarriers && sel_ok; ++i)
+        sel_ok = group_barrier(counter, (++epoch) * (unsigned int)a.cpg, abort_flag, go, a.dev_status, a.wait_limit);
+      if (!sel_ok) break;
+      __syncthreads();      // the selection's buffers are free for the next head
+    }
   }
 }
 
@@ -887,6 +1150,10 @@ __device__ void worker_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, c
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    if (a.sel_keep > 0) {
+      if (!select_worker(cx, a, pl, bh, go)) break;
+      __syncthreads();
+    }
   }
 }
 
@@ -986,6 +1253,19 @@ void fused_plan(const Problem& p, int sm_count, bool reuse_l2, int* groups, int*
   *cpg = sm_count / best_g;
 }
 
+// Whether the score kernel can also pool, select and gather (fixed window): every CTA's share of a head must fit the
+// shared-memory buffers, the window must stay within the staged halo, and the budget must leave something out.
+bool tc_fused_select_supported(const Problem& p, int sm_count, bool reuse_l2, int keep, int W, int gamma) {
+  if (keep < 1 || keep >= p.n_kv) return false;
+  if (W / 2 + (gamma < 0 ? -gamma : gamma) > kSelHalo) return false;
+  int groups, cpg;
+  fused_plan(p, sm_count, reuse_l2, &groups, &cpg);
+  const int tiles = (p.n_kv + kTile - 1) / kTile, per = (tiles + cpg - 1) / cpg;
+  return (long long)per * kTile <= kSelMaxKeys;
+}
+size_t tc_fused_select_sfx_words(int BH, int sm_count) { return (size_t)BH * sm_count * kSelPasses * kSfxStride; }
+size_t tc_fused_select_hist_words(int BH) { return (size_t)BH * kSelPasses * 256; }
+
 bool tc_supported(const Problem& p) {
   if (p.dtype != RESTKV_BF16 || p.d != kHeadDim || p.R != kRows) return false;
   if (p.w != 16 && p.w != 32 && p.w != 64 && p.w != 128) return false;
@@ -1035,7 +1315,7 @@ cudaError_t tc_fused_init() {
 // with the timeout status instead of hanging.  (A cooperative launch would guarantee residency but costs ~25 us.)
 cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
                             const void* V, float ema_decay, int sm_count, bool reuse_l2, bool attention_only,
-                            long long wait_limit, unsigned int* dev_status, cudaStream_t st) {
+                            long long wait_limit, const FusedSelect* sel, unsigned int* dev_status, cudaStream_t st) {
   TcState* ts = (TcState*)state;
   CUtensorMap tmQ, tmK, tmV, tmO, tmAug;
   if (!make_rows_map(ts, &tmQ, Q, p.BH) || !make_rows_map(ts, &tmO, ws.O_m2, p.BH) ||
@@ -1054,6 +1334,15 @@ cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, 
   a.wait_limit = wait_limit;
   cudaError_t e = cudaMemsetAsync(ws.counters, 0, 1024, st);
   if (e != cudaSuccess) return e;
+  if (sel) {
+    a.sel_keep = sel->keep; a.sel_W = sel->W; a.sel_gamma = sel->gamma;
+    a.sel_scores = sel->scores; a.sel_indices = sel->indices;
+    a.sel_hist = ws.sel_hist; a.sel_sfx = ws.sel_sfx;
+    a.K = (const __nv_bfloat16*)K; a.ksb = p.ksb; a.ksh = p.ksh; a.ksn = p.ksn;
+    a.K_out = (__nv_bfloat16*)sel->K_out; a.V_out = (__nv_bfloat16*)sel->V_out;
+    e = cudaMemsetAsync(ws.sel_hist, 0, (size_t)p.BH * kSelPasses * 256 * sizeof(unsigned int), st);
+    if (e != cudaSuccess) return e;
+  }
   const dim3 grid(a.groups * a.cpg), block(kFThreads);
   switch (attention_only ? 32 : p.w) {   // the window length only matters to phase C
     case 16: tc_fused_kernel<16><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a); break;
