@@ -1260,6 +1260,8 @@ bool tc_fused_select_supported(const Problem& p, int sm_count, bool reuse_l2, in
   if (W / 2 + (gamma < 0 ? -gamma : gamma) > kSelHalo) return false;
   int groups, cpg;
   fused_plan(p, sm_count, reuse_l2, &groups, &cpg);
+  // with only a few CTAs per head the separate selection kernel, which puts a cluster of eight on every head, is faster
+  if (cpg < 8) return false;
   const int tiles = (p.n_kv + kTile - 1) / kTile, per = (tiles + cpg - 1) / cpg;
   return (long long)per * kTile <= kSelMaxKeys;
 }

@@ -151,6 +151,51 @@ def test_config2_is_deterministic(handle):
         np.testing.assert_array_equal(x, y)
 
 
+@pytest.mark.parametrize("spec", [("cfg2", 0, 1024, 7, 0), ("cfg2", 32, 1024, 21, 0), ("cfg2", 0, 37, 1, 0), ("cfg2", 0, 1024, 5, -9),
+                                  ("cfg3", 0, 2048, 7, 0), ("cfg3", 0, 16000, 31, 4)])
+def test_selection_inside_the_score_kernel_equals_the_separate_kernel(handle, spec):
+    """restkv_evict on the tensor-core path pools, selects and gathers inside the score kernel by default; with that
+    switched off the separate kernel does: scores, indices and gathered rows must be identical bit for bit."""
+    name, tail, budget, width, shift = spec
+    inp = make_inputs(CONFIGS[name].with_(causal_tail=tail))
+    run = GpuRun(handle, inp, budget=budget)
+    pool = run.pool(width=width, shift=shift)
+    fused = [x.copy() for x in run.evict(pool=pool)]
+    handle.set_fused_select(False)
+    try:
+        separate = run.evict(pool=pool)
+    finally:
+        handle.set_fused_select(True)
+    for x, y in zip(fused, separate):
+        np.testing.assert_array_equal(x, y)
+    ref = oracle_scores(inp, width=width, shift=shift)
+    assert_scores_close(fused[0], ref.scores, TOL["bf16"])
+    assert_selection_valid(fused[1], ref.scores, budget, TOL["bf16"])
+
+
+def test_selection_inside_the_score_kernel_with_ties(handle):
+    """Identical keys (uniform attention) and only two distinct value rows, alternating: the scores of a head fall
+    into two classes of exact ties, so the lower index must win ties exactly as in the separate kernel, also across
+    the boundaries between the head's thread blocks."""
+    case = Case("ties", 1, 4, 1, 128, 5000, 32, 777, 1, 0, 0.9, "bf16", 0, "normal", 3)
+    inp = make_inputs(case)
+    inp.K[...] = inp.K[:, :, :1]
+    va, vb = inp.V[:, :, 0:1].copy(), inp.V[:, :, 1:2].copy()
+    inp.V[:, :, 0::2] = va
+    inp.V[:, :, 1::2] = vb
+    run = GpuRun(handle, inp)
+    fused = [x.copy() for x in run.evict()]
+    handle.set_fused_select(False)
+    try:
+        separate = run.evict()
+    finally:
+        handle.set_fused_select(True)
+    for x, y in zip(fused, separate):
+        np.testing.assert_array_equal(x, y)
+    ref = oracle_scores(inp)
+    assert_selection_valid(fused[1], ref.scores, case.budget, TOL["bf16"])
+
+
 # ------------------------------------------------------------------ config 3 (32 layers, drifting keys)
 @pytest.mark.parametrize("layer", list(range(32)))
 def test_config3_layer(handle, layer):
