@@ -69,10 +69,27 @@ def whole_job_value(tokens_per_rank_step, world, steps, total_ms):
     return world * tokens_per_rank_step * steps / (total_ms / 1e3)
 
 
-# DRAM bytes (read + write) per launch of the score kernel, from the ncu capture summarised in
-# profiles/tc_fused_select_cfg4_ncu_full.md; valid for the kernel as it stood then (set to None when
-# csrc/tc_fused.cu changes in more than comments).
-SCORE_KERNEL_TRAFFIC = {"cfg4": 1008.62e6 + 26.38e6}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from an ncu capture
+# of this workload, together with the digest of the kernel sources the capture was taken on: the figure is reported
+# only while those sources are unchanged, otherwise `traffic` is null.
+KERNEL_TRAFFIC = {"cfg4": {"bytes": 1026520576 + 25419008, "sources_sha256": "2b8344ba553ac6b728c54ef178f6f0f5e42d63d87f25c661464c202f37d9a137"}}
+KERNEL_SOURCES = ("tc_fused.cu", "tc_common.cuh", "sm100_ptx.cuh")
+
+
+def kernel_sources_digest():
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2605_08840_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def measured_traffic(workload):
+    rec = KERNEL_TRAFFIC.get(workload)
+    if not rec or rec["bytes"] is None or rec["sources_sha256"] != kernel_sources_digest():
+        return None
+    return rec["bytes"]
 
 
 class ClockSampler:
@@ -117,7 +134,7 @@ class ClockSampler:
                 self.bits |= int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
             except Exception:
                 break
-            time.sleep(0.002)
+            time.sleep(0.001)
 
     def stop(self):
         if self.nvml is None:
@@ -127,7 +144,7 @@ class ClockSampler:
         sm = sorted(self.sm)
         reasons = sorted(name for name, bit in self.REASONS if self.bits & bit)
         return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": self.max_mhz, "reasons": reasons,
-                "samples": len(sm), "source": "nvml, 2 ms polling during the timed region"}
+                "samples": len(sm), "source": "nvml, 1 ms polling during the timed steps and the per-kernel passes"}
 
     def _smi_once(self):
         fields = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -171,11 +188,11 @@ def cpu_baseline(inp, budget, target_seconds=12.0):
     import oracle
     c = inp.case
     t1 = time_oracle(inp, [0], budget)
-    heads = max(1, min(c.n_kv_heads, int(target_seconds / max(t1, 1e-3))))
-    t = t1 if heads == 1 else time_oracle(inp, list(range(heads)), budget)
+    heads = max(1, min(c.n_kv_heads, int(target_seconds / 3.0 / max(t1, 1e-3))))
+    t = time_oracle(inp, list(range(heads)), budget, repeats=3)     # best of three: the host is shared
     tokens = c.batch * c.n * heads / c.n_kv_heads     # layer-equivalent prefix tokens in the sample
     return {"value": tokens / t, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": "%d of %d KV heads of the workload at full length n=%d (score+select+compact), %.2f s"
+            "sample": "%d of %d KV heads of the workload at full length n=%d (score+select+compact), best of 3: %.2f s"
                       % (heads, c.n_kv_heads, c.n, t)}
 
 
@@ -287,15 +304,11 @@ def main():
     def step():
         handle.evict(shape, Q, K, V, case.ema_decay, pool, case.budget, indices, K_out, V_out, ws)
 
-    # the tensor-core path runs pass 1, the merge and pass 2 in one launch; pooling and the gather run inside the
-    # select kernel
-    kernel_ids = {"score": rk.KERNEL_PASS2, "pool_select_compact": rk.KERNEL_SELECT}
-    if case.batch * case.n_kv_heads * 8 > 148:      # many rows: the gather runs as its own kernel
-        kernel_ids = {"score": rk.KERNEL_PASS2, "pool_select": rk.KERNEL_SELECT, "compact": rk.KERNEL_COMPACT}
     for _ in range(args.warmup):
         flush.zero_()
         step()
     barrier()
+    fused = handle.last_evict_fused_select()
     launches0 = handle.launch_count()
     sampler = ClockSampler(local)
     if rank == 0:
@@ -310,28 +323,45 @@ def main():
         torch.cuda.synchronize()
         step_ms.append(ev0.elapsed_time(ev1))
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
     launches = handle.launch_count() - launches0
 
-    # per-kernel durations in a pass of their own (the event records between the launches would sit inside the
-    # timed region otherwise): CUDA events recorded by the library right around each launch, on the call's stream
-    prof = {}
-    for name, kid in kernel_ids.items():
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(); b.record()
-        prof[name] = (a, b)
-    torch.cuda.synchronize()
-    for name, kid in kernel_ids.items():
-        handle.set_profile_events(kid, *prof[name])
-    kern_ms = {k: [] for k in kernel_ids}
-    for _ in range(max(3, min(args.steps, 20))):
-        flush.zero_()
-        step()
-        torch.cuda.synchronize()
+    # Per-kernel durations in passes of their own (the event records between the launches would sit inside the
+    # timed region otherwise): CUDA events recorded by the library right around each launch, on the call's stream.
+    # On the tensor-core path with a fixed window one persistent launch does everything (pass 1, merge, pass 2,
+    # pooling, selection, gather); a second pass with the selection as its own kernel gives the split.
+    def kernel_pass(kernel_ids, reps):
+        prof = {}
         for name in kernel_ids:
-            kern_ms[name].append(prof[name][0].elapsed_time(prof[name][1]))
-    for kid in kernel_ids.values():
-        handle.set_profile_events(kid, None, None)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); b.record()
+            prof[name] = (a, b)
+        torch.cuda.synchronize()
+        for name, kid in kernel_ids.items():
+            handle.set_profile_events(kid, *prof[name])
+        ms = {k: [] for k in kernel_ids}
+        for _ in range(reps):
+            flush.zero_()
+            step()
+            torch.cuda.synchronize()
+            for name in kernel_ids:
+                ms[name].append(prof[name][0].elapsed_time(prof[name][1]))
+        for kid in kernel_ids.values():
+            handle.set_profile_events(kid, None, None)
+        return {k: float(np.mean(v)) for k, v in ms.items()}
+
+    split_ids = {"score": rk.KERNEL_PASS2, "pool_select_compact": rk.KERNEL_SELECT}
+    if case.batch * case.n_kv_heads * 8 > 148:      # many rows: the gather runs as its own kernel
+        split_ids = {"score": rk.KERNEL_PASS2, "pool_select": rk.KERNEL_SELECT, "compact": rk.KERNEL_COMPACT}
+    reps = max(3, min(args.steps, 20))
+    kmean_split = None
+    if fused:
+        kmean = kernel_pass({"score_pool_select_compact": rk.KERNEL_PASS2}, reps)
+        handle.set_fused_select(False)
+        kmean_split = kernel_pass(split_ids, reps)
+        handle.set_fused_select(True)
+    else:
+        kmean = kernel_pass(split_ids, reps)
+    clocks = sampler.stop() if rank == 0 else None      # sampled through the timed steps and the per-kernel passes
     assert handle.poll_status() == rk.RESTKV_OK
 
     total_ms = max_over_ranks(float(sum(step_ms)), world, "cuda")
@@ -342,7 +372,9 @@ def main():
     # ---- one decode step over the compacted cache and over the full cache (context for the paper's 10.61x) ----
     decode = None
     if rank == 0:
-        qd = torch.randn(case.batch, case.n_q_heads, case.head_dim, device="cuda").to(tdt)
+        from paper_2605_08840_b200.inputs import make_decode_query, round_to_bf16_bits
+        q_np2 = make_decode_query(inp)                 # seeded
+        qd = dev(round_to_bf16_bits(q_np2).view(np.int16) if case.dtype == "bf16" else q_np2)
         dout = torch.empty(case.batch, case.n_q_heads, case.head_dim, dtype=torch.float32, device="cuda")
 
         def time_decode(Kc, Vc, rows):
@@ -380,6 +412,16 @@ def main():
                               indices, K_out, V_out, ws)
         e2e_step()
         barrier()
+        # what came back through the host buffers must be what the device path produced (not timed)
+        step()
+        torch.cuda.synchronize()
+        e2e_ok = bool(torch.equal(h_idx, indices.cpu()) and
+                      torch.equal(h_Ko.view(torch.int16) if case.dtype == "bf16" else h_Ko,
+                                  (K_out.view(torch.int16) if case.dtype == "bf16" else K_out).cpu()) and
+                      torch.equal(h_Vo.view(torch.int16) if case.dtype == "bf16" else h_Vo,
+                                  (V_out.view(torch.int16) if case.dtype == "bf16" else V_out).cpu()))
+        if not e2e_ok:
+            raise SystemExit("bench.py: the host-buffer path returned other results than the device path")
         ms = 0.0
         for _ in range(e2e_steps):
             ev0.record()
@@ -392,7 +434,7 @@ def main():
         h2d = sum(x.numel() * x.element_size() for x in (hQ, hK, hV))
         d2h = sum(x.numel() * x.element_size() for x in (h_idx, h_Ko, h_Vo))
         e2e = {"value": tokens_per_step * e2e_steps / (ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+               "d2h_bytes_per_step": d2h, "steps": e2e_steps, "outputs_equal_device_path": e2e_ok}
 
     if rank != 0:
         if world > 1:
@@ -402,14 +444,17 @@ def main():
     peaks = load_peaks()
     kv_bytes, out_bytes = algorithmic_bytes(case, keep)
     flops = algorithmic_flops(case)
-    kmean = {k: float(np.mean(v)) for k, v in kern_ms.items()}
-    dominant = "score"
-    # algorithmic bytes of the score kernel: K and V once, plus 4 B of score per token and head
-    dom_bytes = kv_bytes + 4 * case.batch * case.n_kv_heads * case.n
+    dominant = "score_pool_select_compact" if fused else "score"
+    # algorithmic bytes of the dominant kernel: K and V once plus 4 B of score per token and head, and, when it also
+    # selects and gathers, the indices and the compacted cache written
+    dom_bytes = kv_bytes + 4 * case.batch * case.n_kv_heads * case.n_kv
+    if fused:
+        dom_bytes += out_bytes + 4 * case.batch * case.n_kv_heads * keep
     achieved = dom_bytes / (kmean[dominant] * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "tc_fused_kernel (score: pass 1 + merge + pass 2)", "achieved": achieved,
-                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                "traffic": SCORE_KERNEL_TRAFFIC.get(args.workload) if args.path == 0 else None,
+    roofline = {"bound": "hbm",
+                "kernel": "tc_fused_kernel (pass 1 + merge + pass 2%s)" % (" + pooling + selection + gather" if fused else ""),
+                "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                "traffic": measured_traffic(args.workload) if args.path == 0 else None,
                 "peak_source": peaks["source"], "algorithmic_bytes_per_launch": dom_bytes,
                 "ms_per_launch": kmean[dominant]}
     t_roof_ms = max((kv_bytes + out_bytes) / (peaks["hbm_gbs"] * 1e9), flops / (peaks["bf16_tflops"] * 1e12)) * 1e3
@@ -422,7 +467,8 @@ def main():
         "dtype": case.dtype, "data": "synthetic",
         "config": workload_config(case, l2="flushed between steps (256 MiB write); inputs 537 MB > 126 MB L2"),
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-        "roofline": roofline, "path_roofline": path_roofline, "kernels_ms": kmean, "decode": decode,
+        "roofline": roofline, "path_roofline": path_roofline, "kernels_ms": kmean,
+        "kernels_ms_selection_as_own_kernel": kmean_split, "decode": decode,
     }
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(inp, case.budget)

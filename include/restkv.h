@@ -239,6 +239,7 @@ restkv_status restkv_set_kernel_path(restkv_handle* h, int path);
  * on).  With 0 the pooling, selection and gather always run as the separate kernel that other paths use; the results
  * are the same.  Meant for timing the two against each other. */
 restkv_status restkv_set_fused_select(restkv_handle* h, int on);
+int restkv_last_evict_fused_select(const restkv_handle* h);   /* 1 if the last restkv_evict ran them inside the score kernel */
 
 /* Bound of every device-side wait of the persistent kernels, in SM clocks (default 2e9, about a second).  A wait
  * that runs out sets the sticky status (RESTKV_ERR_TIMEOUT from restkv_poll_status), the kernel stops issuing

@@ -24,7 +24,7 @@ EXPORTS = [
     "restkv_score", "restkv_select", "restkv_compact", "restkv_evict", "restkv_evict_host", "restkv_decode", "restkv_decode_static",
     "restkv_decode_static_last_cuda_error",
     "restkv_poll_status", "restkv_launch_count", "restkv_last_cuda_error", "restkv_error_string",
-    "restkv_set_kernel_path", "restkv_set_profile_events", "restkv_set_wait_limit", "restkv_set_fused_select",
+    "restkv_set_kernel_path", "restkv_set_profile_events", "restkv_set_wait_limit", "restkv_set_fused_select", "restkv_last_evict_fused_select",
 ]
 KERNEL_NONE, KERNEL_PASS1, KERNEL_COMBINE, KERNEL_PASS2, KERNEL_POOL, KERNEL_SELECT, KERNEL_COMPACT = range(7)
 
@@ -89,6 +89,7 @@ def load_library() -> ctypes.CDLL:
     lib.restkv_set_profile_events.argtypes = [vp, ci, vp, vp]
     lib.restkv_set_wait_limit.argtypes = [vp, ctypes.c_longlong]
     lib.restkv_set_fused_select.argtypes = [vp, ci]
+    lib.restkv_last_evict_fused_select.argtypes = [vp]
     _lib = lib
     return lib
 
@@ -216,6 +217,9 @@ class Handle:
 
     def set_fused_select(self, on: bool):
         self._check(self._lib.restkv_set_fused_select(self._h, int(bool(on))), "restkv_set_fused_select")
+
+    def last_evict_fused_select(self) -> bool:
+        return bool(self._lib.restkv_last_evict_fused_select(self._h))
 
     def set_wait_limit(self, sm_clocks: int):
         self._check(self._lib.restkv_set_wait_limit(self._h, int(sm_clocks)), "restkv_set_wait_limit")

@@ -15,6 +15,7 @@ struct restkv_handle {
   int last_cuda_error;
   int kernel_path;            // 0 auto, 1 SIMT, 2 tensor core required, 3 tensor core in its head-sequential form
   bool fused_select;          // restkv_evict lets the tensor-core score kernel pool, select and gather when it can
+  bool last_evict_fused;      // whether the last restkv_evict did
   long long wait_limit;       // SM clocks a device-side wait may last
   cudaEvent_t prof_start[7], prof_stop[7];   // per restkv_kernel_id, null = not timed
 };
@@ -262,6 +263,7 @@ restkv_status restkv_create(restkv_handle** out) {
   if (tc_init(&h->tc_state) != cudaSuccess || tc_fused_init() != cudaSuccess) h->tc_state = nullptr;
   h->wait_limit = 2000000000ll;
   h->fused_select = true;
+  h->last_evict_fused = false;
   h->launches = 0;
   h->last_cuda_error = 0;
   h->kernel_path = 0;
@@ -371,6 +373,7 @@ restkv_status restkv_evict(restkv_handle* h, const restkv_shape* shape, const vo
   if ((s = run_score(c, p, ws, Q_obs, K, V, ema_decay, pool, nullptr, nullptr, adaptive ? nullptr : &sel, &sel_done)) !=
       RESTKV_OK)
     return s;
+  h->last_evict_fused = sel_done;
   if (sel_done) return RESTKV_OK;
   // Pooling (Eq. 13) runs inside the select kernel, which also writes the pooled scores.  So does the gather
   // (Eq. 14) while the select kernel's clusters fit the GPU in one wave; with more (batch, head) rows than that the
@@ -517,6 +520,8 @@ restkv_status restkv_set_profile_events(restkv_handle* h, int which, void* start
   h->prof_stop[which] = (cudaEvent_t)stop;
   return RESTKV_OK;
 }
+
+int restkv_last_evict_fused_select(const restkv_handle* h) { return h && h->last_evict_fused ? 1 : 0; }
 
 restkv_status restkv_set_fused_select(restkv_handle* h, int on) {
   if (!h) return RESTKV_ERR_INVALID_ARG;
