@@ -114,6 +114,22 @@ restkv_status restkv_score(restkv_handle* h, const restkv_shape* shape, const vo
                            int32_t* pool_used, void* workspace, size_t workspace_bytes, restkv_stream stream);
 
 /*
+ * restkv_score_from_lse -- restkv_score for a caller that already holds the attention statistics of the window
+ * rows.  During prompt prefilling the attention of the last w tokens has been computed anyway (paper, Appendix B,
+ * "prompt prefilling"): its outputs and softmax normalisers are exactly what pass 1 of restkv_score would
+ * recompute (Eq. 3), so with them the indicator (Eq. 7) and its smoothing (Eq. 8-9, Eq. 13) need one read of K and V.
+ *   O_obs    device float [batch, n_q_heads, w, head_dim]: o of every window row over the rows it sees
+ *            (softmax(scale * q K^T) V, before the output projection)
+ *   LSE_obs  device float [batch, n_q_heads, w]: natural-log sum of exp of that row's scaled logits over the same rows
+ *   everything else as for restkv_score; the same kernels, tolerances and error codes apply.
+ * The values must belong to the same Q_obs, K, V and softmax scale; nothing checks that.
+ */
+restkv_status restkv_score_from_lse(restkv_handle* h, const restkv_shape* shape, const void* Q_obs, const void* K,
+                                    const void* V, const float* O_obs, const float* LSE_obs, float ema_decay,
+                                    const restkv_pool_params* pool, float* scores, int32_t* pool_used, void* workspace,
+                                    size_t workspace_bytes, restkv_stream stream);
+
+/*
  * restkv_select -- Eq. 14's argmax_B: per (batch, KV head) the min(budget, n_kv) largest scores,
  * ties to the lower index, indices written in ascending order.
  *   scores   device float [batch, n_kv_heads, n_kv] (+inf allowed, NaN not)

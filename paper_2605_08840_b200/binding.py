@@ -21,7 +21,7 @@ PATH_AUTO, PATH_SIMT, PATH_TENSOR_CORE, PATH_HEAD_SEQUENTIAL = 0, 1, 2, 3
 
 EXPORTS = [
     "restkv_create", "restkv_destroy", "restkv_workspace_bytes", "restkv_workspace_bytes_adaptive",
-    "restkv_score", "restkv_select", "restkv_compact", "restkv_evict", "restkv_evict_host", "restkv_decode", "restkv_decode_static",
+    "restkv_score", "restkv_score_from_lse", "restkv_select", "restkv_compact", "restkv_evict", "restkv_evict_host", "restkv_decode", "restkv_decode_static",
     "restkv_decode_static_last_cuda_error",
     "restkv_poll_status", "restkv_launch_count", "restkv_last_cuda_error", "restkv_error_string",
     "restkv_set_kernel_path", "restkv_set_profile_events", "restkv_set_wait_limit", "restkv_set_fused_select", "restkv_last_evict_fused_select",
@@ -73,6 +73,7 @@ def load_library() -> ctypes.CDLL:
     lib.restkv_workspace_bytes_adaptive.argtypes = [shp, ci]
     lib.restkv_workspace_bytes_adaptive.restype = sz
     lib.restkv_score.argtypes = [vp, shp, vp, vp, vp, cf, pool, vp, vp, vp, sz, vp]
+    lib.restkv_score_from_lse.argtypes = [vp, shp, vp, vp, vp, vp, vp, cf, pool, vp, vp, vp, sz, vp]
     lib.restkv_select.argtypes = [vp, shp, vp, ci, vp, vp, sz, vp]
     lib.restkv_compact.argtypes = [vp, shp, vp, vp, vp, ci, vp, vp, vp]
     lib.restkv_evict.argtypes = [vp, shp, vp, vp, vp, cf, pool, ci, vp, vp, vp, vp, vp, sz, vp]
@@ -173,6 +174,14 @@ class Handle:
                                            float(ema_decay), ctypes.byref(pool), _ptr(scores), _ptr(pool_used),
                                            _ptr(workspace), workspace.numel() * workspace.element_size(),
                                            _stream_ptr(stream)), "restkv_score")
+
+    def score_from_lse(self, shape, Q_obs, K, V, O_obs, LSE_obs, ema_decay, pool, scores, workspace, pool_used=None,
+                       stream=None):
+        self._check(self._lib.restkv_score_from_lse(self._h, ctypes.byref(shape), _ptr(Q_obs), _ptr(K), _ptr(V),
+                                                    _ptr(O_obs), _ptr(LSE_obs), float(ema_decay), ctypes.byref(pool),
+                                                    _ptr(scores), _ptr(pool_used), _ptr(workspace),
+                                                    workspace.numel() * workspace.element_size(),
+                                                    _stream_ptr(stream)), "restkv_score_from_lse")
 
     def select(self, shape, scores, budget, indices, workspace, stream=None):
         self._check(self._lib.restkv_select(self._h, ctypes.byref(shape), _ptr(scores), int(budget), _ptr(indices),

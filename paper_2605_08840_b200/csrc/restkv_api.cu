@@ -191,7 +191,8 @@ struct Call {
 // null the caller pools (the fused path does it inside the select kernel).
 static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, const void* Q, const void* K,
                                const void* V, float ema_decay, const restkv_pool_params* pool, float* scores,
-                               int32_t* pool_used, const FusedSelect* sel = nullptr, bool* sel_done = nullptr) {
+                               int32_t* pool_used, const FusedSelect* sel = nullptr, bool* sel_done = nullptr,
+                               const float* O_given = nullptr, const float* LSE_given = nullptr) {
   const bool adaptive = pool->mode == RESTKV_POOL_ADAPTIVE;
   // the tensor-core pass 2 seeds its EMA chain with 1/alpha, so ema_decay = 1 (alpha = 0) runs on the SIMT kernels
   bool use_tc = tc_supported(p) && c.h->tc_state != nullptr && !adaptive && ema_decay < 1.f;
@@ -205,6 +206,19 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
     if (e == cudaSuccess && adaptive)
       e = cudaMemsetAsync(ws.I_raw, 0, (size_t)p.batch * p.Hq * p.w * p.n * sizeof(float), c.st);
     if (e != cudaSuccess) return c.fail(e);
+  } else if (O_given) {
+    // the window rows' outputs and log-sum-exps come from the caller: pass 1 and the merge are not needed
+    RESTKV_LAUNCH(c, RESTKV_KERNEL_COMBINE, launch_from_lse_prep(p, ws, O_given, LSE_given, use_tc, c.st), 1);
+    if (use_tc) {
+      RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2,
+                    launch_tc_fused(c.h->tc_state, p, ws, Q, K, V, ema_decay, c.h->sm_count, false, false,
+                                    c.h->wait_limit, nullptr, O_given, c.h->dev_status, c.st), 1);
+    } else {
+      Workspace wsl = ws;
+      wsl.O_f32 = const_cast<float*>(O_given);
+      RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2,
+                    launch_simt_pass2(p, wsl, Q, K, V, ema_decay, adaptive ? ws.I_raw : nullptr, c.st), 1);
+    }
   } else if (use_tc) {
     // pass 1, merge and pass 2 in one persistent launch (timed as "pass 2"); path 3 keeps only as many heads in
     // flight as fit in L2 so that pass 2 re-reads K and V from there
@@ -213,7 +227,7 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
                           tc_fused_select_supported(p, c.h->sm_count, reuse_l2, sel->keep, sel->W, sel->gamma);
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2,
                   launch_tc_fused(c.h->tc_state, p, ws, Q, K, V, ema_decay, c.h->sm_count, reuse_l2, false,
-                                  c.h->wait_limit, with_sel ? sel : nullptr, c.h->dev_status, c.st), 1);
+                                  c.h->wait_limit, with_sel ? sel : nullptr, nullptr, c.h->dev_status, c.st), 1);
     if (sel_done) *sel_done = with_sel;
   } else {
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS1, launch_simt_pass1(p, ws, Q, K, V, c.st), 1);
@@ -317,6 +331,27 @@ restkv_status restkv_score(restkv_handle* h, const restkv_shape* shape, const vo
     return s;
   Call c{h, (cudaStream_t)stream};
   return run_score(c, p, ws, Q_obs, K, V, ema_decay, pool, scores, pool_used);
+}
+
+restkv_status restkv_score_from_lse(restkv_handle* h, const restkv_shape* shape, const void* Q_obs, const void* K,
+                                    const void* V, const float* O_obs, const float* LSE_obs, float ema_decay,
+                                    const restkv_pool_params* pool, float* scores, int32_t* pool_used, void* workspace,
+                                    size_t workspace_bytes, restkv_stream stream) {
+  if (!h || !Q_obs || !K || !V || !O_obs || !LSE_obs || !scores) return RESTKV_ERR_INVALID_ARG;
+  if (!aligned16(Q_obs) || !aligned16(K) || !aligned16(V) || !aligned16(O_obs) || !aligned16(scores))
+    return RESTKV_ERR_INVALID_ARG;
+  if (!(ema_decay >= 0.f && ema_decay <= 1.f)) return RESTKV_ERR_INVALID_ARG;
+  Problem p;
+  restkv_status s = make_problem(shape, true, &p);
+  if (s != RESTKV_OK) return s;
+  if ((s = check_pool(pool, p)) != RESTKV_OK) return s;
+  Workspace ws;
+  const bool adaptive = pool->mode == RESTKV_POOL_ADAPTIVE;
+  if ((s = check_ws(p, adaptive ? pool->budget : 0, h->sm_count, adaptive, workspace, workspace_bytes, &ws)) !=
+      RESTKV_OK)
+    return s;
+  Call c{h, (cudaStream_t)stream};
+  return run_score(c, p, ws, Q_obs, K, V, ema_decay, pool, scores, pool_used, nullptr, nullptr, O_obs, LSE_obs);
 }
 
 restkv_status restkv_select(restkv_handle* h, const restkv_shape* shape, const float* scores, int budget,
@@ -463,7 +498,7 @@ restkv_status restkv_decode(restkv_handle* h, const restkv_shape* shape, const v
       RESTKV_LAUNCH(c, RESTKV_KERNEL_NONE, launch_decode_pad(p, q, ws.q_pad, c.st), 1);
       RESTKV_LAUNCH(c, RESTKV_KERNEL_NONE,
                     launch_tc_fused(h->tc_state, pd, ws, ws.q_pad, Kc, Vc, 0.f, h->sm_count, false, true, h->wait_limit,
-                                    nullptr, h->dev_status, c.st), 1);
+                                    nullptr, nullptr, h->dev_status, c.st), 1);
       RESTKV_LAUNCH(c, RESTKV_KERNEL_NONE, launch_decode_extract(p, ws.O_f32, ws.row_M2, out, lse, c.st), 1);
       return RESTKV_OK;
     }

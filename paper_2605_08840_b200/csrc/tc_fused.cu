@@ -35,6 +35,8 @@ struct FusedArgs {
   float scale, ema_decay;
   int groups, cpg;                   // CTA groups and CTAs per group
   int attention_only;                // 1: stop after the merge (phases A and B): plain attention of the 128 rows
+  int from_lse;                      // 1: O and the rows' log-sum-exp are given: phases A and B are skipped, phase C
+                                     //    computes ||v||^2 and finds the tiles with large weights by itself
   float* part_m;                     // [CTA, 128]       running maximum, log2 units (one slot per CTA, reused
   float* part_l;                     // [CTA, 128]        from head to head: a group is past phase B of a head
   float* part_O;                     // [CTA, 128, 128]   before any of its CTAs writes the next head's partial)
@@ -75,6 +77,7 @@ struct FusedBars {
   // phase C
   uint64_t const_full, kv_full[2], kv_empty[2], acc_full[2], acc_empty[2], red_full[4];
   uint64_t drain;   // only after a failed wait: completion of the MMAs issued so far
+  uint64_t vn_full[4];   // from_lse: ||v||^2 of a tile is in shared memory (ring of four tiles)
 };
 
 __device__ __forceinline__ void mbar_inval(uint64_t* bar) {
@@ -99,7 +102,7 @@ __device__ __forceinline__ void wait_issued(uint64_t* bar, uint32_t parity) {
 }
 
 // (Re)initialises every mbarrier of the CTA for one phase.  Called by one thread between two __syncthreads.
-__device__ void init_bars(FusedBars* B, bool first) {
+__device__ void init_bars(FusedBars* B, bool first, bool from_lse) {
   uint64_t* all = reinterpret_cast<uint64_t*>(B);
   constexpr int kCount = sizeof(FusedBars) / sizeof(uint64_t);
   if (!first)
@@ -112,7 +115,7 @@ __device__ void init_bars(FusedBars* B, bool first) {
     mbar_init(&B->p_full[i], 256);
     mbar_init(&B->pv_done[i], 1);
     mbar_init(&B->kv_full[i], 1);
-    mbar_init(&B->kv_empty[i], 1);
+    mbar_init(&B->kv_empty[i], from_lse ? 3 : 1);   // MMA commit (+ the two ||v||^2 warps, which read the V tile)
     mbar_init(&B->acc_full[i], 1);
     mbar_init(&B->acc_empty[i], kFWorkerWarps);
   }
@@ -123,6 +126,7 @@ __device__ void init_bars(FusedBars* B, bool first) {
   mbar_init(&B->const_full, 1);
   mbar_init(&B->drain, 1);
   for (int i = 0; i < 4; ++i) mbar_init(&B->red_full[i], kFWorkerWarps);
+  for (int i = 0; i < 4; ++i) mbar_init(&B->vn_full[i], 2);
   fence_mbar_init();
 }
 
@@ -162,6 +166,7 @@ struct Ctx {
   FusedBars* B;
   int* abort_flag;
   float* sm_stats;         // [6][128] floats: row maxima of the column halves [slot][half], then (m, l) hand-over
+  float* vn_s;             // [4][128] ||v||^2 of the last four tiles of phase C (from_lse only)
   int warp, lane;
 };
 
@@ -599,8 +604,9 @@ __device__ __forceinline__ void load_stage_c(const Ctx& cx, const CUtensorMap* t
 // tensor core (one extra K = 16 step against a block of ones), so with u = exp2(-scale*log2e * S') = 1/A and
 // x = C' + ||v||^2 = ||o - v||^2 the indicator is x * rsqrt(x * (u - 1)^2).
 template <int kW>
-__device__ void phase_c_control(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tmO, const CUtensorMap* tmAug,
-                                const CUtensorMap* tmK, const CUtensorMap* tmV, int bh, int tile0, int T, int pre) {
+__device__ void phase_c_control(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tmQ, const CUtensorMap* tmO,
+                                const CUtensorMap* tmAug, const CUtensorMap* tmK, const CUtensorMap* tmV, int bh,
+                                int tile0, int T, int pre) {
   constexpr int kG = kRows / kW;
   FusedBars* B = cx.B;
   int* abort_flag = cx.abort_flag;
@@ -613,7 +619,11 @@ __device__ void phase_c_control(const Ctx& cx, const FusedArgs& a, const CUtenso
   if (warp == 0) {
     if (lane == 0 && T > 0) {
       fence_proxy_async_all();   // O' and the constant strip were written with ordinary stores by other CTAs
-      mbar_arrive_expect_tx(&B->const_full, kTileBytes + kAugBytes);
+      mbar_arrive_expect_tx(&B->const_full, kTileBytes + kAugBytes + (a.from_lse ? kTileBytes : 0u));
+      if (a.from_lse) {   // no phase A has brought Q in
+        tma_load_3d(cx.gen_base + kOffQ, tmQ, &B->const_full, 0, 0, bh);
+        tma_load_3d(cx.gen_base + kOffQ + kBoxBytes, tmQ, &B->const_full, 64, 0, bh);
+      }
       tma_load_3d(cx.gen_base + kOffO, tmO, &B->const_full, 0, 0, bh);
       tma_load_3d(cx.gen_base + kOffO + kBoxBytes, tmO, &B->const_full, 64, 0, bh);
       tma_load_3d(cx.gen_base + kOffAug, tmAug, &B->const_full, 0, 0, bh);
@@ -652,6 +662,42 @@ __device__ void phase_c_control(const Ctx& cx, const FusedArgs& a, const CUtenso
       if (*(volatile int*)abort_flag) {
         umma_commit(&B->drain);
         wait_issued(&B->drain, 0);
+      }
+    }
+  } else if (a.from_lse) {
+    // ---- ||v||^2 of the tile's tokens from the V tile in shared memory (phase A, which computes it otherwise, does
+    //      not run): warp 2 takes tokens 0-63, warp 3 tokens 64-127, a lane two rows; ring of four tiles ----
+    bool ok = true;
+    for (int it = 0; it < T && ok; ++it) {
+      const int s = it & 1;
+      ok = mbar_wait(&B->kv_full[s], (it >> 1) & 1, abort_flag, dev_status, kDevTimeout, a.wait_limit);
+      if (!ok) break;
+      const uint8_t* vt = cx.gen_base + k_slot_off(2 * s) + kTileBytes;
+#pragma unroll
+      for (int rr = 0; rr < 2; ++rr) {
+        const int row = (warp - 2) * 64 + rr * 32 + lane;
+        f32x2 acc[4] = {f2_make(0.f, 0.f), f2_make(0.f, 0.f), f2_make(0.f, 0.f), f2_make(0.f, 0.f)};
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const uint8_t* rowp = vt + half * kBoxBytes + (row >> 3) * 1024 + (row & 7) * 128;
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            const uint4 u = *reinterpret_cast<const uint4*>(rowp + ((c ^ (row & 7)) << 4));
+            const unsigned int wv[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const f32x2 e = f2_make(__uint_as_float(wv[q] << 16), __uint_as_float(wv[q] & 0xFFFF0000u));
+              acc[q] = f2_fma(e, e, acc[q]);
+            }
+          }
+        }
+        const f32x2 t2 = f2_add(f2_add(acc[0], acc[1]), f2_add(acc[2], acc[3]));
+        cx.vn_s[(it & 3) * kTile + row] = f2_lo(t2) + f2_hi(t2);
+      }
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(&B->vn_full[it & 3]);
+        mbar_arrive(&B->kv_empty[s]);
       }
     }
   }
@@ -704,7 +750,10 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
     tm_next[k] = -INFINITY;
   }
   float vn_next = 0.f;
-  if (T > 0) {
+  // from_lse: no phase A has left ||v||^2 and the tiles' row maxima behind; ||v||^2 comes from the control warps
+  // through shared memory and a warp finds out from the logits themselves whether its part of a tile is heavy
+  const bool from_lse = a.from_lse != 0;
+  if (T > 0 && !from_lse) {
     const int j = (tile0 + T - 1) * kTile + t;
     vn_next = (j < n) ? vn_head[j] : 1.f;
 #pragma unroll
@@ -714,10 +763,15 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
   for (int it = 0; it < T; ++it) {
     const int s = it & 1;
     const uint32_t par = (uint32_t)(it >> 1) & 1u;
-    const float vn = vn_next;
-    const bool tile_heavy = __any_sync(0xffffffffu, tm_next[0] > m2r[0] || tm_next[1] > m2r[1] ||
-                                                        tm_next[2] > m2r[2] || tm_next[3] > m2r[3]);
-    if (it + 1 < T) {   // next tile's ||v||^2 and row maxima, well ahead of their use
+    float vn = vn_next;
+    bool tile_heavy = __any_sync(0xffffffffu, tm_next[0] > m2r[0] || tm_next[1] > m2r[1] ||
+                                                  tm_next[2] > m2r[2] || tm_next[3] > m2r[3]);
+    if (from_lse) {
+      ok = ok && mbar_wait(&B->vn_full[it & 3], (uint32_t)(it >> 2) & 1u, abort_flag, dev_status, kDevTimeout, a.wait_limit);
+      const int jv = (tile0 + T - 1 - it) * kTile + t;
+      vn = (ok && jv < n) ? cx.vn_s[(it & 3) * kTile + t] : 1.f;
+    }
+    if (it + 1 < T && !from_lse) {   // next tile's ||v||^2 and row maxima, well ahead of their use
       const int jn = (tile0 + T - 2 - it) * kTile + t;
       vn_next = (jn < n) ? vn_head[jn] : 1.f;
 #pragma unroll
@@ -743,13 +797,24 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
       const float vnb = vn * 1.0000152587890625f;
       const f32x2 vn2 = f2_make(vnb, vnb);
       f32x2 h2 = f2_make(0.f, 0.f);
+      float sv0[16], cv0[16], sv1[16], cv1[16];
       if (!tile_heavy) {
-        float sv0[16], cv0[16], sv1[16], cv1[16];
         tmem_ld16(tS, sv0);
         tmem_ld16(tC, cv0);
         tmem_wait_ld();
         tmem_ld16(tS + 16, sv1);   // the second half of the columns travels while the first is worked on
         tmem_ld16(tC + 16, cv1);
+        if (from_lse) {
+          // does any of this warp's entries carry a weight above kHeavyA (S' above heavy_thr)?  If so the warp takes
+          // the slow path below, which reads the accumulators again: they are released only after this vote
+          tmem_wait_ld();
+          float mx = fmaxf(sv0[0], sv1[0]);
+#pragma unroll
+          for (int u = 1; u < 16; ++u) mx = fmaxf(mx, fmaxf(sv0[u], sv1[u]));
+          tile_heavy = __any_sync(0xffffffffu, mx > heavy_thr && j < n);
+        }
+      }
+      if (!tile_heavy) {
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
           const float* sv = c == 0 ? sv0 : sv1;
@@ -1085,8 +1150,16 @@ __device__ void control_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, 
   unsigned int epoch = 0;
   for (int bh = pl.group; bh < a.BH; bh += a.groups) {
     if (bh != pl.group) {   // fresh barriers for every head: nothing is in flight between two __syncthreads
-      if (threadIdx.x == 0) init_bars(bars, false);
+      if (threadIdx.x == 0) init_bars(bars, false, a.from_lse != 0);
       __syncthreads();
+    }
+    if (a.from_lse) {
+      // O and the rows' normalisers are given: phase C only, and no CTA waits for another
+      phase_c_control<kW>(cx, a, tmQ, tmO, tmAug, tmK, tmV, bh, pl.tile0, pl.T2, 0);
+      tc_fence_before();
+      __syncthreads();
+      tc_fence_after();
+      continue;
     }
     phase_a_control(cx, a, tmQ, tmK, tmV, bh, pl.rank, pl.tile0, pl.T1);
     // Phase A no longer needs the tile ring: request phase C's first two K/V stages now, so that they arrive
@@ -1106,7 +1179,7 @@ __device__ void control_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, 
       break;
     }
     tc_fence_after();
-    phase_c_control<kW>(cx, a, tmO, tmAug, tmK, tmV, bh, pl.tile0, pl.T2, pre);
+    phase_c_control<kW>(cx, a, tmQ, tmO, tmAug, tmK, tmV, bh, pl.tile0, pl.T2, pre);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -1127,6 +1200,13 @@ __device__ void worker_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, c
                             const CUtensorMap* tmAug, int* go, float (*red)[4][kTile]) {
   for (int bh = pl.group; bh < a.BH; bh += a.groups) {
     if (bh != pl.group) __syncthreads();
+    if (a.from_lse) {
+      phase_c_worker<kW>(cx, a, tmO, tmAug, tmK, tmV, bh, pl.tile0, pl.T2, 0, red);
+      tc_fence_before();
+      __syncthreads();
+      tc_fence_after();
+      continue;
+    }
     phase_a_worker(cx, a, tmQ, tmK, tmV, bh, pl.rank, pl.tile0, pl.T1);
     __syncthreads();
     if (!group_barrier_follow(go)) break;
@@ -1168,6 +1248,7 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag, go_flag;
   __shared__ float sm_stats[6 * kRows];
+  __shared__ float vn_ring[4 * kTile];
   __shared__ float red[4][4][kTile];   // [tile & 3][warpgroup][token]: each warpgroup's share of the score
 
   const int group = blockIdx.x / a.cpg, rank = blockIdx.x % a.cpg;
@@ -1179,12 +1260,13 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   cx.B = &bars;
   cx.abort_flag = &abort_flag;
   cx.sm_stats = sm_stats;
+  cx.vn_s = vn_ring;
   cx.warp = threadIdx.x >> 5;
   cx.lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
-    init_bars(&bars, true);
+    init_bars(&bars, true, a.from_lse != 0);
     prefetch_tensormap(&tmQ);
     prefetch_tensormap(&tmK);
     prefetch_tensormap(&tmV);
@@ -1230,6 +1312,47 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// The window rows' outputs O and log-sum-exps given by the caller (the prefill attention has them): what phase B
+// would have written for phase C.  One warp per query row, lane = four output dims.
+__global__ void from_lse_prep_kernel(int rows, float scale, const float* __restrict__ O, const float* __restrict__ LSE,
+                                     __nv_bfloat16* __restrict__ O_m2, __nv_bfloat16* __restrict__ aug,
+                                     float* __restrict__ row_M2) {
+  const int ri = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (ri >= rows) return;
+  const float4 o = *reinterpret_cast<const float4*>(O + (long long)ri * kHeadDim + lane * 4);
+  const float f0 = __bfloat162float(__float2bfloat16_rn(o.x)), f1 = __bfloat162float(__float2bfloat16_rn(o.y));
+  const float f2 = __bfloat162float(__float2bfloat16_rn(o.z)), f3 = __bfloat162float(__float2bfloat16_rn(o.w));
+  __nv_bfloat16* om = O_m2 + (long long)ri * kHeadDim + lane * 4;   // -2 x is exact for a bf16 x
+  om[0] = __float2bfloat16_rn(-2.f * f0);
+  om[1] = __float2bfloat16_rn(-2.f * f1);
+  om[2] = __float2bfloat16_rn(-2.f * f2);
+  om[3] = __float2bfloat16_rn(-2.f * f3);
+  float on = (f0 * f0 + f1 * f1) + (f2 * f2 + f3 * f3);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) on += __shfl_xor_sync(0xffffffffu, on, off);
+  __nv_bfloat16* arow = aug + (long long)ri * 64;
+  arow[2 * lane] = __float2bfloat16_rn(0.f);
+  arow[2 * lane + 1] = __float2bfloat16_rn(0.f);
+  __syncwarp();
+  if (lane == 0) {
+    const float c2 = scale * kLog2e;
+    const float M2 = LSE[ri] * kLog2e;     // A = exp2(s * c2 - M2)
+    row_M2[ri] = M2;
+    split3(-M2 / c2, arow);
+    split3(on, arow + 16);
+  }
+}
+
+// SIMT kernels: A = exp(s * scale - fin_m) / fin_l with fin_m = LSE and fin_l = 1.
+__global__ void from_lse_prep_simt_kernel(int rows, const float* __restrict__ LSE, float* __restrict__ fin_m,
+                                          float* __restrict__ fin_l) {
+  const int ri = blockIdx.x * blockDim.x + threadIdx.x;
+  if (ri >= rows) return;
+  fin_m[ri] = LSE[ri];
+  fin_l[ri] = 1.f;
+}
+
 }  // namespace
 
 // Number of CTA groups = heads in flight.  With `reuse_l2` only as many as fit a 72 MB share of L2 (phase C then
@@ -1267,6 +1390,16 @@ bool tc_fused_select_supported(const Problem& p, int sm_count, bool reuse_l2, in
 }
 size_t tc_fused_select_sfx_words(int BH, int sm_count) { return (size_t)BH * sm_count * kSelPasses * kSfxStride; }
 size_t tc_fused_select_hist_words(int BH) { return (size_t)BH * kSelPasses * 256; }
+
+cudaError_t launch_from_lse_prep(const Problem& p, const Workspace& ws, const float* O, const float* LSE,
+                                 bool tensor_core, cudaStream_t st) {
+  const int rows = p.BH * p.R;
+  if (tensor_core)
+    from_lse_prep_kernel<<<(rows + 7) / 8, 256, 0, st>>>(rows, p.scale, O, LSE, ws.O_m2, ws.aug, ws.row_M2);
+  else
+    from_lse_prep_simt_kernel<<<(rows + 255) / 256, 256, 0, st>>>(rows, LSE, ws.fin_m, ws.fin_l);
+  return cudaGetLastError();
+}
 
 bool tc_supported(const Problem& p) {
   if (p.dtype != RESTKV_BF16 || p.d != kHeadDim || p.R != kRows) return false;
@@ -1317,7 +1450,8 @@ cudaError_t tc_fused_init() {
 // with the timeout status instead of hanging.  (A cooperative launch would guarantee residency but costs ~25 us.)
 cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
                             const void* V, float ema_decay, int sm_count, bool reuse_l2, bool attention_only,
-                            long long wait_limit, const FusedSelect* sel, unsigned int* dev_status, cudaStream_t st) {
+                            long long wait_limit, const FusedSelect* sel, const float* O_given, unsigned int* dev_status,
+                            cudaStream_t st) {
   TcState* ts = (TcState*)state;
   CUtensorMap tmQ, tmK, tmV, tmO, tmAug;
   if (!make_rows_map(ts, &tmQ, Q, p.BH) || !make_rows_map(ts, &tmO, ws.O_m2, p.BH) ||
@@ -1328,12 +1462,14 @@ cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, 
   a.Hkv = p.Hkv; a.BH = p.BH; a.n = p.n; a.n_kv = p.n_kv; a.w = p.w;
   a.scale = p.scale; a.ema_decay = ema_decay;
   a.attention_only = attention_only ? 1 : 0;
+  a.from_lse = O_given ? 1 : 0;
   fused_plan(p, sm_count, reuse_l2, &a.groups, &a.cpg);
   a.part_m = ws.part_m; a.part_l = ws.part_l; a.part_O = ws.part_O;
   a.O_f32 = ws.O_f32; a.O_m2 = ws.O_m2; a.aug = ws.aug; a.vnorm = ws.vnorm; a.I_hat = ws.I_hat;
   a.V = (const __nv_bfloat16*)V; a.vsb = p.vsb; a.vsh = p.vsh; a.vsn = p.vsn;
   a.counters = ws.counters; a.tile_max = ws.tile_max; a.row_M2 = ws.row_M2; a.dev_status = dev_status;
   a.wait_limit = wait_limit;
+  if (O_given) a.O_f32 = const_cast<float*>(O_given);   // read only in this mode
   cudaError_t e = cudaMemsetAsync(ws.counters, 0, 1024, st);
   if (e != cudaSuccess) return e;
   if (sel) {

@@ -474,6 +474,60 @@ def test_decode_over_compacted_cache_of_config2(handle):
     assert_decode_close(out.cpu().numpy(), ref, q, Kc, Vc, "bf16")
 
 
+# ------------------------------------------------------------------ scores from given window outputs and normalisers
+def _window_stats(inp, with_A_check=True):
+    """(O float32 [b,Hq,w,d], LSE float32 [b,Hq,w]) of the window rows: O is the oracle's own; the log-sum-exp of the
+    scaled logits over the visible rows comes from SciPy on the same inputs and is tied to the oracle's softmax
+    weights (A = exp(s - LSE)) before it is used."""
+    from scipy.special import logsumexp
+    c = inp.case
+    ref = oracle_scores(inp, want_O=True, want_A=with_A_check)
+    G, w, n, n_kv = c.group, c.w, c.n, c.n_kv
+    scale = 1.0 / np.sqrt(c.head_dim)
+    lse = np.empty((c.batch, c.n_q_heads, w), np.float64)
+    for b in range(c.batch):
+        for h in range(c.n_kv_heads):
+            q = inp.Q[b, h * G:(h + 1) * G].astype(np.float64).reshape(G * w, -1)
+            s = scale * (q @ inp.K[b, h].astype(np.float64).T)                      # [G*w, n_kv]
+            if c.causal_tail:
+                i = np.tile(np.arange(w), G)[:, None]
+                s[:, n:] = np.where(np.arange(n_kv - n)[None, :] <= i, s[:, n:], -np.inf)
+            l = logsumexp(s, axis=-1)
+            lse[b, h * G:(h + 1) * G] = l.reshape(G, w)
+            if with_A_check:
+                A = ref.A[b, h * G:(h + 1) * G].reshape(G * w, n_kv)
+                np.testing.assert_allclose(np.exp(s[:, :64] - l[:, None]), A[:, :64], rtol=1e-9, atol=1e-300)
+    return ref, ref.O.astype(np.float32), lse.astype(np.float32)
+
+
+@pytest.mark.parametrize("spec", [("cfg1b", "f32", 0), ("cfg1b", "bf16", 32), ("cfg2", "bf16", 0), ("cfg2", "bf16", 32)])
+def test_score_from_lse_matches_oracle(handle, spec):
+    """restkv_score_from_lse: the window rows' outputs and log-sum-exps are given (as after prompt prefilling), the
+    scores must be the oracle's."""
+    import torch
+    name, dtype, tail = spec
+    inp = make_inputs(CONFIGS[name].with_(dtype=dtype, causal_tail=tail))
+    ref, O, lse = _window_stats(inp)
+    run = GpuRun(handle, inp)
+    handle.score_from_lse(run.shape, run.Q, run.K, run.V, torch.from_numpy(O).cuda(), torch.from_numpy(lse).cuda(),
+                          inp.case.ema_decay, run.pool(), run.scores, run.ws)
+    torch.cuda.synchronize()
+    assert handle.poll_status() == rk.RESTKV_OK
+    assert_scores_close(run.scores.cpu().numpy(), ref.scores, TOL[dtype])
+
+
+def test_score_from_lse_at_full_size(handle):
+    import torch
+    inp = make_inputs(CONFIGS["cfg4"])
+    ref, O, lse = _window_stats(inp, with_A_check=False)
+    run = GpuRun(handle, inp)
+    handle.score_from_lse(run.shape, run.Q, run.K, run.V, torch.from_numpy(O).cuda(), torch.from_numpy(lse).cuda(),
+                          inp.case.ema_decay, run.pool(), run.scores, run.ws)
+    torch.cuda.synchronize()
+    assert handle.poll_status() == rk.RESTKV_OK
+    assert_scores_close(run.scores.cpu().numpy(), ref.scores, TOL["bf16"])
+
+
 # ------------------------------------------------------------------ a device-side wait that runs out
 def test_wait_limit_runs_out_and_the_handle_recovers(handle):
     """With a wait limit of one SM clock the first CTA to reach a group barrier of the persistent score kernel gives
