@@ -603,7 +603,7 @@ __device__ __forceinline__ void load_stage_c(const Ctx& cx, const CUtensorMap* t
 // [32c, 32c + 32)).  Q is still in shared memory from phase A.  The per-query-row constants ride through the
 // tensor core (one extra K = 16 step against a block of ones), so with u = exp2(-scale*log2e * S') = 1/A and
 // x = C' + ||v||^2 = ||o - v||^2 the indicator is x * rsqrt(x * (u - 1)^2).
-template <int kW>
+template <int kW, bool kLse>
 __device__ void phase_c_control(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tmQ, const CUtensorMap* tmO,
                                 const CUtensorMap* tmAug, const CUtensorMap* tmK, const CUtensorMap* tmV, int bh,
                                 int tile0, int T, int pre) {
@@ -619,8 +619,8 @@ __device__ void phase_c_control(const Ctx& cx, const FusedArgs& a, const CUtenso
   if (warp == 0) {
     if (lane == 0 && T > 0) {
       fence_proxy_async_all();   // O' and the constant strip were written with ordinary stores by other CTAs
-      mbar_arrive_expect_tx(&B->const_full, kTileBytes + kAugBytes + (a.from_lse ? kTileBytes : 0u));
-      if (a.from_lse) {   // no phase A has brought Q in
+      mbar_arrive_expect_tx(&B->const_full, kTileBytes + kAugBytes + (kLse ? kTileBytes : 0u));
+      if (kLse) {   // no phase A has brought Q in
         tma_load_3d(cx.gen_base + kOffQ, tmQ, &B->const_full, 0, 0, bh);
         tma_load_3d(cx.gen_base + kOffQ + kBoxBytes, tmQ, &B->const_full, 64, 0, bh);
       }
@@ -664,7 +664,7 @@ __device__ void phase_c_control(const Ctx& cx, const FusedArgs& a, const CUtenso
         wait_issued(&B->drain, 0);
       }
     }
-  } else if (a.from_lse) {
+  } else if (kLse) {
     // ---- ||v||^2 of the tile's tokens from the V tile in shared memory (phase A, which computes it otherwise, does
     //      not run): warp 2 takes tokens 0-63, warp 3 tokens 64-127, a lane two rows; ring of four tiles ----
     bool ok = true;
@@ -703,7 +703,7 @@ __device__ void phase_c_control(const Ctx& cx, const FusedArgs& a, const CUtenso
   }
 }
 
-template <int kW>
+template <int kW, bool kLse>
 __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tmO, const CUtensorMap* tmAug,
                         const CUtensorMap* tmK, const CUtensorMap* tmV, int bh, int tile0, int T, int pre,
                         float (*red)[4][kTile]) {
@@ -752,7 +752,7 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
   float vn_next = 0.f;
   // from_lse: no phase A has left ||v||^2 and the tiles' row maxima behind; ||v||^2 comes from the control warps
   // through shared memory and a warp finds out from the logits themselves whether its part of a tile is heavy
-  const bool from_lse = a.from_lse != 0;
+  constexpr bool from_lse = kLse;
   if (T > 0 && !from_lse) {
     const int j = (tile0 + T - 1) * kTile + t;
     vn_next = (j < n) ? vn_head[j] : 1.f;
@@ -1142,7 +1142,7 @@ __device__ bool select_worker(const Ctx& cx, const FusedArgs& a, const Plan& pl,
 // barrier, phase C, and a closing __syncthreads.
 
 // Warps 0-3: TMA producer, MMA issuer, the two ||v||^2 warps; thread 0 also runs the group barriers.
-template <int kW>
+template <int kW, bool kLse>
 __device__ void control_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, const CUtensorMap* tmQ,
                              const CUtensorMap* tmK, const CUtensorMap* tmV, const CUtensorMap* tmO,
                              const CUtensorMap* tmAug, FusedBars* bars, int* abort_flag, int* go) {
@@ -1150,12 +1150,12 @@ __device__ void control_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, 
   unsigned int epoch = 0;
   for (int bh = pl.group; bh < a.BH; bh += a.groups) {
     if (bh != pl.group) {   // fresh barriers for every head: nothing is in flight between two __syncthreads
-      if (threadIdx.x == 0) init_bars(bars, false, a.from_lse != 0);
+      if (threadIdx.x == 0) init_bars(bars, false, kLse);
       __syncthreads();
     }
-    if (a.from_lse) {
+    if (kLse) {
       // O and the rows' normalisers are given: phase C only, and no CTA waits for another
-      phase_c_control<kW>(cx, a, tmQ, tmO, tmAug, tmK, tmV, bh, pl.tile0, pl.T2, 0);
+      phase_c_control<kW, kLse>(cx, a, tmQ, tmO, tmAug, tmK, tmV, bh, pl.tile0, pl.T2, 0);
       tc_fence_before();
       __syncthreads();
       tc_fence_after();
@@ -1179,7 +1179,7 @@ __device__ void control_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, 
       break;
     }
     tc_fence_after();
-    phase_c_control<kW>(cx, a, tmQ, tmO, tmAug, tmK, tmV, bh, pl.tile0, pl.T2, pre);
+    phase_c_control<kW, kLse>(cx, a, tmQ, tmO, tmAug, tmK, tmV, bh, pl.tile0, pl.T2, pre);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -1194,14 +1194,14 @@ __device__ void control_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, 
 }
 
 // Warps 4-19: softmax in phase A, the merge of the partials in phase B, the indicator epilogue in phase C.
-template <int kW>
+template <int kW, bool kLse>
 __device__ void worker_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, const CUtensorMap* tmQ,
                             const CUtensorMap* tmK, const CUtensorMap* tmV, const CUtensorMap* tmO,
                             const CUtensorMap* tmAug, int* go, float (*red)[4][kTile]) {
   for (int bh = pl.group; bh < a.BH; bh += a.groups) {
     if (bh != pl.group) __syncthreads();
-    if (a.from_lse) {
-      phase_c_worker<kW>(cx, a, tmO, tmAug, tmK, tmV, bh, pl.tile0, pl.T2, 0, red);
+    if (kLse) {
+      phase_c_worker<kW, kLse>(cx, a, tmO, tmAug, tmK, tmV, bh, pl.tile0, pl.T2, 0, red);
       tc_fence_before();
       __syncthreads();
       tc_fence_after();
@@ -1226,7 +1226,7 @@ __device__ void worker_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, c
     }
     if (!group_barrier_follow(go)) break;
     tc_fence_after();
-    phase_c_worker<kW>(cx, a, tmO, tmAug, tmK, tmV, bh, pl.tile0, pl.T2, 0, red);
+    phase_c_worker<kW, kLse>(cx, a, tmO, tmAug, tmK, tmV, bh, pl.tile0, pl.T2, 0, red);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -1238,7 +1238,7 @@ __device__ void worker_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, c
 }
 
 // ------------------------------------------------------------------------------------------------
-template <int kW>
+template <int kW, bool kLse>
 __global__ void __launch_bounds__(kFThreads, 1)
 tc_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -1266,7 +1266,7 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
-    init_bars(&bars, true, a.from_lse != 0);
+    init_bars(&bars, true, kLse);
     prefetch_tensormap(&tmQ);
     prefetch_tensormap(&tmK);
     prefetch_tensormap(&tmV);
@@ -1298,10 +1298,10 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   // compiled for more registers than the launch gives every thread.
   if (cx.warp < kFFirstWorker) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kFRegsControl));
-    control_main<kW>(cx, a, pl, &tmQ, &tmK, &tmV, &tmO, &tmAug, &bars, &abort_flag, &go_flag);
+    control_main<kW, kLse>(cx, a, pl, &tmQ, &tmK, &tmV, &tmO, &tmAug, &bars, &abort_flag, &go_flag);
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kFRegsWorker));
-    worker_main<kW>(cx, a, pl, &tmQ, &tmK, &tmV, &tmO, &tmAug, &go_flag, red);
+    worker_main<kW, kLse>(cx, a, pl, &tmQ, &tmK, &tmV, &tmO, &tmAug, &go_flag, red);
   }
 
   tc_fence_before();
@@ -1430,17 +1430,19 @@ static cudaError_t check_launch_regs(K kernel) {
 }
 
 cudaError_t tc_fused_init() {
-  {
-    cudaError_t c = check_launch_regs(tc_fused_kernel<16>);
-    if (c == cudaSuccess) c = check_launch_regs(tc_fused_kernel<32>);
-    if (c == cudaSuccess) c = check_launch_regs(tc_fused_kernel<64>);
-    if (c == cudaSuccess) c = check_launch_regs(tc_fused_kernel<128>);
-    if (c != cudaSuccess) return c;
-  }
-  cudaError_t e = cudaFuncSetAttribute(tc_fused_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmem);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fused_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmem);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fused_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmem);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fused_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmem);
+  cudaError_t e = cudaSuccess;
+  auto prepare = [&](auto kernel) {
+    if (e == cudaSuccess) e = check_launch_regs(kernel);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmem);
+  };
+  prepare(tc_fused_kernel<16, false>);
+  prepare(tc_fused_kernel<32, false>);
+  prepare(tc_fused_kernel<64, false>);
+  prepare(tc_fused_kernel<128, false>);
+  prepare(tc_fused_kernel<16, true>);
+  prepare(tc_fused_kernel<32, true>);
+  prepare(tc_fused_kernel<64, true>);
+  prepare(tc_fused_kernel<128, true>);
   return e;
 }
 
@@ -1483,10 +1485,22 @@ cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, 
   }
   const dim3 grid(a.groups * a.cpg), block(kFThreads);
   switch (attention_only ? 32 : p.w) {   // the window length only matters to phase C
-    case 16: tc_fused_kernel<16><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a); break;
-    case 32: tc_fused_kernel<32><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a); break;
-    case 64: tc_fused_kernel<64><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a); break;
-    case 128: tc_fused_kernel<128><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a); break;
+    case 16:
+      if (a.from_lse) tc_fused_kernel<16, true><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a);
+      else tc_fused_kernel<16, false><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a);
+      break;
+    case 32:
+      if (a.from_lse) tc_fused_kernel<32, true><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a);
+      else tc_fused_kernel<32, false><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a);
+      break;
+    case 64:
+      if (a.from_lse) tc_fused_kernel<64, true><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a);
+      else tc_fused_kernel<64, false><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a);
+      break;
+    case 128:
+      if (a.from_lse) tc_fused_kernel<128, true><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a);
+      else tc_fused_kernel<128, false><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a);
+      break;
     default: return cudaErrorInvalidValue;
   }
   return cudaGetLastError();
