@@ -63,7 +63,7 @@ size_t plan_workspace(const Problem& p, int budget, int sm_count, bool adaptive,
   w.tile_max = (float*)take(BH * (size_t)((p.n_kv + 127) / 128) * 128 * sizeof(float));
   w.row_M2 = (float*)take(BH * 128 * sizeof(float));
   w.sel_hist = (unsigned int*)take(tc_fused_select_hist_words(p.BH) * sizeof(unsigned int));
-  w.sel_sfx = (unsigned int*)take(tc_fused_select_sfx_words(p.BH, sm_count) * sizeof(unsigned int));
+  w.sel_sfx = (unsigned int*)take(tc_fused_select_sfx_words(sm_count) * sizeof(unsigned int));
   w.q_pad = (__nv_bfloat16*)take(BH * 128 * 128 * sizeof(__nv_bfloat16));
   w.vnorm = (float*)take(BH * (size_t)p.n_kv * sizeof(float));
   w.fin_m = (float*)take(BH * R * sizeof(float));

@@ -37,7 +37,7 @@ struct Workspace {
   float* tile_max;        // [BH, tiles, 128] per-tile row maxima of the persistent score kernel
   float* row_M2;          // [BH, 128] log2 normaliser of each query row
   unsigned int* sel_hist; // [BH, 4, 256] digit histograms of the selection inside the score kernel
-  unsigned int* sel_sfx;  // [BH, SMs, 4, 260] per-CTA suffix sums of those histograms
+  unsigned int* sel_sfx;  // [SMs, 4, 260] per-CTA suffix sums of those histograms
   __nv_bfloat16* q_pad;   // [BH, 128, 128] decode queries padded to the kernel's 128 rows
   float* fin_m;           // [BH, R]    row max of the scaled logits (natural units)
   float* fin_l;           // [BH, R]    sum of exp(s - m)
@@ -100,7 +100,7 @@ cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, 
 cudaError_t launch_from_lse_prep(const Problem& p, const Workspace& ws, const float* O, const float* LSE,
                                  bool tensor_core, cudaStream_t st);
 bool tc_fused_select_supported(const Problem& p, int sm_count, bool reuse_l2, int keep, int W, int gamma);
-size_t tc_fused_select_sfx_words(int BH, int sm_count);
+size_t tc_fused_select_sfx_words(int sm_count);
 size_t tc_fused_select_hist_words(int BH);
 cudaError_t launch_decode_pad(const Problem& p, const void* q, __nv_bfloat16* q_pad, cudaStream_t st);
 cudaError_t launch_decode_extract(const Problem& p, const float* O_f32, const float* row_M2, float* out, float* lse,

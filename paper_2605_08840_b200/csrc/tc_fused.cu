@@ -58,7 +58,7 @@ struct FusedArgs {
   float* sel_scores;                 // [BH, n_kv] pooled scores
   int32_t* sel_indices;              // [BH, keep]
   unsigned int* sel_hist;            // [BH, 4, 256] digit histograms of the group, zero at launch
-  unsigned int* sel_sfx;             // [BH, cpg, 4, kSfxStride] per CTA: suffix sums of its own digit histograms
+  unsigned int* sel_sfx;             // [CTA, 4, kSfxStride] per CTA: suffix sums of its own digit histograms
   const __nv_bfloat16* K;
   long long ksb, ksh, ksn;
   __nv_bfloat16* K_out;              // [BH, keep, 128]
@@ -973,7 +973,9 @@ __device__ bool select_worker(const Ctx& cx, const FusedArgs& a, const Plan& pl,
   }
   // ---- 2. radix passes ----
   unsigned int prefix = 0, remaining = (unsigned int)keep;
-  unsigned int* sfx_mine = a.sel_sfx + ((long long)bh * a.cpg + pl.rank) * kSelPasses * kSfxStride;
+  // one slot per CTA, reused from head to head: a CTA has read its peers' sums of a head before it passes that
+  // head's last group barrier, and the peers write the next head's only after it
+  unsigned int* sfx_mine = a.sel_sfx + ((long long)pl.group * a.cpg + pl.rank) * kSelPasses * kSfxStride;
 #pragma unroll 1
   for (int p = 0; p < kSelPasses; ++p) {
     const int lo = 24 - 8 * p;
@@ -1042,7 +1044,7 @@ __device__ bool select_worker(const Ctx& cx, const FusedArgs& a, const Plan& pl,
       // keys of the lower ranks above the chosen digit (and, in the last pass, equal to the threshold key)
       unsigned int g = 0, e = 0;
       for (int r = lane; r < pl.rank; r += 32) {
-        const unsigned int* sr = a.sel_sfx + (((long long)bh * a.cpg + r) * kSelPasses + p) * kSfxStride;
+        const unsigned int* sr = a.sel_sfx + (((long long)pl.group * a.cpg + r) * kSelPasses + p) * kSfxStride;
         const unsigned int above = __ldcg(sr + d + 1);
         g += above;
         if (p == kSelPasses - 1) e += __ldcg(sr + d) - above;
@@ -1388,7 +1390,7 @@ bool tc_fused_select_supported(const Problem& p, int sm_count, bool reuse_l2, in
   const int tiles = (p.n_kv + kTile - 1) / kTile, per = (tiles + cpg - 1) / cpg;
   return (long long)per * kTile <= kSelMaxKeys;
 }
-size_t tc_fused_select_sfx_words(int BH, int sm_count) { return (size_t)BH * sm_count * kSelPasses * kSfxStride; }
+size_t tc_fused_select_sfx_words(int sm_count) { return (size_t)sm_count * kSelPasses * kSfxStride; }
 size_t tc_fused_select_hist_words(int BH) { return (size_t)BH * kSelPasses * 256; }
 
 cudaError_t launch_from_lse_prep(const Problem& p, const Workspace& ws, const float* O, const float* LSE,
