@@ -72,7 +72,7 @@ def whole_job_value(tokens_per_rank_step, world, steps, total_ms):
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from an ncu capture
 # of this workload, together with the digest of the kernel sources the capture was taken on: the figure is reported
 # only while those sources are unchanged, otherwise `traffic` is null.
-KERNEL_TRAFFIC = {"cfg4": {"bytes": 1026520576 + 25419008, "sources_sha256": "2b8344ba553ac6b728c54ef178f6f0f5e42d63d87f25c661464c202f37d9a137"}}
+KERNEL_TRAFFIC = {"cfg4": {"bytes": 1027409664 + 26176256, "sources_sha256": "595146513b8956870b53db3635e0ce99c42d3f6c9114f6dc45ba2ce04fc327a4"}}
 KERNEL_SOURCES = ("tc_fused.cu", "tc_common.cuh", "sm100_ptx.cuh")
 
 
