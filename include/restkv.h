@@ -130,6 +130,17 @@ restkv_status restkv_score_from_lse(restkv_handle* h, const restkv_shape* shape,
                                     size_t workspace_bytes, restkv_stream stream);
 
 /*
+ * restkv_evict_from_lse -- restkv_evict with the window rows' O_obs and LSE_obs given as for
+ * restkv_score_from_lse (Appendix B; Eq. 3, 7-9, 13, 14): score, select and compact with one read of K and V.
+ * All other arguments, outputs and error codes as for restkv_evict.
+ */
+restkv_status restkv_evict_from_lse(restkv_handle* h, const restkv_shape* shape, const void* Q_obs, const void* K,
+                                    const void* V, const float* O_obs, const float* LSE_obs, float ema_decay,
+                                    const restkv_pool_params* pool, int budget, float* scores_out, int32_t* indices,
+                                    void* K_out, void* V_out, void* workspace, size_t workspace_bytes,
+                                    restkv_stream stream);
+
+/*
  * restkv_select -- Eq. 14's argmax_B: per (batch, KV head) the min(budget, n_kv) largest scores,
  * ties to the lower index, indices written in ascending order.
  *   scores   device float [batch, n_kv_heads, n_kv] (+inf allowed, NaN not)

@@ -21,7 +21,7 @@ PATH_AUTO, PATH_SIMT, PATH_TENSOR_CORE, PATH_HEAD_SEQUENTIAL = 0, 1, 2, 3
 
 EXPORTS = [
     "restkv_create", "restkv_destroy", "restkv_workspace_bytes", "restkv_workspace_bytes_adaptive",
-    "restkv_score", "restkv_score_from_lse", "restkv_select", "restkv_compact", "restkv_evict", "restkv_evict_host", "restkv_decode", "restkv_decode_static",
+    "restkv_score", "restkv_score_from_lse", "restkv_select", "restkv_compact", "restkv_evict", "restkv_evict_from_lse", "restkv_evict_host", "restkv_decode", "restkv_decode_static",
     "restkv_decode_static_last_cuda_error",
     "restkv_poll_status", "restkv_launch_count", "restkv_last_cuda_error", "restkv_error_string",
     "restkv_set_kernel_path", "restkv_set_profile_events", "restkv_set_wait_limit", "restkv_set_fused_select", "restkv_last_evict_fused_select",
@@ -77,6 +77,7 @@ def load_library() -> ctypes.CDLL:
     lib.restkv_select.argtypes = [vp, shp, vp, ci, vp, vp, sz, vp]
     lib.restkv_compact.argtypes = [vp, shp, vp, vp, vp, ci, vp, vp, vp]
     lib.restkv_evict.argtypes = [vp, shp, vp, vp, vp, cf, pool, ci, vp, vp, vp, vp, vp, sz, vp]
+    lib.restkv_evict_from_lse.argtypes = [vp, shp, vp, vp, vp, vp, vp, cf, pool, ci, vp, vp, vp, vp, vp, sz, vp]
     lib.restkv_evict_host.argtypes = [vp, shp, vp, vp, vp, cf, pool, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.restkv_decode.argtypes = [vp, shp, vp, vp, vp, ci, vp, vp, vp, sz, vp]
     lib.restkv_decode_static.argtypes = [shp, vp, vp, vp, ci, vp, vp, vp]
@@ -200,6 +201,15 @@ class Handle:
                                            _ptr(indices), _ptr(K_out), _ptr(V_out), _ptr(workspace),
                                            workspace.numel() * workspace.element_size(), _stream_ptr(stream)),
                     "restkv_evict")
+
+    def evict_from_lse(self, shape, Q_obs, K, V, O_obs, LSE_obs, ema_decay, pool, budget, indices, K_out, V_out,
+                       workspace, scores_out=None, stream=None):
+        self._check(self._lib.restkv_evict_from_lse(self._h, ctypes.byref(shape), _ptr(Q_obs), _ptr(K), _ptr(V),
+                                                    _ptr(O_obs), _ptr(LSE_obs), float(ema_decay), ctypes.byref(pool),
+                                                    int(budget), _ptr(scores_out), _ptr(indices), _ptr(K_out),
+                                                    _ptr(V_out), _ptr(workspace),
+                                                    workspace.numel() * workspace.element_size(), _stream_ptr(stream)),
+                    "restkv_evict_from_lse")
 
     def evict_host(self, shape, Q_host, K_host, V_host, ema_decay, pool, budget, indices_host, K_out_host,
                    V_out_host, d_Q, d_K, d_V, d_indices, d_K_out, d_V_out, workspace, stream=None):

@@ -210,9 +210,12 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
     // the window rows' outputs and log-sum-exps come from the caller: pass 1 and the merge are not needed
     RESTKV_LAUNCH(c, RESTKV_KERNEL_COMBINE, launch_from_lse_prep(p, ws, O_given, LSE_given, use_tc, c.st), 1);
     if (use_tc) {
+      const bool with_sel = sel && c.h->fused_select &&
+                            tc_fused_select_supported(p, c.h->sm_count, false, sel->keep, sel->W, sel->gamma);
       RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2,
                     launch_tc_fused(c.h->tc_state, p, ws, Q, K, V, ema_decay, c.h->sm_count, false, false,
-                                    c.h->wait_limit, nullptr, O_given, c.h->dev_status, c.st), 1);
+                                    c.h->wait_limit, with_sel ? sel : nullptr, O_given, c.h->dev_status, c.st), 1);
+      if (sel_done) *sel_done = with_sel;
     } else {
       Workspace wsl = ws;
       wsl.O_f32 = const_cast<float*>(O_given);
@@ -381,10 +384,11 @@ restkv_status restkv_compact(restkv_handle* h, const restkv_shape* shape, const 
   return RESTKV_OK;
 }
 
-restkv_status restkv_evict(restkv_handle* h, const restkv_shape* shape, const void* Q_obs, const void* K,
-                           const void* V, float ema_decay, const restkv_pool_params* pool, int budget,
-                           float* scores_out, int32_t* indices, void* K_out, void* V_out, void* workspace,
-                           size_t workspace_bytes, restkv_stream stream) {
+static restkv_status evict_impl(restkv_handle* h, const restkv_shape* shape, const void* Q_obs, const void* K,
+                                const void* V, const float* O_obs, const float* LSE_obs, float ema_decay,
+                                const restkv_pool_params* pool, int budget, float* scores_out, int32_t* indices,
+                                void* K_out, void* V_out, void* workspace, size_t workspace_bytes,
+                                restkv_stream stream) {
   if (!h || !Q_obs || !K || !V || !indices || !K_out || !V_out || budget < 1) return RESTKV_ERR_INVALID_ARG;
   if (!aligned16(Q_obs) || !aligned16(K) || !aligned16(V) || !aligned16(K_out) || !aligned16(V_out))
     return RESTKV_ERR_INVALID_ARG;
@@ -405,8 +409,8 @@ restkv_status restkv_evict(restkv_handle* h, const restkv_shape* shape, const vo
   const int keep_rows = budget < p.n_kv ? budget : p.n_kv;
   FusedSelect sel{keep_rows, pool->width, pool->shift, scores, indices, K_out, V_out};
   bool sel_done = false;
-  if ((s = run_score(c, p, ws, Q_obs, K, V, ema_decay, pool, nullptr, nullptr, adaptive ? nullptr : &sel, &sel_done)) !=
-      RESTKV_OK)
+  if ((s = run_score(c, p, ws, Q_obs, K, V, ema_decay, pool, nullptr, nullptr, adaptive ? nullptr : &sel, &sel_done,
+                     O_obs, LSE_obs)) != RESTKV_OK)
     return s;
   h->last_evict_fused = sel_done;
   if (sel_done) return RESTKV_OK;
@@ -424,6 +428,24 @@ restkv_status restkv_evict(restkv_handle* h, const restkv_shape* shape, const vo
                   launch_compact(p, K, V, indices, n_sel, K_out, V_out, h->dev_status, c.st), 1);
   }
   return RESTKV_OK;
+}
+
+restkv_status restkv_evict(restkv_handle* h, const restkv_shape* shape, const void* Q_obs, const void* K,
+                           const void* V, float ema_decay, const restkv_pool_params* pool, int budget,
+                           float* scores_out, int32_t* indices, void* K_out, void* V_out, void* workspace,
+                           size_t workspace_bytes, restkv_stream stream) {
+  return evict_impl(h, shape, Q_obs, K, V, nullptr, nullptr, ema_decay, pool, budget, scores_out, indices, K_out, V_out,
+                    workspace, workspace_bytes, stream);
+}
+
+restkv_status restkv_evict_from_lse(restkv_handle* h, const restkv_shape* shape, const void* Q_obs, const void* K,
+                                    const void* V, const float* O_obs, const float* LSE_obs, float ema_decay,
+                                    const restkv_pool_params* pool, int budget, float* scores_out, int32_t* indices,
+                                    void* K_out, void* V_out, void* workspace, size_t workspace_bytes,
+                                    restkv_stream stream) {
+  if (!O_obs || !LSE_obs || !aligned16(O_obs)) return RESTKV_ERR_INVALID_ARG;
+  return evict_impl(h, shape, Q_obs, K, V, O_obs, LSE_obs, ema_decay, pool, budget, scores_out, indices, K_out, V_out,
+                    workspace, workspace_bytes, stream);
 }
 
 restkv_status restkv_evict_host(restkv_handle* h, const restkv_shape* shape, const void* Q_host, const void* K_host,

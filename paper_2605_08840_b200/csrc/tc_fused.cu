@@ -804,16 +804,8 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
         tmem_wait_ld();
         tmem_ld16(tS + 16, sv1);   // the second half of the columns travels while the first is worked on
         tmem_ld16(tC + 16, cv1);
-        if (from_lse) {
-          // does any of this warp's entries carry a weight above kHeavyA (S' above heavy_thr)?  If so the warp takes
-          // the slow path below, which reads the accumulators again: they are released only after this vote
-          tmem_wait_ld();
-          float mx = fmaxf(sv0[0], sv1[0]);
-#pragma unroll
-          for (int u = 1; u < 16; ++u) mx = fmaxf(mx, fmaxf(sv0[u], sv1[u]));
-          tile_heavy = __any_sync(0xffffffffu, mx > heavy_thr && j < n);
-        }
       }
+      bool redo_heavy = false;   // from_lse: this warp found a weight above kHeavyA among the logits it holds
       if (!tile_heavy) {
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
@@ -825,6 +817,16 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&B->acc_empty[s]);
+            if (from_lse) {
+              // no pass 1 has flagged the tiles with large weights: the warp looks at the logits it now holds in
+              // registers (S' above heavy_thr <=> A > kHeavyA) and, if it finds one, does its part of the tile again
+              // below with exact distances, from those registers (the accumulators are already released)
+              float mx = fmaxf(sv0[0], sv1[0]);
+#pragma unroll
+              for (int u = 1; u < 16; ++u) mx = fmaxf(mx, fmaxf(sv0[u], sv1[u]));
+              redo_heavy = __any_sync(0xffffffffu, mx > heavy_thr && j < n);
+              if (redo_heavy) break;
+            }
           }
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
@@ -839,6 +841,38 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
           if ((c * 16 + 16) % kRun == 0) {   // end of a run
             tot += fmaf(f2_lo(h2), ema_decay, f2_hi(h2));
             h2 = f2_make(0.f, 0.f);
+          }
+        }
+        if (from_lse && redo_heavy) {
+          tot = 0.f;
+          h2 = f2_make(0.f, 0.f);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const float* sv = (c < 2 ? sv0 : sv1) + (c & 1) * 8;
+            const float* cv = (c < 2 ? cv0 : cv1) + (c & 1) * 8;
+            float I[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const float um = ex2_approx(sv[u] * neg_c2) - 1.f;
+              float x = cv[u] + vnb;
+              unsigned int todo = __ballot_sync(0xffffffffu, sv[u] > heavy_thr && j < n);
+              while (todo) {
+                const int src = __ffs(todo) - 1;
+                todo &= todo - 1;
+                const int js = __shfl_sync(0xffffffffu, j, src);
+                const float d2x = exact_dist2_warp(O_head + (cgp * 32 + c * 8 + u) * kHeadDim,
+                                                   V_head + (long long)js * a.vsn, lane);
+                if (lane == src) x = d2x;
+              }
+              I[u] = x * rsqrt_approx(fmaf(x * um, um, 1e-36f));
+            }
+            if ((c * 8) % kRun == 0) I[0] *= seed_coef;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) h2 = f2_fma(h2, d2, f2_make(I[2 * q], I[2 * q + 1]));
+            if ((c * 8 + 8) % kRun == 0) {   // end of a run
+              tot += fmaf(f2_lo(h2), ema_decay, f2_hi(h2));
+              h2 = f2_make(0.f, 0.f);
+            }
           }
         }
       } else {
@@ -1161,6 +1195,13 @@ __device__ void control_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, 
       tc_fence_before();
       __syncthreads();
       tc_fence_after();
+      if (a.sel_keep > 0) {   // as below: the worker warps pool, select and gather; this side runs the group barriers
+        bool sel_ok = true;
+        for (int i = 0; i < kSelBarriers && sel_ok; ++i)
+          sel_ok = group_barrier(counter, (++epoch) * (unsigned int)a.cpg, abort_flag, go, a.dev_status, a.wait_limit);
+        if (!sel_ok) break;
+        __syncthreads();
+      }
       continue;
     }
     phase_a_control(cx, a, tmQ, tmK, tmV, bh, pl.rank, pl.tile0, pl.T1);
@@ -1207,6 +1248,10 @@ __device__ void worker_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, c
       tc_fence_before();
       __syncthreads();
       tc_fence_after();
+      if (a.sel_keep > 0) {
+        if (!select_worker(cx, a, pl, bh, go)) break;
+        __syncthreads();
+      }
       continue;
     }
     phase_a_worker(cx, a, tmQ, tmK, tmV, bh, pl.rank, pl.tile0, pl.T1);

@@ -516,16 +516,49 @@ def test_score_from_lse_matches_oracle(handle, spec):
     assert_scores_close(run.scores.cpu().numpy(), ref.scores, TOL[dtype])
 
 
+@pytest.mark.parametrize("spec", [("cfg2", 0), ("cfg2", 32), ("cfg1b", 0)])
+def test_evict_from_lse_matches_oracle(handle, spec):
+    """restkv_evict_from_lse: score, select and compact from given window statistics, all three acceptance rules."""
+    import torch
+    name, tail = spec
+    inp = make_inputs(CONFIGS[name].with_(causal_tail=tail))
+    c = inp.case
+    ref, O, lse = _window_stats(inp, with_A_check=False)
+    run = GpuRun(handle, inp)
+    handle.evict_from_lse(run.shape, run.Q, run.K, run.V, torch.from_numpy(O).cuda(), torch.from_numpy(lse).cuda(),
+                          c.ema_decay, run.pool(), run.budget, run.indices, run.K_out, run.V_out, run.ws,
+                          scores_out=run.scores)
+    torch.cuda.synchronize()
+    assert handle.poll_status() == rk.RESTKV_OK
+    idx = run.indices.cpu().numpy()
+    assert_scores_close(run.scores.cpu().numpy(), ref.scores, TOL[c.dtype])
+    assert_selection_valid(idx, ref.scores, run.budget, TOL[c.dtype])
+    _, kbits, vbits = inp.device_arrays()
+    assert_compaction_exact(idx, kbits, run._bits(run.K_out))
+    assert_compaction_exact(idx, vbits, run._bits(run.V_out))
+
+
 def test_score_from_lse_at_full_size(handle):
     import torch
     inp = make_inputs(CONFIGS["cfg4"])
     ref, O, lse = _window_stats(inp, with_A_check=False)
     run = GpuRun(handle, inp)
-    handle.score_from_lse(run.shape, run.Q, run.K, run.V, torch.from_numpy(O).cuda(), torch.from_numpy(lse).cuda(),
-                          inp.case.ema_decay, run.pool(), run.scores, run.ws)
+    dO, dL = torch.from_numpy(O).cuda(), torch.from_numpy(lse).cuda()
+    handle.score_from_lse(run.shape, run.Q, run.K, run.V, dO, dL, inp.case.ema_decay, run.pool(), run.scores, run.ws)
     torch.cuda.synchronize()
     assert handle.poll_status() == rk.RESTKV_OK
     assert_scores_close(run.scores.cpu().numpy(), ref.scores, TOL["bf16"])
+    run.scores.zero_()
+    handle.evict_from_lse(run.shape, run.Q, run.K, run.V, dO, dL, inp.case.ema_decay, run.pool(), run.budget,
+                          run.indices, run.K_out, run.V_out, run.ws, scores_out=run.scores)
+    torch.cuda.synchronize()
+    assert handle.poll_status() == rk.RESTKV_OK
+    idx = run.indices.cpu().numpy()
+    assert_scores_close(run.scores.cpu().numpy(), ref.scores, TOL["bf16"])
+    assert_selection_valid(idx, ref.scores, run.budget, TOL["bf16"])
+    _, kbits, vbits = inp.device_arrays()
+    assert_compaction_exact(idx, kbits, run._bits(run.K_out))
+    assert_compaction_exact(idx, vbits, run._bits(run.V_out))
 
 
 # ------------------------------------------------------------------ a device-side wait that runs out
