@@ -21,11 +21,15 @@
  *   adaptive window parameters     Eq. 10-12
  *   box pooling (final indicator)  Eq. 13
  *   top-B and gather               Eq. 14
+ *   ablation variants              Appendix G.1 (indicators: attention weight alone, attention weight times
+ *                                  the value's norm), Appendix G.2 (temporal: none, mean, inverted EMA;
+ *                                  spatial: max instead of mean over the box)
  *
  * Pins (tests that do not depend on this file's own arithmetic): brute-force token
  * deletion (Eq. 6) in NumPy, the renormalisation relation of Appendix A, uniform-logit
  * and two-token closed forms, EMA closed-form weights, pooling identities, a library
- * stable sort for the selection, library softmax attention for decode.
+ * stable sort for the selection, library softmax attention for decode; for the variants:
+ * library softmax and norms, closed-form temporal weights, time reversal, a library maximum filter.
  * Readings with no independent pin ("parity unpinned"): mean over the query heads of a
  * GQA group (the paper is silent), and how a fixed kernel width combines with the
  * adaptive width (box of width W_s + base_width - 1).
@@ -101,6 +105,12 @@ static int top_indices(const double* x, int n, int count, int* out) {
  *  budget       adaptive mode: B of Eq. 10
  *  literal_gamma  adaptive mode: 1 = Eq. 12 exactly as printed, 0 = truncate toward zero
  *  group_mode   0 = mean over the G query heads of a KV head, 1 = max over them
+ *  indicator_mode  0 = Eq. 7;  1 = the attention weight A[j] alone;  2 = A[j] * ||v_j||_2   (Appendix G.1)
+ *  temporal_mode   0 = EMA of Eq. 8-9;  1 = mean over the w queries;  2 = the EMA recursion run from the newest
+ *                  query to the oldest ("Inv-EMA": the oldest query weighs most);  3 = none: the newest query's
+ *                  indicator alone   (Appendix G.2)
+ *  spatial_mode    0 = box mean of Eq. 13;  1 = maximum over the same box, taps outside the scored rows count
+ *                  as 0 as they do in the mean   (Appendix G.2)
  *
  * Optional outputs (NULL to skip):
  *  A_out     [batch, Hq, w, n_kv]  attention weights (Eq. 3)
@@ -111,14 +121,17 @@ static int top_indices(const double* x, int n, int count, int* out) {
  *  D_out     [batch, Hkv, 2]       (D_front, D_rear), adaptive mode only
  * Required: scores [batch, Hkv, n_kv].
  */
-int restkv_oracle_score(const float* Q, const float* K, const float* V,
+int restkv_oracle_score_variant(const float* Q, const float* K, const float* V,
                         int batch, int Hq, int Hkv, int d, int n_kv, int w, int causal_tail,
                         double scale, double ema_decay,
                         int pool_mode, int width, int shift, double beta, int base_width,
                         int budget, int literal_gamma, int group_mode,
+                        int indicator_mode, int temporal_mode, int spatial_mode,
                         double* A_out, double* O_out, double* I_raw, double* I_hat,
                         int* pool_out, double* D_out, double* scores) {
   if (!Q || !K || !V || !scores) return ORACLE_BAD_ARG;
+  if (indicator_mode < 0 || indicator_mode > 2 || temporal_mode < 0 || temporal_mode > 3) return ORACLE_BAD_ARG;
+  if (spatial_mode < 0 || spatial_mode > 1) return ORACLE_BAD_ARG;
   if (batch < 1 || Hq < 1 || Hkv < 1 || d < 1 || w < 1 || n_kv < 1) return ORACLE_BAD_ARG;
   if (Hq % Hkv != 0) return ORACLE_BAD_ARG;
   if (causal_tail != 0 && causal_tail != w) return ORACLE_BAD_ARG;
@@ -169,7 +182,7 @@ int restkv_oracle_score(const float* Q, const float* K, const float* V,
         for (int j = 0; j < visible; ++j)
           for (int k = 0; k < d; ++k) o[k] += a[j] * (double)Vh[(size_t)j * d + k]; /* z_t = A_t V */
         /* Eq. 7 with W_O = identity: I[j] = A[j] / (1 - A[j]) * || z_t - v_j ||_2 */
-        for (int j = 0; j < n; ++j) {
+        for (int j = 0; j < n && indicator_mode == 0; ++j) {
           double ss = 0.0;
           for (int k = 0; k < d; ++k) {
             double df = o[k] - (double)Vh[(size_t)j * d + k];
@@ -178,6 +191,12 @@ int restkv_oracle_score(const float* Q, const float* K, const float* V,
           double one_minus = 1.0 - a[j];
           /* a single visible row has A = 1 and nothing to redistribute to: define I = 0 */
           Ih[((size_t)g * w + i) * n + j] = (visible == 1) ? 0.0 : a[j] / one_minus * sqrt(ss);
+        }
+        /* Appendix G.1: the attention weight alone, or weighted by the norm of the value */
+        for (int j = 0; j < n && indicator_mode != 0; ++j) {
+          double vv = 0.0;
+          for (int k = 0; k < d; ++k) vv += (double)Vh[(size_t)j * d + k] * (double)Vh[(size_t)j * d + k];
+          Ih[((size_t)g * w + i) * n + j] = (indicator_mode == 1) ? a[j] : a[j] * sqrt(vv);
         }
         if (A_out) memcpy(A_out + (((size_t)b * Hq + hq) * w + i) * n_kv, a, (size_t)n_kv * sizeof(double));
         if (O_out) memcpy(O_out + (((size_t)b * Hq + hq) * w + i) * d, o, (size_t)d * sizeof(double));
@@ -193,9 +212,21 @@ int restkv_oracle_score(const float* Q, const float* K, const float* V,
       for (int j = 0; j < n; ++j) {
         double red = 0.0;
         for (int g = 0; g < G; ++g) {
-          double ema = Ih[((size_t)g * w + 0) * n + j];              /* t1 == t2 */
-          for (int i = 1; i < w; ++i)
-            ema = alpha * Ih[((size_t)g * w + i) * n + j] + (1.0 - alpha) * ema;
+          const double* col = Ih + (size_t)g * w * n + j;              /* col[i * n] = I of query i */
+          double ema;
+          if (temporal_mode == 0) {
+            ema = col[0];                                               /* t1 == t2 */
+            for (int i = 1; i < w; ++i) ema = alpha * col[(size_t)i * n] + (1.0 - alpha) * ema;
+          } else if (temporal_mode == 1) {                              /* Appendix G.2: mean */
+            ema = 0.0;
+            for (int i = 0; i < w; ++i) ema += col[(size_t)i * n];
+            ema /= (double)w;
+          } else if (temporal_mode == 2) {                              /* Appendix G.2: EMA in reversed time */
+            ema = col[(size_t)(w - 1) * n];
+            for (int i = w - 2; i >= 0; --i) ema = alpha * col[(size_t)i * n] + (1.0 - alpha) * ema;
+          } else {                                                      /* Appendix G.2: no temporal smoothing */
+            ema = col[(size_t)(w - 1) * n];
+          }
           if (group_mode == 0) red += ema;
           else red = (g == 0 || ema > red) ? ema : red;
         }
@@ -243,12 +274,12 @@ int restkv_oracle_score(const float* Q, const float* K, const float* V,
       double* sc = scores + ((size_t)b * Hkv + h) * n_kv;
       const int half = W / 2;
       for (int j = 0; j < n; ++j) {
-        double s = 0.0;
+        double s = 0.0, mxv = 0.0;
         for (int k = -half + gamma; k <= half + gamma; ++k) {
           long t = (long)j + k;
-          if (t >= 0 && t < n) s += ihat[t];
+          if (t >= 0 && t < n) { s += ihat[t]; if (ihat[t] > mxv) mxv = ihat[t]; }
         }
-        sc[j] = s / (double)W;
+        sc[j] = (spatial_mode == 0) ? s / (double)W : mxv;
       }
       for (int j = n; j < n_kv; ++j) sc[j] = INFINITY;
 
@@ -256,6 +287,19 @@ int restkv_oracle_score(const float* Q, const float* K, const float* V,
     }
   }
   return status;
+}
+
+/* The method itself: Eq. 7, Eq. 8-9 and Eq. 13 as they are printed. */
+int restkv_oracle_score(const float* Q, const float* K, const float* V,
+                        int batch, int Hq, int Hkv, int d, int n_kv, int w, int causal_tail,
+                        double scale, double ema_decay,
+                        int pool_mode, int width, int shift, double beta, int base_width,
+                        int budget, int literal_gamma, int group_mode,
+                        double* A_out, double* O_out, double* I_raw, double* I_hat,
+                        int* pool_out, double* D_out, double* scores) {
+  return restkv_oracle_score_variant(Q, K, V, batch, Hq, Hkv, d, n_kv, w, causal_tail, scale, ema_decay,
+                                     pool_mode, width, shift, beta, base_width, budget, literal_gamma, group_mode,
+                                     0, 0, 0, A_out, O_out, I_raw, I_hat, pool_out, D_out, scores);
 }
 
 /* Eq. 14: per row of `scores` [rows, n_kv], the min(budget, n_kv) largest entries

@@ -371,3 +371,111 @@ def test_oracle_rejects_bad_arguments():
         oracle.score(Q, K, V, causal_tail=2)           # neither 0 nor w
     with pytest.raises(TypeError):
         oracle.score(Q.astype(np.float64), K, V)
+
+
+# ---------------------------------------------------------------- Appendix G variants
+def _library_attention(Q, K, causal_tail=0):
+    """A [b, Hq, w, n_kv] from scipy's softmax; query i of the window sees trailing row j' only if j' <= i."""
+    b, Hq, w, d = Q.shape
+    Hkv, n_kv = K.shape[1], K.shape[2]
+    G = Hq // Hkv
+    n = n_kv - causal_tail
+    A = np.zeros((b, Hq, w, n_kv))
+    for bi in range(b):
+        for hq in range(Hq):
+            logits = Q[bi, hq].astype(np.float64) @ K[bi, hq // G].astype(np.float64).T / np.sqrt(d)
+            for i in range(w):
+                vis = n_kv if causal_tail == 0 else n + i + 1
+                A[bi, hq, i, :vis] = softmax(logits[i, :vis])
+    return A
+
+
+@pytest.mark.parametrize("causal_tail", [0, 4])
+def test_variant_attention_weight_indicator_is_library_softmax(causal_tail):
+    # Appendix G.1 "attention weights": with mean over time and over the group it is the window-mean of A
+    Q, K, V = _qkv(b=2, Hq=4, Hkv=2, w=4, d=16, n_kv=30 + causal_tail, seed=11, kscale=2.0)
+    n = 30
+    res = oracle.score(Q, K, V, causal_tail=causal_tail, indicator_mode=1, temporal_mode=1, want_I_raw=True)
+    A = _library_attention(Q, K, causal_tail)
+    np.testing.assert_allclose(res.I_raw, A[..., :n], rtol=1e-12, atol=1e-15)
+    expect = A[..., :n].reshape(2, 2, 2, 4, n).mean(axis=(2, 3))
+    np.testing.assert_allclose(res.I_hat, expect, rtol=1e-12)
+    np.testing.assert_allclose(res.scores[..., :n], expect, rtol=1e-12)
+    assert np.isinf(res.scores[..., n:]).all()
+
+
+def test_variant_attention_times_value_norm():
+    Q, K, V = _qkv(b=1, Hq=2, Hkv=2, w=3, d=8, n_kv=20, seed=12, kscale=2.0)
+    V[0, 0, 5] *= np.float32(8.0)       # a long value must lift its token in proportion
+    res = oracle.score(Q, K, V, indicator_mode=2, want_I_raw=True)
+    A = _library_attention(Q, K)
+    expect = A * np.linalg.norm(V.astype(np.float64), axis=-1)[:, :, None, :]
+    np.testing.assert_allclose(res.I_raw, expect, rtol=1e-12)
+    plain = oracle.score(Q, K, V, indicator_mode=1, want_I_raw=True).I_raw
+    assert not np.allclose(res.I_raw, plain)
+
+
+@pytest.mark.parametrize("decay", [0.0, 0.3, 0.9])
+def test_variant_temporal_weights_closed_form(decay):
+    w, n = 6, 18
+    Q, K, V = _qkv(b=1, Hq=1, Hkv=1, w=w, d=8, n_kv=n, seed=13, kscale=2.0)
+    raw = oracle.score(Q, K, V, want_I_raw=True).I_raw[0, 0]          # [w, n]
+    alpha = 1.0 - decay
+    i = np.arange(w)
+    ema_w = np.where(i == 0, decay ** (w - 1), alpha * decay ** (w - 1.0 - i))
+    inv_w = np.where(i == w - 1, decay ** (w - 1), alpha * decay ** (1.0 * i))
+    last_w = (i == w - 1).astype(np.float64)
+    mean_w = np.full(w, 1.0 / w)
+    for mode, wt in ((0, ema_w), (1, mean_w), (2, inv_w), (3, last_w)):
+        assert abs(wt.sum() - 1.0) < 1e-12
+        got = oracle.score(Q, K, V, ema_decay=decay, temporal_mode=mode).I_hat[0, 0]
+        np.testing.assert_allclose(got, wt @ raw, rtol=1e-12, err_msg="temporal mode %d" % mode)
+
+
+def test_variant_inverted_ema_is_ema_of_the_reversed_window():
+    Q, K, V = _qkv(b=1, Hq=2, Hkv=1, w=5, d=8, n_kv=16, seed=14, kscale=2.0)
+    inv = oracle.score(Q, K, V, ema_decay=0.6, temporal_mode=2).I_hat
+    fwd = oracle.score(np.ascontiguousarray(Q[:, :, ::-1]), K, V, ema_decay=0.6).I_hat
+    np.testing.assert_allclose(inv, fwd, rtol=1e-12)
+    assert not np.allclose(inv, oracle.score(Q, K, V, ema_decay=0.6).I_hat)
+
+
+def test_variant_no_temporal_smoothing_is_the_newest_query_alone():
+    Q, K, V = _qkv(b=1, Hq=2, Hkv=1, w=5, d=8, n_kv=16, seed=15, kscale=2.0)
+    none = oracle.score(Q, K, V, ema_decay=0.6, temporal_mode=3).I_hat
+    only_last = oracle.score(np.ascontiguousarray(Q[:, :, -1:]), K, V, ema_decay=0.6).I_hat
+    np.testing.assert_allclose(none, only_last, rtol=1e-12)
+    np.testing.assert_allclose(none, oracle.score(Q, K, V, ema_decay=0.0).I_hat, rtol=1e-12)
+
+
+@pytest.mark.parametrize("width,shift", [(1, 0), (3, 0), (5, 2), (7, -3), (9, 30)])
+def test_variant_max_pool_matches_library_maximum_filter(width, shift):
+    from scipy.ndimage import maximum_filter1d
+    Q, K, V = _qkv(b=1, Hq=2, Hkv=2, w=3, d=8, n_kv=25, seed=16, kscale=2.0)
+    res = oracle.score(Q, K, V, width=width, shift=shift, spatial_mode=1)
+    half = width // 2
+    for h in range(2):
+        x = res.I_hat[0, h]
+        # out[j] = max x[j - half + shift .. j + half + shift]: pad by |shift| + half zeros and filter, then cut
+        pad = abs(shift) + half + 1
+        xp = np.concatenate([np.zeros(pad), x, np.zeros(pad)])
+        filt = maximum_filter1d(xp, size=width, mode="constant", cval=0.0)
+        expect = filt[pad + shift: pad + shift + x.size]
+        np.testing.assert_allclose(res.scores[0, h], expect, rtol=0, atol=0)
+    mean = oracle.score(Q, K, V, width=width, shift=shift).scores
+    assert (res.scores >= mean - 1e-15).all()
+
+
+def test_variant_group_max_is_max_over_separately_scored_heads():
+    Q, K, V = _qkv(b=1, Hq=4, Hkv=1, w=3, d=8, n_kv=20, seed=17, kscale=2.0)
+    got = oracle.score(Q, K, V, group_mode=1).I_hat[0, 0]
+    per_head = [oracle.score(np.ascontiguousarray(Q[:, g:g + 1]), K, V).I_hat[0, 0] for g in range(4)]
+    np.testing.assert_allclose(got, np.max(per_head, axis=0), rtol=1e-12)
+    np.testing.assert_allclose(oracle.score(Q, K, V).I_hat[0, 0], np.mean(per_head, axis=0), rtol=1e-12)
+
+
+def test_variant_modes_are_validated():
+    Q, K, V = _qkv()
+    for bad in (dict(indicator_mode=3), dict(temporal_mode=4), dict(spatial_mode=2), dict(indicator_mode=-1)):
+        with pytest.raises(RuntimeError):
+            oracle.score(Q, K, V, **bad)
