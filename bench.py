@@ -450,6 +450,32 @@ def main():
                                      "contractions (Q K^T, V O^T) instead of three"}
         del O_obs, L_obs, sc_out
 
+    # ---- the ablation variants of Appendix G as modes of the same path (beside the headline) ----
+    variants = None
+    if rank == 0:
+        labelled = (("attention_weight__mean_over_window", (rk.INDICATOR_ATTENTION, rk.TEMPORAL_MEAN, 0, 0)),
+                    ("attention_weight_times_value_norm__ema", (rk.INDICATOR_ATTENTION_VNORM, rk.TEMPORAL_EMA, 0, 0)),
+                    ("reconstruction__inverted_ema__max_pool__group_max",
+                     (rk.INDICATOR_RECONSTRUCTION, rk.TEMPORAL_INV_EMA, rk.SPATIAL_MAX, rk.GROUP_MAX)))
+        variants = {"note": "restkv_evict under restkv_set_variant, same workload and timing as the headline step",
+                    "evict_ms": {}}
+        for label, v in labelled:
+            handle.set_variant(*v)
+            try:
+                tv = []
+                for it in range(11):
+                    flush.zero_()
+                    ev0.record()
+                    step()
+                    ev1.record()
+                    torch.cuda.synchronize()
+                    if it >= 3:
+                        tv.append(ev0.elapsed_time(ev1))
+            finally:
+                handle.set_variant()
+            assert handle.poll_status() == rk.RESTKV_OK
+            variants["evict_ms"][label] = float(np.median(tv))
+
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----
     e2e = None
     if not args.no_e2e:
@@ -522,6 +548,7 @@ def main():
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roofline, "path_roofline": path_roofline, "kernels_ms": kmean,
         "kernels_ms_selection_as_own_kernel": kmean_split, "decode": decode, "from_lse": from_lse,
+        "variants": variants,
     }
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(inp, case.budget)

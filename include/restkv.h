@@ -274,6 +274,43 @@ int restkv_last_evict_fused_select(const restkv_handle* h);   /* 1 if the last r
  * that path and for callers that want to fail faster.  The paper has no counterpart. */
 restkv_status restkv_set_wait_limit(restkv_handle* h, long long sm_clocks);
 
+/* Ablation variants (Appendix G) as modes of the same kernels.  A handle starts with every field 0: the method as
+ * Sections 3.2-3.3 define it.  The setting applies to every later restkv_score, restkv_evict, restkv_evict_host,
+ * restkv_score_from_lse and restkv_evict_from_lse call through the handle; restkv_select, restkv_compact and the
+ * decode calls do not depend on it.
+ *   indicator (Appendix G.1, indicator table), per query t and token j:
+ *     RECONSTRUCTION  A_t[j] / (1 - A_t[j]) * ||o_t - v_j||_2, Eq. 7
+ *     ATTENTION       A_t[j], the attention weight alone
+ *     ATTENTION_VNORM A_t[j] * ||v_j||_2
+ *   temporal (Appendix G.2, smoothing table), over the w window queries, oldest first, alpha = 1 - ema_decay:
+ *     EMA      Eq. 8-9: the recursion from the oldest query on (the newest weighs alpha, the oldest (1-alpha)^(w-1))
+ *     MEAN     1/w each
+ *     INV_EMA  the same recursion run from the newest query to the oldest (the oldest weighs alpha)
+ *     NONE     the newest query's indicator alone
+ *   spatial (same table): MEAN = the box mean of Eq. 13; MAX = the maximum over the same box, taps outside the scored
+ *     rows counting as 0 like in the mean.  Applies to the fixed and to the adaptive window.
+ *   group: MEAN or MAX over the query heads that share a KV head (the paper leaves grouped-query attention open).
+ * Every combination is accepted.  The tensor-core kernel carries all of them except where its fp32 temporal chain
+ * cannot (EMA with ema_decay = 1; INV_EMA with ema_decay = 0, = 1 or (1/ema_decay)^(w-1) > 2^40): those run on the
+ * fp32 SIMT kernels, or return RESTKV_ERR_UNSUPPORTED under restkv_set_kernel_path(h, 2 or 3).  With
+ * indicator != RECONSTRUCTION a cache of one visible row scores A = 1 (times ||v||), not the 0 that Eq. 7's 0/0 is
+ * defined as.  v == NULL restores the defaults.  RESTKV_ERR_INVALID_ARG on a field out of range. */
+typedef enum {
+  RESTKV_INDICATOR_RECONSTRUCTION = 0, RESTKV_INDICATOR_ATTENTION = 1, RESTKV_INDICATOR_ATTENTION_VNORM = 2
+} restkv_indicator;
+typedef enum {
+  RESTKV_TEMPORAL_EMA = 0, RESTKV_TEMPORAL_MEAN = 1, RESTKV_TEMPORAL_INV_EMA = 2, RESTKV_TEMPORAL_NONE = 3
+} restkv_temporal;
+typedef enum { RESTKV_SPATIAL_MEAN = 0, RESTKV_SPATIAL_MAX = 1 } restkv_spatial;
+typedef enum { RESTKV_GROUP_MEAN = 0, RESTKV_GROUP_MAX = 1 } restkv_group;
+typedef struct {
+  int indicator;   /* restkv_indicator */
+  int temporal;    /* restkv_temporal */
+  int spatial;     /* restkv_spatial */
+  int group;       /* restkv_group */
+} restkv_variant;
+restkv_status restkv_set_variant(restkv_handle* h, const restkv_variant* v);   /* v: host pointer, read during the call */
+
 #ifdef __cplusplus
 }
 #endif

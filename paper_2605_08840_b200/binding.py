@@ -25,6 +25,7 @@ EXPORTS = [
     "restkv_decode_static_last_cuda_error",
     "restkv_poll_status", "restkv_launch_count", "restkv_last_cuda_error", "restkv_error_string",
     "restkv_set_kernel_path", "restkv_set_profile_events", "restkv_set_wait_limit", "restkv_set_fused_select", "restkv_last_evict_fused_select",
+    "restkv_set_variant",
 ]
 KERNEL_NONE, KERNEL_PASS1, KERNEL_COMBINE, KERNEL_PASS2, KERNEL_POOL, KERNEL_SELECT, KERNEL_COMPACT = range(7)
 
@@ -42,6 +43,18 @@ class Shape(ctypes.Structure):
 class PoolParams(ctypes.Structure):
     _fields_ = [("mode", ctypes.c_int), ("width", ctypes.c_int), ("shift", ctypes.c_int), ("beta", ctypes.c_float),
                 ("base_width", ctypes.c_int), ("budget", ctypes.c_int)]
+
+
+class Variant(ctypes.Structure):
+    """restkv_variant: the ablation variants of Appendix G as modes of the score calls (all 0 = the method)."""
+    _fields_ = [("indicator", ctypes.c_int), ("temporal", ctypes.c_int), ("spatial", ctypes.c_int),
+                ("group", ctypes.c_int)]
+
+
+INDICATOR_RECONSTRUCTION, INDICATOR_ATTENTION, INDICATOR_ATTENTION_VNORM = 0, 1, 2
+TEMPORAL_EMA, TEMPORAL_MEAN, TEMPORAL_INV_EMA, TEMPORAL_NONE = 0, 1, 2, 3
+SPATIAL_MEAN, SPATIAL_MAX = 0, 1
+GROUP_MEAN, GROUP_MAX = 0, 1
 
 
 class RestKVError(RuntimeError):
@@ -92,6 +105,7 @@ def load_library() -> ctypes.CDLL:
     lib.restkv_set_wait_limit.argtypes = [vp, ctypes.c_longlong]
     lib.restkv_set_fused_select.argtypes = [vp, ci]
     lib.restkv_last_evict_fused_select.argtypes = [vp]
+    lib.restkv_set_variant.argtypes = [vp, ctypes.POINTER(Variant)]
     _lib = lib
     return lib
 
@@ -239,6 +253,10 @@ class Handle:
 
     def last_evict_fused_select(self) -> bool:
         return bool(self._lib.restkv_last_evict_fused_select(self._h))
+
+    def set_variant(self, indicator: int = 0, temporal: int = 0, spatial: int = 0, group: int = 0):
+        v = Variant(int(indicator), int(temporal), int(spatial), int(group))
+        self._check(self._lib.restkv_set_variant(self._h, ctypes.byref(v)), "restkv_set_variant")
 
     def set_wait_limit(self, sm_clocks: int):
         self._check(self._lib.restkv_set_wait_limit(self._h, int(sm_clocks)), "restkv_set_wait_limit")

@@ -12,25 +12,30 @@ namespace cg = cooperative_groups;
 // ------------------------------------------------------------------------------------------------
 // Box mean of Eq. 13 at row j of one head: (1/W) * sum_{k=-W/2+gamma}^{W/2+gamma} I_hat[j+k], taps outside
 // [0,n) are zero; rows n..n_kv-1 (the window's own tokens) get +inf.
-__device__ __forceinline__ float box_mean(const float* __restrict__ src, int n, int j, int W, int gamma) {
+// pool_max (Appendix G.2): the maximum over the same taps instead, taps outside counting as 0 as well.
+__device__ __forceinline__ float box_mean(const float* __restrict__ src, int n, int j, int W, int gamma, bool pool_max) {
   if (j >= n) return INFINITY;
   const int half = W / 2;
   const long long lo64 = (long long)j - half + gamma, hi64 = (long long)j + half + gamma;
   const int lo = lo64 < 0 ? 0 : (int)(lo64 < n ? lo64 : n), hi = hi64 > n - 1 ? n - 1 : (int)(hi64 > -1 ? hi64 : -1);
   float s = 0.f;
+  if (pool_max) {
+    for (int t = lo; t <= hi; ++t) s = fmaxf(s, src[t]);
+    return s;
+  }
   for (int t = lo; t <= hi; ++t) s += src[t];
   return s / (float)W;
 }
 
 // grid (ceil(n_kv/256), BH).  The window (W, gamma) comes from `pool` (per head, device) when it is non-null.
 __global__ void pool_kernel(int n, int n_kv, const float* __restrict__ I_hat, const int* __restrict__ pool, int W,
-                            int gamma, float* __restrict__ scores, int32_t* __restrict__ pool_used) {
+                            int gamma, bool pool_max, float* __restrict__ scores, int32_t* __restrict__ pool_used) {
   const int bh = blockIdx.y;
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   if (pool) { W = pool[2 * bh]; gamma = pool[2 * bh + 1]; }
   if (pool_used && j == 0) { pool_used[2 * bh] = W; pool_used[2 * bh + 1] = gamma; }
   if (j >= n_kv) return;
-  scores[(long long)bh * n_kv + j] = box_mean(I_hat + (long long)bh * n, n, j, W, gamma);
+  scores[(long long)bh * n_kv + j] = box_mean(I_hat + (long long)bh * n, n, j, W, gamma, pool_max);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -126,8 +131,8 @@ __device__ __forceinline__ void pool_staged(const float* __restrict__ staged, in
 // index wins ties).
 __global__ void __launch_bounds__(kSelThreads, 1)
 select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const int* __restrict__ pool, int W,
-              int gamma, float* scores, int32_t* __restrict__ indices, int32_t* __restrict__ pool_used, int per,
-              int use_smem, int stage_taps, GatherArgs ga) {
+              int gamma, int pool_max, float* scores, int32_t* __restrict__ indices, int32_t* __restrict__ pool_used,
+              int per, int use_smem, int stage_taps, GatherArgs ga) {
   cg::cluster_group cluster = cg::this_cluster();
   const unsigned int CS = cluster.num_blocks(), rank = cluster.block_rank();
   const int row = blockIdx.x / CS;
@@ -151,7 +156,7 @@ select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const 
     if (pool) { W = pool[2 * row]; gamma = pool[2 * row + 1]; }
     if (pool_used && rank == 0 && tid == 0) { pool_used[2 * row] = W; pool_used[2 * row + 1] = gamma; }
     const float* src = I_hat + (long long)row * n;
-    if (stage_taps && W <= kSelMaxStagedWidth && cnt > 0) {
+    if (stage_taps && !pool_max && W <= kSelMaxStagedWidth && cnt > 0) {
       // the taps of the whole slice (slice + halo) are staged in shared memory once, then summed from there in
       // the same order as box_mean does
       float* staged = reinterpret_cast<float*>(skeys + per);
@@ -184,7 +189,7 @@ select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const 
       }
     } else {
       for (int jj = tid; jj < cnt; jj += kSelThreads) {
-        const float out = box_mean(src, n, (int)(j0 + jj), W, gamma);
+        const float out = box_mean(src, n, (int)(j0 + jj), W, gamma, pool_max != 0);
         srow[j0 + jj] = out;
         if (use_smem) skeys[jj] = float_key(out);
       }
@@ -435,14 +440,15 @@ __global__ void compact_kernel(int Hkv, int n_kv, int n_sel, int row_chunks, lon
 cudaError_t launch_pool(const Problem& p, const Workspace& ws, const int* pool_dev, int W, int gamma, float* scores,
                         int32_t* pool_used, cudaStream_t st) {
   dim3 grid((p.n_kv + 255) / 256, p.BH);
-  pool_kernel<<<grid, 256, 0, st>>>(p.n, p.n_kv, ws.I_hat, pool_dev, W, gamma, scores, pool_used);
+  pool_kernel<<<grid, 256, 0, st>>>(p.n, p.n_kv, ws.I_hat, pool_dev, W, gamma, p.spatial == RESTKV_SPATIAL_MAX, scores,
+                                    pool_used);
   return cudaGetLastError();
 }
 
 // rows x n_kv scores -> rows x min(budget, n_kv) indices.  I_hat non-null: pool first (n scored rows per row of
 // I_hat, window from pool_dev or (W, gamma)) and write the pooled scores.
 cudaError_t launch_select(int rows, int n, int n_kv, int budget, const float* I_hat, const int* pool_dev, int W,
-                          int gamma, float* scores, int32_t* indices, int32_t* pool_used, const Problem* gather,
+                          int gamma, bool pool_max, float* scores, int32_t* indices, int32_t* pool_used, const Problem* gather,
                           const void* K, const void* V, void* K_out, void* V_out, cudaStream_t st) {
   GatherArgs ga{};
   if (gather) {
@@ -482,8 +488,8 @@ cudaError_t launch_select(int rows, int n, int n_kv, int budget, const float* I_
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, select_kernel, n, n_kv, keep, I_hat, pool_dev, W, gamma, scores, indices, pool_used,
-                            per, use_smem, stage_taps, ga);
+  return cudaLaunchKernelEx(&cfg, select_kernel, n, n_kv, keep, I_hat, pool_dev, W, gamma, pool_max ? 1 : 0, scores, indices,
+                            pool_used, per, use_smem, stage_taps, ga);
 }
 
 cudaError_t launch_compact(const Problem& p, const void* K, const void* V, const int32_t* indices, int n_sel,

@@ -17,6 +17,7 @@ struct restkv_handle {
   bool fused_select;          // restkv_evict lets the tensor-core score kernel pool, select and gather when it can
   bool last_evict_fused;      // whether the last restkv_evict did
   long long wait_limit;       // SM clocks a device-side wait may last
+  restkv_variant variant;     // ablation variant of the score calls (all 0: the method as printed)
   cudaEvent_t prof_start[7], prof_stop[7];   // per restkv_kernel_id, null = not timed
 };
 
@@ -149,6 +150,11 @@ static restkv_status make_problem(const restkv_shape* s, bool need_kv, Problem* 
   return RESTKV_OK;
 }
 
+static void apply_variant(const restkv_handle* h, Problem* p) {
+  p->indicator = h->variant.indicator; p->temporal = h->variant.temporal;
+  p->spatial = h->variant.spatial; p->group = h->variant.group;
+}
+
 static restkv_status check_pool(const restkv_pool_params* pp, const Problem& p) {
   if (!pp) return RESTKV_ERR_INVALID_ARG;
   if (pp->mode == RESTKV_POOL_FIXED) {
@@ -194,12 +200,14 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
                                int32_t* pool_used, const FusedSelect* sel = nullptr, bool* sel_done = nullptr,
                                const float* O_given = nullptr, const float* LSE_given = nullptr) {
   const bool adaptive = pool->mode == RESTKV_POOL_ADAPTIVE;
-  // the tensor-core pass 2 seeds its EMA chain with 1/alpha, so ema_decay = 1 (alpha = 0) runs on the SIMT kernels
-  bool use_tc = tc_supported(p) && c.h->tc_state != nullptr && !adaptive && ema_decay < 1.f;
+  // the tensor-core pass 2 carries the temporal weights as an fp32 Horner chain, which Eq. 9 with alpha = 0 and
+  // some inverted EMAs do not fit: those run on the SIMT kernels
+  bool use_tc = tc_supported(p) && c.h->tc_state != nullptr && !adaptive && tc_variant_supported(p, ema_decay);
+  if (p.n_kv == 1 && p.indicator != RESTKV_INDICATOR_RECONSTRUCTION) use_tc = false;
   if (c.h->kernel_path == 1) use_tc = false;
   if (c.h->kernel_path >= 2 && !use_tc) return RESTKV_ERR_UNSUPPORTED;
   if (!use_tc && !simt_supported(p)) return RESTKV_ERR_UNSUPPORTED;
-  if (p.n_kv == 1) {
+  if (p.n_kv == 1 && p.indicator == RESTKV_INDICATOR_RECONSTRUCTION) {
     // A single visible row has A = 1 and nothing to redistribute its weight to: the indicator is
     // 0/0 there and is defined as 0 (Eq. 7 has no value), so no kernel is needed.
     cudaError_t e = cudaMemsetAsync(ws.I_hat, 0, (size_t)p.BH * p.n * sizeof(float), c.st);
@@ -281,6 +289,7 @@ restkv_status restkv_create(restkv_handle** out) {
   h->wait_limit = 2000000000ll;
   h->fused_select = true;
   h->last_evict_fused = false;
+  h->variant = restkv_variant{0, 0, 0, 0};
   h->launches = 0;
   h->last_cuda_error = 0;
   h->kernel_path = 0;
@@ -326,6 +335,7 @@ restkv_status restkv_score(restkv_handle* h, const restkv_shape* shape, const vo
   Problem p;
   restkv_status s = make_problem(shape, true, &p);
   if (s != RESTKV_OK) return s;
+  apply_variant(h, &p);
   if ((s = check_pool(pool, p)) != RESTKV_OK) return s;
   Workspace ws;
   const bool adaptive = pool->mode == RESTKV_POOL_ADAPTIVE;
@@ -347,6 +357,7 @@ restkv_status restkv_score_from_lse(restkv_handle* h, const restkv_shape* shape,
   Problem p;
   restkv_status s = make_problem(shape, true, &p);
   if (s != RESTKV_OK) return s;
+  apply_variant(h, &p);
   if ((s = check_pool(pool, p)) != RESTKV_OK) return s;
   Workspace ws;
   const bool adaptive = pool->mode == RESTKV_POOL_ADAPTIVE;
@@ -367,7 +378,7 @@ restkv_status restkv_select(restkv_handle* h, const restkv_shape* shape, const f
   if ((s = check_ws(p, budget, h->sm_count, false, workspace, workspace_bytes, &ws)) != RESTKV_OK) return s;
   Call c{h, (cudaStream_t)stream};
   RESTKV_LAUNCH(c, RESTKV_KERNEL_SELECT,
-                launch_select(p.BH, p.n, p.n_kv, budget, nullptr, nullptr, 1, 0, const_cast<float*>(scores), indices, nullptr,
+                launch_select(p.BH, p.n, p.n_kv, budget, nullptr, nullptr, 1, 0, false, const_cast<float*>(scores), indices, nullptr,
                               nullptr, nullptr, nullptr, nullptr, nullptr, c.st), 1);
   return RESTKV_OK;
 }
@@ -397,6 +408,7 @@ static restkv_status evict_impl(restkv_handle* h, const restkv_shape* shape, con
   Problem p;
   restkv_status s = make_problem(shape, true, &p);
   if (s != RESTKV_OK) return s;
+  apply_variant(h, &p);
   if ((s = check_pool(pool, p)) != RESTKV_OK) return s;
   Workspace ws;
   const bool adaptive = pool->mode == RESTKV_POOL_ADAPTIVE;
@@ -420,8 +432,8 @@ static restkv_status evict_impl(restkv_handle* h, const restkv_shape* shape, con
   const bool fuse_gather = p.BH * 8 <= h->sm_count;
   RESTKV_LAUNCH(c, RESTKV_KERNEL_SELECT,
                 launch_select(p.BH, p.n, p.n_kv, budget, ws.I_hat, adaptive ? ws.pool : nullptr, pool->width,
-                              pool->shift, scores, indices, nullptr, fuse_gather ? &p : nullptr, K, V, K_out, V_out,
-                              c.st), 1);
+                              pool->shift, p.spatial == RESTKV_SPATIAL_MAX, scores, indices, nullptr,
+                              fuse_gather ? &p : nullptr, K, V, K_out, V_out, c.st), 1);
   if (!fuse_gather) {
     const int n_sel = budget < p.n_kv ? budget : p.n_kv;
     RESTKV_LAUNCH(c, RESTKV_KERNEL_COMPACT,
@@ -589,6 +601,20 @@ restkv_status restkv_set_fused_select(restkv_handle* h, int on) {
 restkv_status restkv_set_wait_limit(restkv_handle* h, long long sm_clocks) {
   if (!h || sm_clocks < 1) return RESTKV_ERR_INVALID_ARG;
   h->wait_limit = sm_clocks;
+  return RESTKV_OK;
+}
+
+restkv_status restkv_set_variant(restkv_handle* h, const restkv_variant* v) {
+  if (!h) return RESTKV_ERR_INVALID_ARG;
+  if (!v) {
+    h->variant = restkv_variant{0, 0, 0, 0};
+    return RESTKV_OK;
+  }
+  if (v->indicator < 0 || v->indicator > RESTKV_INDICATOR_ATTENTION_VNORM) return RESTKV_ERR_INVALID_ARG;
+  if (v->temporal < 0 || v->temporal > RESTKV_TEMPORAL_NONE) return RESTKV_ERR_INVALID_ARG;
+  if (v->spatial < 0 || v->spatial > RESTKV_SPATIAL_MAX) return RESTKV_ERR_INVALID_ARG;
+  if (v->group < 0 || v->group > RESTKV_GROUP_MAX) return RESTKV_ERR_INVALID_ARG;
+  h->variant = *v;
   return RESTKV_OK;
 }
 

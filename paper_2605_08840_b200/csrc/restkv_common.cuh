@@ -24,6 +24,7 @@ struct Problem {
   float scale;            // softmax scale
   long long ksb, ksh, ksn, vsb, vsh, vsn;  // element strides
   restkv_dtype dtype;
+  int indicator, temporal, spatial, group;   // restkv_variant; all 0 = the method as the paper prints it
 };
 
 // Workspace carve-up (all offsets 256-byte aligned).
@@ -77,7 +78,7 @@ cudaError_t launch_simt_pass2(const Problem& p, const Workspace& ws, const void*
 cudaError_t launch_pool(const Problem& p, const Workspace& ws, const int* pool_dev, int W, int gamma, float* scores,
                         int32_t* pool_used, cudaStream_t st);
 cudaError_t launch_select(int rows, int n, int n_kv, int budget, const float* I_hat, const int* pool_dev, int W,
-                          int gamma, float* scores, int32_t* indices, int32_t* pool_used, const Problem* gather,
+                          int gamma, bool pool_max, float* scores, int32_t* indices, int32_t* pool_used, const Problem* gather,
                           const void* K, const void* V, void* K_out, void* V_out, cudaStream_t st);
 cudaError_t launch_compact(const Problem& p, const void* K, const void* V, const int32_t* indices, int n_sel,
                            void* K_out, void* V_out, unsigned int* dev_status, cudaStream_t st);
@@ -99,6 +100,8 @@ cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, 
 // normalisers; otherwise fin_m = LSE, fin_l = 1.
 cudaError_t launch_from_lse_prep(const Problem& p, const Workspace& ws, const float* O, const float* LSE,
                                  bool tensor_core, cudaStream_t st);
+// Whether the tensor-core kernel's temporal chain can carry the variant's weights for this decay and window.
+bool tc_variant_supported(const Problem& p, float ema_decay);
 bool tc_fused_select_supported(const Problem& p, int sm_count, bool reuse_l2, int keep, int W, int gamma);
 size_t tc_fused_select_sfx_words(int sm_count);
 size_t tc_fused_select_hist_words(int BH);

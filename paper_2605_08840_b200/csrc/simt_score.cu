@@ -175,11 +175,22 @@ __global__ void simt_pass2_kernel(Problem p, const T* __restrict__ Q, const T* _
   const float* kr = Kt + t * ld;
   const float* vr = Vt + t * ld;
 
-  float group_sum = 0.f;
+  // variants of Appendix G: p.indicator picks the per-query indicator, p.temporal the weights over the window
+  // queries, p.group the reduction over the query heads of the group
+  const bool gmax = p.group == RESTKV_GROUP_MAX;
+  float group_red = 0.f;
   if (t < valid) {
+    float vlen = 1.f;
+    if (p.indicator == RESTKV_INDICATOR_ATTENTION_VNORM) {
+      float vv = 0.f;
+      for (int k = 0; k < d; ++k) vv = fmaf(vr[k], vr[k], vv);
+      vlen = sqrtf(vv);
+    }
     for (int g = slot; g < p.G; g += GP) {
-      float ema = 0.f;
+      float ema = 0.f, pw = 1.f;   // pw = ema_decay^i for the inverted EMA
       for (int i = 0; i < p.w; ++i) {
+        // without temporal smoothing only the newest query counts (the raw indicators still want every query)
+        if (p.temporal == RESTKV_TEMPORAL_NONE && i != p.w - 1 && !I_raw) continue;
         const int r = g * p.w + i;
         const T* qr = Qh + (long long)r * d;
         const float* orow = Oh + (long long)r * d;
@@ -192,21 +203,41 @@ __global__ void simt_pass2_kernel(Problem p, const T* __restrict__ Q, const T* _
         const long long ri = (long long)bh * p.R + r;
         const float l = fin_l[ri];
         const float e = expf(s * p.scale - fin_m[ri]);
-        // 1 - A formed as (l - e) / l; clamped so that A -> 1 stays finite
-        const float one_minus = fmaxf((l - e) / l, 5.9604645e-8f);
-        const float I = (e / l) / one_minus * sqrtf(ss);
+        float I;
+        if (p.indicator == RESTKV_INDICATOR_RECONSTRUCTION) {
+          // 1 - A formed as (l - e) / l; clamped so that A -> 1 stays finite
+          const float one_minus = fmaxf((l - e) / l, 5.9604645e-8f);
+          I = (e / l) / one_minus * sqrtf(ss);
+        } else {
+          I = (e / l) * vlen;
+        }
         if (I_raw) I_raw[(((long long)b * p.Hq + (long long)h * p.G + g) * p.w + i) * p.n + j] = I;
-        ema = (i == 0) ? I : fmaf(alpha, I, ema_decay * ema);   // Eq. 9, oldest query first
+        switch (p.temporal) {
+          case RESTKV_TEMPORAL_EMA:   // Eq. 9, oldest query first
+            ema = (i == 0) ? I : fmaf(alpha, I, ema_decay * ema);
+            break;
+          case RESTKV_TEMPORAL_MEAN:
+            ema += I;
+            break;
+          case RESTKV_TEMPORAL_INV_EMA:   // the recursion run backwards: weights alpha d^i, d^(w-1) for the newest
+            ema = fmaf((i == p.w - 1) ? pw : alpha * pw, I, ema);
+            pw *= ema_decay;
+            break;
+          default:
+            if (i == p.w - 1) ema = I;
+            break;
+        }
       }
-      group_sum += ema;
+      if (p.temporal == RESTKV_TEMPORAL_MEAN) ema /= (float)p.w;
+      group_red = gmax ? fmaxf(group_red, ema) : group_red + ema;
     }
   }
-  red[slot * kP2Tile + t] = group_sum;
+  red[slot * kP2Tile + t] = group_red;
   __syncthreads();
   if (slot == 0 && t < valid) {
     float tot = 0.f;
-    for (int sl = 0; sl < GP; ++sl) tot += red[sl * kP2Tile + t];
-    I_hat[(long long)bh * p.n + j] = tot / (float)p.G;
+    for (int sl = 0; sl < GP; ++sl) tot = gmax ? fmaxf(tot, red[sl * kP2Tile + t]) : tot + red[sl * kP2Tile + t];
+    I_hat[(long long)bh * p.n + j] = gmax ? tot : tot / (float)p.G;
   }
 }
 

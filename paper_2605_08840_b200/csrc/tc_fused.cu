@@ -32,7 +32,12 @@ constexpr int kFVSlots = 3;                       // phase A: V slots = ring 2, 
 
 struct FusedArgs {
   int Hkv, BH, n, n_kv, w;
-  float scale, ema_decay;
+  float scale;
+  // Temporal weights (Eq. 9 and the variants of Appendix G.2) as a Horner chain: the score of a token is
+  // t_scale * sum_i c_i I_i t_decay^(w-1-i) with c_0 = t_seed_first, c_(w-1) = t_seed_last, c_i = 1 otherwise (w >= 16 here).
+  float t_decay, t_seed_first, t_seed_last, t_scale;
+  int group_max;                     // 1: maximum over the query heads of a group instead of their mean
+  int pool_max;                      // 1: the selection phase takes the maximum over the box instead of the mean
   int groups, cpg;                   // CTA groups and CTAs per group
   int attention_only;                // 1: stop after the merge (phases A and B): plain attention of the 128 rows
   int from_lse;                      // 1: O and the rows' log-sum-exp are given: phases A and B are skipped, phase C
@@ -703,7 +708,8 @@ __device__ void phase_c_control(const Ctx& cx, const FusedArgs& a, const CUtenso
   }
 }
 
-template <int kW, bool kLse>
+// kInd: 0 = Eq. 7; 1 = the attention weight alone; 2 = attention weight times ||v|| (Appendix G.1).
+template <int kW, bool kLse, int kInd>
 __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tmO, const CUtensorMap* tmAug,
                         const CUtensorMap* tmK, const CUtensorMap* tmV, int bh, int tile0, int T, int pre,
                         float (*red)[4][kTile]) {
@@ -720,20 +726,29 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
   const int quad = warp & 3;                       // TMEM lane quarter this warp may touch
   const int t = quad * 32 + lane;
   const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-  const float ema_decay = a.ema_decay;
+  const float ema_decay = a.t_decay;
   const float neg_c2 = -a.scale * kLog2e;
   const float heavy_thr = log2f(1.f / kHeavyA) / neg_c2;   // S' above this <=> A > kHeavyA
-  const float alpha = 1.f - ema_decay;                     // > 0 on this path
-  // Eq. 9 over a run of consecutive window positions i_a..i_b as a Horner chain H = sum c_i I_i decay^(i_b - i),
-  // c_0 = 1/alpha (the seed), c_i = 1: the run contributes alpha * decay^(w-1-i_b) * H.  Even and odd columns
-  // of a run are chained separately in decay^2 (one packed FMA per column pair): H = decay * H_even + H_odd.
+  // The temporal weights over a run of consecutive window positions i_a..i_b as a Horner chain
+  // H = sum c_i I_i decay^(i_b - i): the run contributes t_scale * decay^(w-1-i_b) * H.  For Eq. 9 decay = 1 - alpha,
+  // c_0 = 1/alpha (the seed), t_scale = alpha.  Even and odd columns of a run are chained separately in decay^2
+  // (one packed FMA per column pair): H = decay * H_even + H_odd.
   constexpr int kRun = kW < 32 ? kW : 32;                  // columns of one run inside this warpgroup
   const int i_first = (cgp * 32) % kW;
-  const float seed_coef = (i_first == 0) ? 1.f / alpha : 1.f;
-  const float fin_scale = alpha * powf(ema_decay, (float)(kW - 1 - (i_first + kRun - 1))) / (float)kG;
+  const float seed_coef = (i_first == 0) ? a.t_seed_first : 1.f;
+  const float last_coef = (i_first + kRun == kW) ? a.t_seed_last : 1.f;
+  const bool group_max = a.group_max != 0;
+  const float fin_scale = a.t_scale * powf(ema_decay, (float)(kW - 1 - (i_first + kRun - 1))) / (group_max ? 1.f : (float)kG);
   const f32x2 d2 = f2_make(ema_decay * ema_decay, ema_decay * ema_decay);
   const f32x2 nc2 = f2_make(neg_c2, neg_c2), m1 = f2_make(-1.f, -1.f), tiny2 = f2_make(1e-36f, 1e-36f);
-  const f32x2 seed2 = f2_make(seed_coef, 1.f);
+  const f32x2 seed2 = f2_make(seed_coef, 1.f), last2 = f2_make(1.f, last_coef);
+  // the shares of the four warpgroups: every 32 columns are one query head's window when w = 32, several whole
+  // windows when w < 32, half a window when w = 64 and a quarter when w = 128
+  auto join_shares = [group_max](float r0, float r1, float r2, float r3) {
+    if (!group_max || kW == 128) return (r0 + r1) + (r2 + r3);
+    if (kW == 64) return fmaxf(r0 + r1, r2 + r3);
+    return fmaxf(fmaxf(r0, r1), fmaxf(r2, r3));
+  };
   const float* O_head = a.O_f32 + (long long)bh * kRows * kHeadDim;
   const __nv_bfloat16* V_head = a.V + (long long)b * a.vsb + (long long)h * a.vsh;
   const float* vn_head = a.vnorm + (long long)bh * a.n_kv;
@@ -764,8 +779,9 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
     const int s = it & 1;
     const uint32_t par = (uint32_t)(it >> 1) & 1u;
     float vn = vn_next;
-    bool tile_heavy = __any_sync(0xffffffffu, tm_next[0] > m2r[0] || tm_next[1] > m2r[1] ||
-                                                  tm_next[2] > m2r[2] || tm_next[3] > m2r[3]);
+    // only Eq. 7 has the factor 1 / (1 - A) and the distance that need the exact form near A = 1
+    const bool tile_heavy = kInd == 0 && __any_sync(0xffffffffu, tm_next[0] > m2r[0] || tm_next[1] > m2r[1] ||
+                                                                     tm_next[2] > m2r[2] || tm_next[3] > m2r[3]);
     if (from_lse) {
       ok = ok && mbar_wait(&B->vn_full[it & 3], (uint32_t)(it >> 2) & 1u, abort_flag, dev_status, kDevTimeout, a.wait_limit);
       const int jv = (tile0 + T - 1 - it) * kTile + t;
@@ -784,7 +800,7 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
       const int rs = (it - 1) & 3;
       ok = ok && mbar_wait(&B->red_full[rs], (uint32_t)((it - 1) >> 2) & 1u, abort_flag, dev_status, kDevTimeout, a.wait_limit);
       const int jp = (tile0 + T - it) * kTile + t;
-      if (ok && jp < n) I_head[jp] = (red[rs][0][t] + red[rs][1][t]) + (red[rs][2][t] + red[rs][3][t]);
+      if (ok && jp < n) I_head[jp] = join_shares(red[rs][0][t], red[rs][1][t], red[rs][2][t], red[rs][3][t]);
     }
     ok = ok && mbar_wait(&B->acc_full[s], par, abort_flag, dev_status, kDevTimeout, a.wait_limit);
     float tot = 0.f;
@@ -796,14 +812,16 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
       // the sum positive when the expansion cancels, so that no clamp is needed.
       const float vnb = vn * 1.0000152587890625f;
       const f32x2 vn2 = f2_make(vnb, vnb);
+      const float vlen = kInd == 2 ? sqrtf(vn) : 1.f;          // ||v_j||
+      const f32x2 vlen2 = f2_make(vlen, vlen);
       f32x2 h2 = f2_make(0.f, 0.f);
       float sv0[16], cv0[16], sv1[16], cv1[16];
       if (!tile_heavy) {
         tmem_ld16(tS, sv0);
-        tmem_ld16(tC, cv0);
+        if (kInd == 0) tmem_ld16(tC, cv0);
         tmem_wait_ld();
         tmem_ld16(tS + 16, sv1);   // the second half of the columns travels while the first is worked on
-        tmem_ld16(tC + 16, cv1);
+        if (kInd == 0) tmem_ld16(tC + 16, cv1);
       }
       bool redo_heavy = false;   // from_lse: this warp found a weight above kHeavyA among the logits it holds
       if (!tile_heavy) {
@@ -817,7 +835,7 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&B->acc_empty[s]);
-            if (from_lse) {
+            if (from_lse && kInd == 0) {
               // no pass 1 has flagged the tiles with large weights: the warp looks at the logits it now holds in
               // registers (S' above heavy_thr <=> A > kHeavyA) and, if it finds one, does its part of the tile again
               // below with exact distances, from those registers (the accumulators are already released)
@@ -831,19 +849,27 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
             const f32x2 nt = f2_mul(f2_make(sv[2 * q], sv[2 * q + 1]), nc2);
-            const f32x2 um = f2_add(f2_make(ex2_approx(f2_lo(nt)), ex2_approx(f2_hi(nt))), m1);   // 1/A - 1
-            const f32x2 x = f2_add(f2_make(cv[2 * q], cv[2 * q + 1]), vn2);                       // ||o - v||^2
-            const f32x2 bq = f2_fma(f2_mul(x, um), um, tiny2);                                    // x (1/A - 1)^2
-            f32x2 Iq = f2_mul(x, f2_make(rsqrt_approx(f2_lo(bq)), rsqrt_approx(f2_hi(bq))));
+            f32x2 Iq;
+            if (kInd == 0) {
+              const f32x2 um = f2_add(f2_make(ex2_approx(f2_lo(nt)), ex2_approx(f2_hi(nt))), m1);   // 1/A - 1
+              const f32x2 x = f2_add(f2_make(cv[2 * q], cv[2 * q + 1]), vn2);                       // ||o - v||^2
+              const f32x2 bq = f2_fma(f2_mul(x, um), um, tiny2);                                    // x (1/A - 1)^2
+              Iq = f2_mul(x, f2_make(rsqrt_approx(f2_lo(bq)), rsqrt_approx(f2_hi(bq))));
+            } else {
+              Iq = f2_make(ex2_approx(-f2_lo(nt)), ex2_approx(-f2_hi(nt)));                         // A
+              if (kInd == 2) Iq = f2_mul(Iq, vlen2);
+            }
             if (q == 0 && (c * 16) % kRun == 0) Iq = f2_mul(Iq, seed2);
+            if (q == 7 && (c * 16 + 16) % kRun == 0) Iq = f2_mul(Iq, last2);
             h2 = f2_fma(h2, d2, Iq);
           }
           if ((c * 16 + 16) % kRun == 0) {   // end of a run
-            tot += fmaf(f2_lo(h2), ema_decay, f2_hi(h2));
+            const float run = fmaf(f2_lo(h2), ema_decay, f2_hi(h2));
+            tot = group_max ? fmaxf(tot, run) : tot + run;
             h2 = f2_make(0.f, 0.f);
           }
         }
-        if (from_lse && redo_heavy) {
+        if (from_lse && kInd == 0 && redo_heavy) {
           tot = 0.f;
           h2 = f2_make(0.f, 0.f);
 #pragma unroll
@@ -867,10 +893,12 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
               I[u] = x * rsqrt_approx(fmaf(x * um, um, 1e-36f));
             }
             if ((c * 8) % kRun == 0) I[0] *= seed_coef;
+            if ((c * 8 + 8) % kRun == 0) I[7] *= last_coef;
 #pragma unroll
             for (int q = 0; q < 4; ++q) h2 = f2_fma(h2, d2, f2_make(I[2 * q], I[2 * q + 1]));
             if ((c * 8 + 8) % kRun == 0) {   // end of a run
-              tot += fmaf(f2_lo(h2), ema_decay, f2_hi(h2));
+              const float run = fmaf(f2_lo(h2), ema_decay, f2_hi(h2));
+              tot = group_max ? fmaxf(tot, run) : tot + run;
               h2 = f2_make(0.f, 0.f);
             }
           }
@@ -900,10 +928,12 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
             I[u] = x * rsqrt_approx(fmaf(x * um, um, 1e-36f));
           }
           if ((c * 8) % kRun == 0) I[0] *= seed_coef;
+          if ((c * 8 + 8) % kRun == 0) I[7] *= last_coef;
 #pragma unroll
           for (int q = 0; q < 4; ++q) h2 = f2_fma(h2, d2, f2_make(I[2 * q], I[2 * q + 1]));
           if ((c * 8 + 8) % kRun == 0) {   // end of a run
-            tot += fmaf(f2_lo(h2), ema_decay, f2_hi(h2));
+            const float run = fmaf(f2_lo(h2), ema_decay, f2_hi(h2));
+            tot = group_max ? fmaxf(tot, run) : tot + run;
             h2 = f2_make(0.f, 0.f);
           }
         }
@@ -923,7 +953,7 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
     const int rs = (T - 1) & 3;
     ok = ok && mbar_wait(&B->red_full[rs], (uint32_t)((T - 1) >> 2) & 1u, abort_flag, dev_status, kDevTimeout, a.wait_limit);
     const int jl = tile0 * kTile + t;   // the last tile processed is the first of the share
-    if (ok && jl < n) I_head[jl] = (red[rs][0][t] + red[rs][1][t]) + (red[rs][2][t] + red[rs][3][t]);
+    if (ok && jl < n) I_head[jl] = join_shares(red[rs][0][t], red[rs][1][t], red[rs][2][t], red[rs][3][t]);
   }
 }
 
@@ -996,8 +1026,13 @@ __device__ bool select_worker(const Ctx& cx, const FusedArgs& a, const Plan& pl,
         const long long a64 = (long long)j - half + gamma, b64 = (long long)j + half + gamma;
         const int ta = a64 < s_lo ? s_lo : (int)(a64 <= s_hi ? a64 : s_hi + 1), tb = b64 > s_hi ? s_hi : (int)(b64 >= s_lo ? b64 : s_lo - 1);
         float acc = 0.f;
-        for (int t = ta; t <= tb; ++t) acc += staged[t - s_lo];
-        out = acc / fw;
+        if (a.pool_max) {   // Appendix G.2: maximum over the box, taps outside the scored rows count as 0
+          for (int t = ta; t <= tb; ++t) acc = fmaxf(acc, staged[t - s_lo]);
+          out = acc;
+        } else {
+          for (int t = ta; t <= tb; ++t) acc += staged[t - s_lo];
+          out = acc / fw;
+        }
       }
       srow[jj] = out;
       keys[jj] = sel_key(out);
@@ -1237,14 +1272,14 @@ __device__ void control_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, 
 }
 
 // Warps 4-19: softmax in phase A, the merge of the partials in phase B, the indicator epilogue in phase C.
-template <int kW, bool kLse>
+template <int kW, bool kLse, int kInd>
 __device__ void worker_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, const CUtensorMap* tmQ,
                             const CUtensorMap* tmK, const CUtensorMap* tmV, const CUtensorMap* tmO,
                             const CUtensorMap* tmAug, int* go, float (*red)[4][kTile]) {
   for (int bh = pl.group; bh < a.BH; bh += a.groups) {
     if (bh != pl.group) __syncthreads();
     if (kLse) {
-      phase_c_worker<kW, kLse>(cx, a, tmO, tmAug, tmK, tmV, bh, pl.tile0, pl.T2, 0, red);
+      phase_c_worker<kW, kLse, kInd>(cx, a, tmO, tmAug, tmK, tmV, bh, pl.tile0, pl.T2, 0, red);
       tc_fence_before();
       __syncthreads();
       tc_fence_after();
@@ -1273,7 +1308,7 @@ __device__ void worker_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, c
     }
     if (!group_barrier_follow(go)) break;
     tc_fence_after();
-    phase_c_worker<kW, kLse>(cx, a, tmO, tmAug, tmK, tmV, bh, pl.tile0, pl.T2, 0, red);
+    phase_c_worker<kW, kLse, kInd>(cx, a, tmO, tmAug, tmK, tmV, bh, pl.tile0, pl.T2, 0, red);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -1285,7 +1320,7 @@ __device__ void worker_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, c
 }
 
 // ------------------------------------------------------------------------------------------------
-template <int kW, bool kLse>
+template <int kW, bool kLse, int kInd>
 __global__ void __launch_bounds__(kFThreads, 1)
 tc_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -1348,7 +1383,7 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     control_main<kW, kLse>(cx, a, pl, &tmQ, &tmK, &tmV, &tmO, &tmAug, &bars, &abort_flag, &go_flag);
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kFRegsWorker));
-    worker_main<kW, kLse>(cx, a, pl, &tmQ, &tmK, &tmV, &tmO, &tmAug, &go_flag, red);
+    worker_main<kW, kLse, kInd>(cx, a, pl, &tmQ, &tmK, &tmV, &tmO, &tmAug, &go_flag, red);
   }
 
   tc_fence_before();
@@ -1476,21 +1511,72 @@ static cudaError_t check_launch_regs(K kernel) {
   return fa.numRegs == kFRegsLaunch ? cudaSuccess : cudaErrorInvalidConfiguration;
 }
 
+using FusedKernel = void (*)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, FusedArgs);
+
+template <int kW>
+static FusedKernel pick_fused_w(bool from_lse, int indicator) {
+  if (from_lse) {
+    if (indicator == 0) return tc_fused_kernel<kW, true, 0>;
+    return indicator == 1 ? tc_fused_kernel<kW, true, 1> : tc_fused_kernel<kW, true, 2>;
+  }
+  if (indicator == 0) return tc_fused_kernel<kW, false, 0>;
+  return indicator == 1 ? tc_fused_kernel<kW, false, 1> : tc_fused_kernel<kW, false, 2>;
+}
+
+// The instantiation for a window length (it only matters to phase C), input form and indicator; null if there is none.
+static FusedKernel pick_fused(int w, bool from_lse, int indicator) {
+  if (indicator < 0 || indicator > 2) return nullptr;
+  switch (w) {
+    case 16: return pick_fused_w<16>(from_lse, indicator);
+    case 32: return pick_fused_w<32>(from_lse, indicator);
+    case 64: return pick_fused_w<64>(from_lse, indicator);
+    case 128: return pick_fused_w<128>(from_lse, indicator);
+    default: return nullptr;
+  }
+}
+
 cudaError_t tc_fused_init() {
   cudaError_t e = cudaSuccess;
-  auto prepare = [&](auto kernel) {
-    if (e == cudaSuccess) e = check_launch_regs(kernel);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmem);
-  };
-  prepare(tc_fused_kernel<16, false>);
-  prepare(tc_fused_kernel<32, false>);
-  prepare(tc_fused_kernel<64, false>);
-  prepare(tc_fused_kernel<128, false>);
-  prepare(tc_fused_kernel<16, true>);
-  prepare(tc_fused_kernel<32, true>);
-  prepare(tc_fused_kernel<64, true>);
-  prepare(tc_fused_kernel<128, true>);
+  const int widths[4] = {16, 32, 64, 128};
+  for (int w : widths)
+    for (int lse = 0; lse < 2; ++lse)
+      for (int ind = 0; ind < 3; ++ind) {
+        FusedKernel kernel = pick_fused(w, lse != 0, ind);
+        if (e == cudaSuccess) e = check_launch_regs(kernel);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmem);
+      }
   return e;
+}
+
+// Temporal weights of the variant as the kernel's Horner chain (see FusedArgs).  False when the chain cannot carry
+// them in fp32: Eq. 9 with alpha = 0, or the inverted EMA when its growth factor (1 / decay)^(w-1) is too large.
+static bool temporal_chain(int mode, float ema_decay, int w, float* decay, float* seed_first, float* seed_last,
+                           float* scale) {
+  const float alpha = 1.f - ema_decay;
+  *seed_first = 1.f; *seed_last = 1.f;
+  switch (mode) {
+    case RESTKV_TEMPORAL_EMA:        // weights alpha * d^(w-1-i), d^(w-1) for the oldest query
+      if (!(alpha > 0.f)) return false;
+      *decay = ema_decay; *seed_first = 1.f / alpha; *scale = alpha;
+      return true;
+    case RESTKV_TEMPORAL_MEAN:
+      *decay = 1.f; *scale = 1.f / (float)w;
+      return true;
+    case RESTKV_TEMPORAL_NONE:       // the newest query alone
+      *decay = 0.f; *scale = 1.f;
+      return true;
+    case RESTKV_TEMPORAL_INV_EMA:    // weights alpha * d^i, d^(w-1) for the newest query: a chain in 1 / d
+      if (!(alpha > 0.f) || !(ema_decay > 0.f)) return false;
+      if ((float)(w - 1) * log2f(1.f / ema_decay) > 40.f) return false;
+      *decay = 1.f / ema_decay; *seed_last = 1.f / alpha; *scale = alpha * powf(ema_decay, (float)(w - 1));
+      return true;
+    default: return false;
+  }
+}
+
+bool tc_variant_supported(const Problem& p, float ema_decay) {
+  float d, sf, sl, sc;
+  return temporal_chain(p.temporal, ema_decay, p.w, &d, &sf, &sl, &sc);
 }
 
 // One launch for pass 1, the merge and pass 2 of every head.  The CTAs of a group wait for one another, so all of
@@ -1509,7 +1595,14 @@ cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, 
     return cudaErrorInvalidValue;
   FusedArgs a{};
   a.Hkv = p.Hkv; a.BH = p.BH; a.n = p.n; a.n_kv = p.n_kv; a.w = p.w;
-  a.scale = p.scale; a.ema_decay = ema_decay;
+  a.scale = p.scale;
+  if (attention_only) {
+    a.t_decay = 0.f; a.t_seed_first = a.t_seed_last = a.t_scale = 1.f;
+  } else if (!temporal_chain(p.temporal, ema_decay, p.w, &a.t_decay, &a.t_seed_first, &a.t_seed_last, &a.t_scale)) {
+    return cudaErrorInvalidValue;
+  }
+  a.group_max = p.group == RESTKV_GROUP_MAX ? 1 : 0;
+  a.pool_max = p.spatial == RESTKV_SPATIAL_MAX ? 1 : 0;
   a.attention_only = attention_only ? 1 : 0;
   a.from_lse = O_given ? 1 : 0;
   fused_plan(p, sm_count, reuse_l2, &a.groups, &a.cpg);
@@ -1531,25 +1624,9 @@ cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, 
     if (e != cudaSuccess) return e;
   }
   const dim3 grid(a.groups * a.cpg), block(kFThreads);
-  switch (attention_only ? 32 : p.w) {   // the window length only matters to phase C
-    case 16:
-      if (a.from_lse) tc_fused_kernel<16, true><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a);
-      else tc_fused_kernel<16, false><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a);
-      break;
-    case 32:
-      if (a.from_lse) tc_fused_kernel<32, true><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a);
-      else tc_fused_kernel<32, false><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a);
-      break;
-    case 64:
-      if (a.from_lse) tc_fused_kernel<64, true><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a);
-      else tc_fused_kernel<64, false><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a);
-      break;
-    case 128:
-      if (a.from_lse) tc_fused_kernel<128, true><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a);
-      else tc_fused_kernel<128, false><<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a);
-      break;
-    default: return cudaErrorInvalidValue;
-  }
+  FusedKernel kernel = attention_only ? pick_fused(32, false, 0) : pick_fused(p.w, a.from_lse != 0, p.indicator);
+  if (!kernel) return cudaErrorInvalidValue;
+  kernel<<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a);
   return cudaGetLastError();
 }
 

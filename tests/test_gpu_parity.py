@@ -561,6 +561,183 @@ def test_score_from_lse_at_full_size(handle):
     assert_compaction_exact(idx, vbits, run._bits(run.V_out))
 
 
+# ------------------------------------------------------------------ ablation variants (Appendix G)
+REC, ATT, ATTV = rk.INDICATOR_RECONSTRUCTION, rk.INDICATOR_ATTENTION, rk.INDICATOR_ATTENTION_VNORM
+EMA, MEAN, INV, NONE = rk.TEMPORAL_EMA, rk.TEMPORAL_MEAN, rk.TEMPORAL_INV_EMA, rk.TEMPORAL_NONE
+VARIANTS = [
+    # (indicator, temporal, spatial, group)
+    (ATT, MEAN, rk.SPATIAL_MEAN, rk.GROUP_MEAN),     # window mean of the attention weights, pooled
+    (ATTV, EMA, rk.SPATIAL_MEAN, rk.GROUP_MEAN),
+    (REC, INV, rk.SPATIAL_MEAN, rk.GROUP_MEAN),
+    (REC, NONE, rk.SPATIAL_MAX, rk.GROUP_MEAN),
+    (REC, MEAN, rk.SPATIAL_MEAN, rk.GROUP_MAX),
+    (ATT, INV, rk.SPATIAL_MAX, rk.GROUP_MAX),
+    (ATTV, NONE, rk.SPATIAL_MEAN, rk.GROUP_MAX),
+    (REC, EMA, rk.SPATIAL_MAX, rk.GROUP_MAX),
+]
+
+
+def variant_check(handle, inp, variant, path=rk.PATH_AUTO, from_lse=False, ema_decay=None, budget=None, fused=None):
+    """evict (or evict_from_lse) under a variant against the oracle run with the same modes: all three rules."""
+    import torch
+    ind, tmp, spa, grp = variant
+    c = inp.case
+    decay = c.ema_decay if ema_decay is None else ema_decay
+    handle.set_kernel_path(path)
+    handle.set_variant(ind, tmp, spa, grp)
+    try:
+        run = GpuRun(handle, inp, budget=budget)
+        if from_lse:
+            _, O, lse = _window_stats(inp, with_A_check=False)
+            handle.evict_from_lse(run.shape, run.Q, run.K, run.V, torch.from_numpy(O).cuda(),
+                                  torch.from_numpy(lse).cuda(), decay, run.pool(), run.budget, run.indices,
+                                  run.K_out, run.V_out, run.ws, scores_out=run.scores)
+        else:
+            handle.evict(run.shape, run.Q, run.K, run.V, decay, run.pool(), run.budget, run.indices, run.K_out,
+                         run.V_out, run.ws, scores_out=run.scores)
+        torch.cuda.synchronize()
+        assert handle.poll_status() == rk.RESTKV_OK
+        if fused is not None:
+            assert handle.last_evict_fused_select() == fused
+    finally:
+        handle.set_kernel_path(rk.PATH_AUTO)
+        handle.set_variant()
+    ref = oracle_scores(inp, ema_decay=decay, indicator_mode=ind, temporal_mode=tmp, spatial_mode=spa, group_mode=grp)
+    tol = TOL[c.dtype]
+    idx = run.indices.cpu().numpy()
+    assert_scores_close(run.scores.cpu().numpy(), ref.scores, tol)
+    assert_selection_valid(idx, ref.scores, run.budget, tol)
+    _, kbits, vbits = inp.device_arrays()
+    assert_compaction_exact(idx, kbits, run._bits(run.K_out))
+    assert_compaction_exact(idx, vbits, run._bits(run.V_out))
+    return ref
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("spec", [("cfg1b", "f32", 0), ("cfg1b", "bf16", 32)])
+def test_variants_on_the_simt_kernels(handle, variant, spec):
+    name, dtype, tail = spec
+    variant_check(handle, make_inputs(CONFIGS[name].with_(dtype=dtype, causal_tail=tail)), variant)
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("tail", [0, 32])
+def test_variants_on_the_tensor_core_kernel(handle, variant, tail):
+    # cfg2 qualifies for the selection inside the score kernel, so its max-pooling is covered here too
+    inp = make_inputs(CONFIGS["cfg2"].with_(causal_tail=tail))
+    ref = variant_check(handle, inp, variant, path=rk.PATH_TENSOR_CORE, fused=True)
+    # the variant must have changed the scores, or the test compares the default with itself
+    base = oracle_scores(inp).scores
+    fin = np.isfinite(base)
+    assert not np.allclose(ref.scores[fin], base[fin], rtol=1e-3)
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_variants_from_given_window_statistics(handle, variant):
+    variant_check(handle, make_inputs(CONFIGS["cfg2"]), variant, path=rk.PATH_TENSOR_CORE, from_lse=True)
+
+
+@pytest.mark.parametrize("variant", [VARIANTS[0], VARIANTS[4], VARIANTS[5]])
+def test_variants_with_the_selection_as_its_own_kernel(handle, variant):
+    handle.set_fused_select(False)
+    try:
+        variant_check(handle, make_inputs(CONFIGS["cfg2"]), variant, path=rk.PATH_TENSOR_CORE, fused=False)
+    finally:
+        handle.set_fused_select(True)
+
+
+@pytest.mark.parametrize("variant", [VARIANTS[2], VARIANTS[4], VARIANTS[5], VARIANTS[7]])
+@pytest.mark.parametrize("spec", [(16, 2, 16), (4, 2, 64), (2, 2, 128), (8, 1, 16)])
+def test_variants_at_other_window_lengths(handle, variant, spec):
+    """The group reduction and the temporal chain of the tensor-core kernel are laid out differently for each window
+    length (a 32-column slice is two windows, one, half of one or a quarter)."""
+    Hq, Hkv, w = spec
+    case = Case("variant_w%d" % w, 2, Hq, Hkv, 128, 3000, w, 200, 5, 0, 0.9, "bf16", 0, "normal", 55)
+    variant_check(handle, make_inputs(case), variant, path=rk.PATH_TENSOR_CORE)
+
+
+@pytest.mark.parametrize("decay,expect_tc", [(0.9, True), (0.5, True), (0.2, False), (0.0, False), (1.0, False)])
+def test_inverted_ema_leaves_the_tensor_core_kernel_when_its_chain_would_overflow(handle, decay, expect_tc):
+    inp = make_inputs(CONFIGS["cfg2"])
+    variant = (REC, INV, rk.SPATIAL_MEAN, rk.GROUP_MEAN)
+    variant_check(handle, inp, variant, ema_decay=decay)            # automatic choice: always served
+    if not expect_tc:
+        handle.set_kernel_path(rk.PATH_TENSOR_CORE)
+        handle.set_variant(*variant)
+        try:
+            run = GpuRun(handle, inp)
+            with pytest.raises(rk.RestKVError) as e:
+                handle.evict(run.shape, run.Q, run.K, run.V, decay, run.pool(), run.budget, run.indices, run.K_out,
+                             run.V_out, run.ws)
+            assert e.value.status == rk.ERR_UNSUPPORTED
+        finally:
+            handle.set_kernel_path(rk.PATH_AUTO)
+            handle.set_variant()
+    else:
+        variant_check(handle, inp, variant, path=rk.PATH_TENSOR_CORE, ema_decay=decay)
+
+
+@pytest.mark.parametrize("variant", [VARIANTS[0], VARIANTS[5], VARIANTS[1]])
+def test_variants_with_the_adaptive_window(handle, variant):
+    ind, tmp, spa, grp = variant
+    inp = make_inputs(CONFIGS["cfg1b"])
+    c = inp.case
+    B = c.budget
+    modes = dict(indicator_mode=ind, temporal_mode=tmp, spatial_mode=spa, group_mode=grp)
+    probe = oracle_scores(inp, pool_mode=1, beta=1e9, base_width=1, budget=B, **modes)
+    delta = abs(probe.D[..., 0] - probe.D[..., 1]).min()
+    assert delta > 0
+    compared = 0
+    for target, base in ((0.5, 3), (1.5, 1), (2.5, 3)):
+        beta = float(delta / target)
+        ref = oracle_scores(inp, pool_mode=1, beta=beta, base_width=base, budget=B, **modes)
+        x = (ref.D[..., 0] - ref.D[..., 1]) / beta
+        if np.any(np.abs(x - np.round(x)) < 0.05):
+            continue   # too close to a rounding boundary for an fp32-vs-fp64 ranking comparison
+        handle.set_variant(ind, tmp, spa, grp)
+        try:
+            run = GpuRun(handle, inp, adaptive_budget=B)
+            scores = run.score(pool=rk.adaptive_pool(beta, base, B))
+        finally:
+            handle.set_variant()
+        np.testing.assert_array_equal(run.pool_used.cpu().numpy(), ref.pool)
+        assert_scores_close(scores, ref.scores, TOL[c.dtype])
+        compared += 1
+    assert compared > 0, "every beta landed on a rounding boundary: nothing was compared"
+
+
+def test_variants_score_a_single_row_cache(handle):
+    # Eq. 7 is 0/0 on a cache of one row (defined as 0); the attention-weight indicators are 1 and ||v|| there
+    case = Case("one_row", 1, 4, 2, 64, 1, 4, 1, 1, 0, 0.7, "f32", 0, "normal", 5)
+    inp = make_inputs(case)
+    for ind, expect in ((REC, None), (ATT, 1.0), (ATTV, None)):
+        handle.set_variant(ind)
+        try:
+            got = GpuRun(handle, inp).score()
+        finally:
+            handle.set_variant()
+        ref = oracle.score(inp.Q, inp.K, inp.V, ema_decay=case.ema_decay, width=1, indicator_mode=ind).scores
+        np.testing.assert_allclose(got, ref, rtol=1e-6, atol=0)
+        if expect is not None:
+            np.testing.assert_allclose(got, expect, rtol=1e-6)
+    assert np.all(oracle.score(inp.Q, inp.K, inp.V, width=1).scores == 0.0)
+
+
+def test_variant_at_full_size(handle):
+    """The long-context workload under two variants, in the launch configuration the benchmark times."""
+    inp = make_inputs(CONFIGS["cfg4"])
+    variant_check(handle, inp, VARIANTS[0], fused=True)
+    variant_check(handle, inp, VARIANTS[5], fused=True)
+
+
+def test_set_variant_validates_its_fields(handle):
+    for bad in ((3, 0, 0, 0), (0, 4, 0, 0), (0, 0, 2, 0), (0, 0, 0, 2), (-1, 0, 0, 0)):
+        with pytest.raises(rk.RestKVError) as e:
+            handle.set_variant(*bad)
+        assert e.value.status == rk.ERR_INVALID_ARG
+    handle.set_variant()
+
+
 # ------------------------------------------------------------------ a device-side wait that runs out
 def test_wait_limit_runs_out_and_the_handle_recovers(handle):
     """With a wait limit of one SM clock the first CTA to reach a group barrier of the persistent score kernel gives
