@@ -476,6 +476,36 @@ def main():
             assert handle.poll_status() == rk.RESTKV_OK
             variants["evict_ms"][label] = float(np.median(tv))
 
+    # ---- the adaptive window of Eq. 10-12 (per-query top-B of the raw indicator, D_front / D_rear) ----
+    adaptive = None
+    if rank == 0:
+        apool = rk.adaptive_pool(2000.0, case.width, case.budget)
+        ws_a = torch.empty(handle.workspace_bytes(shape, case.budget, adaptive=True), dtype=torch.uint8, device="cuda")
+
+        def time_adaptive(path, reps):
+            handle.set_kernel_path(path)
+            try:
+                ta = []
+                for it in range(reps + 2):
+                    flush.zero_()
+                    ev0.record()
+                    handle.evict(shape, Q, K, V, case.ema_decay, apool, case.budget, indices, K_out, V_out, ws_a)
+                    ev1.record()
+                    torch.cuda.synchronize()
+                    if it >= 2:
+                        ta.append(ev0.elapsed_time(ev1))
+            finally:
+                handle.set_kernel_path(rk.PATH_AUTO)
+            assert handle.poll_status() == rk.RESTKV_OK
+            return float(np.median(ta))
+
+        adaptive = {"note": "restkv_evict with the adaptive window (beta 2000, B = the budget): the score kernel also "
+                            "writes the per-query indicators [b, Hq, w, n] fp32, from which %d rows of top-B are taken"
+                            % (case.batch * case.n_q_heads * case.w),
+                    "evict_ms": time_adaptive(rk.PATH_AUTO, 5), "evict_ms_simt_kernels": time_adaptive(rk.PATH_SIMT, 2),
+                    "raw_indicator_bytes": 4 * case.batch * case.n_q_heads * case.w * case.n}
+        del ws_a
+
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----
     e2e = None
     if not args.no_e2e:
@@ -548,7 +578,7 @@ def main():
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roofline, "path_roofline": path_roofline, "kernels_ms": kmean,
         "kernels_ms_selection_as_own_kernel": kmean_split, "decode": decode, "from_lse": from_lse,
-        "variants": variants,
+        "variants": variants, "adaptive_window": adaptive,
     }
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(inp, case.budget)

@@ -202,7 +202,10 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
   const bool adaptive = pool->mode == RESTKV_POOL_ADAPTIVE;
   // the tensor-core pass 2 carries the temporal weights as an fp32 Horner chain, which Eq. 9 with alpha = 0 and
   // some inverted EMAs do not fit: those run on the SIMT kernels
-  bool use_tc = tc_supported(p) && c.h->tc_state != nullptr && !adaptive && tc_variant_supported(p, ema_decay);
+  // (the adaptive window needs the per-query indicators, which the tensor-core kernel writes out only when it runs
+  // pass 1 itself)
+  bool use_tc = tc_supported(p) && c.h->tc_state != nullptr && !(adaptive && O_given) &&
+                tc_variant_supported(p, ema_decay);
   if (p.n_kv == 1 && p.indicator != RESTKV_INDICATOR_RECONSTRUCTION) use_tc = false;
   if (c.h->kernel_path == 1) use_tc = false;
   if (c.h->kernel_path >= 2 && !use_tc) return RESTKV_ERR_UNSUPPORTED;
@@ -222,7 +225,7 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
                             tc_fused_select_supported(p, c.h->sm_count, false, sel->keep, sel->W, sel->gamma);
       RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2,
                     launch_tc_fused(c.h->tc_state, p, ws, Q, K, V, ema_decay, c.h->sm_count, false, false,
-                                    c.h->wait_limit, with_sel ? sel : nullptr, O_given, c.h->dev_status, c.st), 1);
+                                    c.h->wait_limit, with_sel ? sel : nullptr, O_given, nullptr, c.h->dev_status, c.st), 1);
       if (sel_done) *sel_done = with_sel;
     } else {
       Workspace wsl = ws;
@@ -238,7 +241,8 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
                           tc_fused_select_supported(p, c.h->sm_count, reuse_l2, sel->keep, sel->W, sel->gamma);
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2,
                   launch_tc_fused(c.h->tc_state, p, ws, Q, K, V, ema_decay, c.h->sm_count, reuse_l2, false,
-                                  c.h->wait_limit, with_sel ? sel : nullptr, nullptr, c.h->dev_status, c.st), 1);
+                                  c.h->wait_limit, with_sel ? sel : nullptr, nullptr, adaptive ? ws.I_raw : nullptr,
+                                  c.h->dev_status, c.st), 1);
     if (sel_done) *sel_done = with_sel;
   } else {
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS1, launch_simt_pass1(p, ws, Q, K, V, c.st), 1);
@@ -532,7 +536,7 @@ restkv_status restkv_decode(restkv_handle* h, const restkv_shape* shape, const v
       RESTKV_LAUNCH(c, RESTKV_KERNEL_NONE, launch_decode_pad(p, q, ws.q_pad, c.st), 1);
       RESTKV_LAUNCH(c, RESTKV_KERNEL_NONE,
                     launch_tc_fused(h->tc_state, pd, ws, ws.q_pad, Kc, Vc, 0.f, h->sm_count, false, true, h->wait_limit,
-                                    nullptr, nullptr, h->dev_status, c.st), 1);
+                                    nullptr, nullptr, nullptr, h->dev_status, c.st), 1);
       RESTKV_LAUNCH(c, RESTKV_KERNEL_NONE, launch_decode_extract(p, ws.O_f32, ws.row_M2, out, lse, c.st), 1);
       return RESTKV_OK;
     }

@@ -93,8 +93,8 @@ cudaError_t tc_init(void** state);   // resolves the driver entry point for tens
 cudaError_t tc_fused_init();
 cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
                             const void* V, float ema_decay, int sm_count, bool reuse_l2, bool attention_only,
-                            long long wait_limit, const FusedSelect* sel, const float* O_given, unsigned int* dev_status,
-                            cudaStream_t st);
+                            long long wait_limit, const FusedSelect* sel, const float* O_given, float* I_raw,
+                            unsigned int* dev_status, cudaStream_t st);
 // Given the window rows' outputs O [BH, R, d] and log-sum-exps LSE [BH, R] (natural log): what the score kernels read
 // instead of the results of pass 1 and the merge.  tensor_core: -2 bf16(O), the constant strip, the rows' log2
 // normalisers; otherwise fin_m = LSE, fin_l = 1.

@@ -52,6 +52,8 @@ struct FusedArgs {
   float* tile_max;                   // [BH, tiles, 128] largest scaled logit (log2 units) of each query row in each tile
   float* row_M2;                     // [BH, 128] m*log2e + log2 l of each query row (written by the merge)
   float* I_hat;                      // [BH, n]
+  float* I_raw;                      // [BH, 128, n] or null: the per-query indicators, for the adaptive window of
+                                     //  Eq. 10-12; every tile then takes the slower epilogue that holds them
   const __nv_bfloat16* V;
   long long vsb, vsh, vsn;
   unsigned int* counters;            // [groups] (at most 256), zero at launch
@@ -753,6 +755,7 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
   const __nv_bfloat16* V_head = a.V + (long long)b * a.vsb + (long long)h * a.vsh;
   const float* vn_head = a.vnorm + (long long)bh * a.n_kv;
   float* I_head = a.I_hat + (long long)bh * n;
+  float* raw_head = (a.I_raw && !kLse) ? a.I_raw + (long long)bh * kRows * n : nullptr;
   bool ok = true;
   const int nt_all = (a.n_kv + kTile - 1) / kTile;
   // a tile needs exact distances iff some row's largest logit in it reaches that row's M2 - log2(1 / kHeavyA);
@@ -780,8 +783,9 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
     const uint32_t par = (uint32_t)(it >> 1) & 1u;
     float vn = vn_next;
     // only Eq. 7 has the factor 1 / (1 - A) and the distance that need the exact form near A = 1
-    const bool tile_heavy = kInd == 0 && __any_sync(0xffffffffu, tm_next[0] > m2r[0] || tm_next[1] > m2r[1] ||
-                                                                     tm_next[2] > m2r[2] || tm_next[3] > m2r[3]);
+    const bool tile_heavy = raw_head != nullptr ||
+                            (kInd == 0 && __any_sync(0xffffffffu, tm_next[0] > m2r[0] || tm_next[1] > m2r[1] ||
+                                                                      tm_next[2] > m2r[2] || tm_next[3] > m2r[3]));
     if (from_lse) {
       ok = ok && mbar_wait(&B->vn_full[it & 3], (uint32_t)(it >> 2) & 1u, abort_flag, dev_status, kDevTimeout, a.wait_limit);
       const int jv = (tile0 + T - 1 - it) * kTile + t;
@@ -904,7 +908,8 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
           }
         }
       } else {
-        // rare: the tile may hold large attention weights; those entries take the exact distance
+        // rare: the tile may hold large attention weights; those entries take the exact distance.  Also the
+        // epilogue of every tile when the per-query indicators are wanted.
 #pragma unroll 1
         for (int c = 0; c < 4; ++c) {
           float sv[8], cv[8], I[8];
@@ -913,19 +918,27 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
           tmem_wait_ld();
 #pragma unroll
           for (int u = 0; u < 8; ++u) {
-            const float um = ex2_approx(sv[u] * neg_c2) - 1.f;
-            float x = cv[u] + vnb;
-            // the whole warp computes the exact distance of each of its lanes' heavy entries in turn
-            unsigned int todo = __ballot_sync(0xffffffffu, sv[u] > heavy_thr && j < n);
-            while (todo) {
-              const int src = __ffs(todo) - 1;
-              todo &= todo - 1;
-              const int js = __shfl_sync(0xffffffffu, j, src);
-              const float d2x = exact_dist2_warp(O_head + (cgp * 32 + c * 8 + u) * kHeadDim,
-                                                 V_head + (long long)js * a.vsn, lane);
-              if (lane == src) x = d2x;
+            if (kInd == 0) {
+              const float um = ex2_approx(sv[u] * neg_c2) - 1.f;
+              float x = cv[u] + vnb;
+              // the whole warp computes the exact distance of each of its lanes' heavy entries in turn
+              unsigned int todo = __ballot_sync(0xffffffffu, sv[u] > heavy_thr && j < n);
+              while (todo) {
+                const int src = __ffs(todo) - 1;
+                todo &= todo - 1;
+                const int js = __shfl_sync(0xffffffffu, j, src);
+                const float d2x = exact_dist2_warp(O_head + (cgp * 32 + c * 8 + u) * kHeadDim,
+                                                   V_head + (long long)js * a.vsn, lane);
+                if (lane == src) x = d2x;
+              }
+              I[u] = x * rsqrt_approx(fmaf(x * um, um, 1e-36f));
+            } else {
+              I[u] = ex2_approx(-sv[u] * neg_c2) * vlen;
             }
-            I[u] = x * rsqrt_approx(fmaf(x * um, um, 1e-36f));
+          }
+          if (raw_head && j < n) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) raw_head[(long long)(cgp * 32 + c * 8 + u) * n + j] = I[u];
           }
           if ((c * 8) % kRun == 0) I[0] *= seed_coef;
           if ((c * 8 + 8) % kRun == 0) I[7] *= last_coef;
@@ -1585,8 +1598,8 @@ bool tc_variant_supported(const Problem& p, float ema_decay) {
 // with the timeout status instead of hanging.  (A cooperative launch would guarantee residency but costs ~25 us.)
 cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, const void* Q, const void* K,
                             const void* V, float ema_decay, int sm_count, bool reuse_l2, bool attention_only,
-                            long long wait_limit, const FusedSelect* sel, const float* O_given, unsigned int* dev_status,
-                            cudaStream_t st) {
+                            long long wait_limit, const FusedSelect* sel, const float* O_given, float* I_raw,
+                            unsigned int* dev_status, cudaStream_t st) {
   TcState* ts = (TcState*)state;
   CUtensorMap tmQ, tmK, tmV, tmO, tmAug;
   if (!make_rows_map(ts, &tmQ, Q, p.BH) || !make_rows_map(ts, &tmO, ws.O_m2, p.BH) ||
@@ -1611,6 +1624,7 @@ cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, 
   a.V = (const __nv_bfloat16*)V; a.vsb = p.vsb; a.vsh = p.vsh; a.vsn = p.vsn;
   a.counters = ws.counters; a.tile_max = ws.tile_max; a.row_M2 = ws.row_M2; a.dev_status = dev_status;
   a.wait_limit = wait_limit;
+  a.I_raw = O_given ? nullptr : I_raw;
   if (O_given) a.O_f32 = const_cast<float*>(O_given);   // read only in this mode
   cudaError_t e = cudaMemsetAsync(ws.counters, 0, 1024, st);
   if (e != cudaSuccess) return e;

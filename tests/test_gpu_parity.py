@@ -122,25 +122,56 @@ def test_head_sequential_kernel_at_full_size(handle):
     full_check(handle, make_inputs(CONFIGS["cfg4"]), path=rk.PATH_HEAD_SEQUENTIAL)
 
 
-def test_config2_adaptive_window(handle):
-    """Eq. 10-12 on the 8B-shaped layer: D_front / D_rear from the per-query top-B, window width and shift."""
-    case = CONFIGS["cfg2"]
-    inp = make_inputs(case)
+def _adaptive_check(handle, inp, path, base=5, evict=False):
+    """Eq. 10-12: D_front / D_rear from the per-query top-B, window width and shift, then the pooled scores; heads
+    whose (D_front - D_rear) / beta lands too close to a rounding boundary are not compared."""
+    case = inp.case
     B = case.budget
     probe = oracle_scores(inp, pool_mode=1, beta=1e9, base_width=1, budget=B)
     delta = abs(probe.D[..., 0] - probe.D[..., 1]).min()
     assert delta > 0
     beta = float(delta / 1.5)                     # (D_front - D_rear) / beta = +-1.5 on the head with the smallest gap
-    ref = oracle_scores(inp, pool_mode=1, beta=beta, base_width=5, budget=B)
+    ref = oracle_scores(inp, pool_mode=1, beta=beta, base_width=base, budget=B)
     x = (ref.D[..., 0] - ref.D[..., 1]) / beta
-    keep = np.abs(x - np.round(x)) >= 0.05        # heads too close to a rounding boundary are not compared
-    run = GpuRun(handle, inp, adaptive_budget=B)
-    scores = run.score(pool=rk.adaptive_pool(beta, 5, B))
-    used = run.pool_used.cpu().numpy()
+    keep = np.abs(x - np.round(x)) >= 0.05
     assert keep.any()
-    np.testing.assert_array_equal(used[keep], ref.pool[keep])
+    handle.set_kernel_path(path)
+    try:
+        run = GpuRun(handle, inp, adaptive_budget=B)
+        pool = rk.adaptive_pool(beta, base, B)
+        if evict:
+            scores, idx, K_out, V_out = run.evict(pool=pool)
+        else:
+            scores = run.score(pool=pool)
+            used = run.pool_used.cpu().numpy()
+            np.testing.assert_array_equal(used[keep], ref.pool[keep])
+    finally:
+        handle.set_kernel_path(rk.PATH_AUTO)
     for b, h in zip(*np.nonzero(keep)):
         assert_scores_close(scores[b, h], ref.scores[b, h], TOL[case.dtype])
+        if evict:
+            assert_selection_valid(idx[b, h], ref.scores[b, h], B, TOL[case.dtype])
+    if evict:
+        _, kbits, vbits = inp.device_arrays()
+        assert_compaction_exact(idx, kbits, K_out)
+        assert_compaction_exact(idx, vbits, V_out)
+    return keep
+
+
+@pytest.mark.parametrize("path", [rk.PATH_TENSOR_CORE, rk.PATH_SIMT])
+def test_config2_adaptive_window(handle, path):
+    _adaptive_check(handle, make_inputs(CONFIGS["cfg2"]), path)
+
+
+@pytest.mark.parametrize("tail", [0, 32])
+def test_config2_adaptive_window_evict_on_the_tensor_core_kernel(handle, tail):
+    _adaptive_check(handle, make_inputs(CONFIGS["cfg2"].with_(causal_tail=tail)), rk.PATH_TENSOR_CORE, evict=True)
+
+
+def test_adaptive_window_at_full_size(handle):
+    """The long-context workload with the adaptive window: 1024 per-query top-B selections over 131072 tokens each."""
+    keep = _adaptive_check(handle, make_inputs(CONFIGS["cfg4"]), rk.PATH_TENSOR_CORE, evict=True)
+    assert keep.sum() >= 4
 
 
 def test_config2_is_deterministic(handle):
