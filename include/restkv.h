@@ -274,9 +274,26 @@ int restkv_last_evict_fused_select(const restkv_handle* h);   /* 1 if the last r
  * that path and for callers that want to fail faster.  The paper has no counterpart. */
 restkv_status restkv_set_wait_limit(restkv_handle* h, long long sm_clocks);
 
+/*
+ * restkv_evict_budgets -- restkv_evict with a budget of its own for every (batch, KV head): what the layer-wise and
+ * head-wise budget allocation strategies of Appendix C hand to the eviction step (the strategies themselves are
+ * not part of this library).
+ *   budgets      device int32 [batch, n_kv_heads]; head r keeps min(max(budgets[r], 1), max_budget, n_kv) rows
+ *   max_budget   >= 1: with S = min(max_budget, n_kv), the row stride of the outputs
+ *   indices      device int32 [batch, n_kv_heads, S]: the kept rows of a head ascending, then -1 up to S
+ *   K_out, V_out device [batch, n_kv_heads, S, head_dim]: rows past a head's count are left untouched
+ *   scores_out, workspace (restkv_workspace_bytes[_adaptive](shape, max_budget)), pool, errors: as restkv_evict.
+ * The selection and the gather run in the cluster select kernel (never inside the score kernel).
+ */
+restkv_status restkv_evict_budgets(restkv_handle* h, const restkv_shape* shape, const void* Q_obs, const void* K,
+                                   const void* V, float ema_decay, const restkv_pool_params* pool,
+                                   const int32_t* budgets, int max_budget, float* scores_out, int32_t* indices,
+                                   void* K_out, void* V_out, void* workspace, size_t workspace_bytes,
+                                   restkv_stream stream);
+
 /* Ablation variants (Appendix G) as modes of the same kernels.  A handle starts with every field 0: the method as
  * Sections 3.2-3.3 define it.  The setting applies to every later restkv_score, restkv_evict, restkv_evict_host,
- * restkv_score_from_lse and restkv_evict_from_lse call through the handle; restkv_select, restkv_compact and the
+ * restkv_score_from_lse, restkv_evict_from_lse and restkv_evict_budgets call through the handle; restkv_select, restkv_compact and the
  * decode calls do not depend on it.
  *   indicator (Appendix G.1, indicator table), per query t and token j:
  *     RECONSTRUCTION  A_t[j] / (1 - A_t[j]) * ||o_t - v_j||_2, Eq. 7

@@ -25,7 +25,7 @@ EXPORTS = [
     "restkv_decode_static_last_cuda_error",
     "restkv_poll_status", "restkv_launch_count", "restkv_last_cuda_error", "restkv_error_string",
     "restkv_set_kernel_path", "restkv_set_profile_events", "restkv_set_wait_limit", "restkv_set_fused_select", "restkv_last_evict_fused_select",
-    "restkv_set_variant",
+    "restkv_set_variant", "restkv_evict_budgets",
 ]
 KERNEL_NONE, KERNEL_PASS1, KERNEL_COMBINE, KERNEL_PASS2, KERNEL_POOL, KERNEL_SELECT, KERNEL_COMPACT = range(7)
 
@@ -91,6 +91,7 @@ def load_library() -> ctypes.CDLL:
     lib.restkv_compact.argtypes = [vp, shp, vp, vp, vp, ci, vp, vp, vp]
     lib.restkv_evict.argtypes = [vp, shp, vp, vp, vp, cf, pool, ci, vp, vp, vp, vp, vp, sz, vp]
     lib.restkv_evict_from_lse.argtypes = [vp, shp, vp, vp, vp, vp, vp, cf, pool, ci, vp, vp, vp, vp, vp, sz, vp]
+    lib.restkv_evict_budgets.argtypes = [vp, shp, vp, vp, vp, cf, pool, vp, ci, vp, vp, vp, vp, vp, sz, vp]
     lib.restkv_evict_host.argtypes = [vp, shp, vp, vp, vp, cf, pool, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.restkv_decode.argtypes = [vp, shp, vp, vp, vp, ci, vp, vp, vp, sz, vp]
     lib.restkv_decode_static.argtypes = [shp, vp, vp, vp, ci, vp, vp, vp]
@@ -215,6 +216,15 @@ class Handle:
                                            _ptr(indices), _ptr(K_out), _ptr(V_out), _ptr(workspace),
                                            workspace.numel() * workspace.element_size(), _stream_ptr(stream)),
                     "restkv_evict")
+
+    def evict_budgets(self, shape, Q_obs, K, V, ema_decay, pool, budgets, max_budget, indices, K_out, V_out,
+                      workspace, scores_out=None, stream=None):
+        self._check(self._lib.restkv_evict_budgets(self._h, ctypes.byref(shape), _ptr(Q_obs), _ptr(K), _ptr(V),
+                                                   float(ema_decay), ctypes.byref(pool), _ptr(budgets),
+                                                   int(max_budget), _ptr(scores_out), _ptr(indices), _ptr(K_out),
+                                                   _ptr(V_out), _ptr(workspace),
+                                                   workspace.numel() * workspace.element_size(), _stream_ptr(stream)),
+                    "restkv_evict_budgets")
 
     def evict_from_lse(self, shape, Q_obs, K, V, O_obs, LSE_obs, ema_decay, pool, budget, indices, K_out, V_out,
                        workspace, scores_out=None, stream=None):

@@ -57,7 +57,7 @@ cudaError_t launch_adaptive_params(const Problem& p, const Workspace& ws, int bu
   if (Bp > p.n) Bp = p.n;
   const int rows = p.batch * p.Hq * p.w;
   *n_launches = 0;
-  cudaError_t e = launch_select(rows, p.n, p.n, Bp, nullptr, nullptr, 1, 0, false, ws.I_raw, ws.adaptive_idx, nullptr, nullptr, nullptr,
+  cudaError_t e = launch_select(rows, p.n, p.n, Bp, nullptr, nullptr, nullptr, 1, 0, false, ws.I_raw, ws.adaptive_idx, nullptr, nullptr, nullptr,
                                 nullptr, nullptr, nullptr, st);
   if (e != cudaSuccess) return e;
   ++*n_launches;

@@ -129,8 +129,10 @@ __device__ __forceinline__ void pool_staged(const float* __restrict__ staged, in
 // the key T of the keep-th largest score and how many scores equal to T are kept; an ordered pass then writes,
 // in ascending index order, every index whose key is > T plus the first kept ones whose key equals T (lower
 // index wins ties).
+// keep_rows non-null: row r keeps min(max(keep_rows[r], 1), keep) entries instead of `keep` (non-uniform budgets);
+// its outputs still have a row stride of `keep`, the unused tail of its indices is set to -1.
 __global__ void __launch_bounds__(kSelThreads, 1)
-select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const int* __restrict__ pool, int W,
+select_kernel(int n, int n_kv, int keep, const int* __restrict__ keep_rows, const float* __restrict__ I_hat, const int* __restrict__ pool, int W,
               int gamma, int pool_max, float* scores, int32_t* __restrict__ indices, int32_t* __restrict__ pool_used,
               int per, int use_smem, int stage_taps, GatherArgs ga) {
   cg::cluster_group cluster = cg::this_cluster();
@@ -149,7 +151,13 @@ select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const 
   const long long j0 = (long long)rank * per;
   const int cnt = (int)max(0ll, min((long long)n_kv, j0 + per) - j0);
   float* srow = scores + (long long)row * n_kv;
-  int32_t* dst = indices + (long long)row * keep;
+  const int out_stride = keep;
+  int32_t* dst = indices + (long long)row * out_stride;
+  if (keep_rows) {
+    keep = min(max(keep_rows[row], 1), out_stride);
+    if (rank == 0)
+      for (int pos = keep + tid; pos < out_stride; pos += kSelThreads) dst[pos] = -1;
+  }
 
   // ---- keys of the slice ----
   if (I_hat) {
@@ -214,7 +222,7 @@ select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const 
         const int chunk = isV ? c - ga.row_chunks : c;
         const long long j = j0 + r;
         const uint4* src = reinterpret_cast<const uint4*>((isV ? Vh + j * ga.vsn * ga.esize : Kh + j * ga.ksn * ga.esize)) + chunk;
-        uint4* out = reinterpret_cast<uint4*>((isV ? ga.V_out : ga.K_out) + ((long long)row * keep + j) * ga.row_chunks * 16) + chunk;
+        uint4* out = reinterpret_cast<uint4*>((isV ? ga.V_out : ga.K_out) + ((long long)row * out_stride + j) * ga.row_chunks * 16) + chunk;
         *out = __ldg(src);
       }
     }
@@ -370,7 +378,7 @@ select_kernel(int n, int n_kv, int keep, const float* __restrict__ I_hat, const 
     const int b = row / ga.Hkv, h = row % ga.Hkv;
     const unsigned char* Kh = ga.K + ((long long)b * ga.ksb + (long long)h * ga.ksh) * ga.esize;
     const unsigned char* Vh = ga.V + ((long long)b * ga.vsb + (long long)h * ga.vsh) * ga.esize;
-    const long long out_row0 = (long long)row * keep;
+    const long long out_row0 = (long long)row * out_stride;
     const int rc2 = 2 * ga.row_chunks;
     // four chunks per thread and round, the index loads first and then the row loads, so that they overlap
     const unsigned int total = mine * (unsigned int)rc2;
@@ -447,7 +455,7 @@ cudaError_t launch_pool(const Problem& p, const Workspace& ws, const int* pool_d
 
 // rows x n_kv scores -> rows x min(budget, n_kv) indices.  I_hat non-null: pool first (n scored rows per row of
 // I_hat, window from pool_dev or (W, gamma)) and write the pooled scores.
-cudaError_t launch_select(int rows, int n, int n_kv, int budget, const float* I_hat, const int* pool_dev, int W,
+cudaError_t launch_select(int rows, int n, int n_kv, int budget, const int* keep_rows, const float* I_hat, const int* pool_dev, int W,
                           int gamma, bool pool_max, float* scores, int32_t* indices, int32_t* pool_used, const Problem* gather,
                           const void* K, const void* V, void* K_out, void* V_out, cudaStream_t st) {
   GatherArgs ga{};
@@ -488,7 +496,7 @@ cudaError_t launch_select(int rows, int n, int n_kv, int budget, const float* I_
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, select_kernel, n, n_kv, keep, I_hat, pool_dev, W, gamma, pool_max ? 1 : 0, scores, indices,
+  return cudaLaunchKernelEx(&cfg, select_kernel, n, n_kv, keep, keep_rows, I_hat, pool_dev, W, gamma, pool_max ? 1 : 0, scores, indices,
                             pool_used, per, use_smem, stage_taps, ga);
 }
 

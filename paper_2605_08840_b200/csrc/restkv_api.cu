@@ -382,7 +382,7 @@ restkv_status restkv_select(restkv_handle* h, const restkv_shape* shape, const f
   if ((s = check_ws(p, budget, h->sm_count, false, workspace, workspace_bytes, &ws)) != RESTKV_OK) return s;
   Call c{h, (cudaStream_t)stream};
   RESTKV_LAUNCH(c, RESTKV_KERNEL_SELECT,
-                launch_select(p.BH, p.n, p.n_kv, budget, nullptr, nullptr, 1, 0, false, const_cast<float*>(scores), indices, nullptr,
+                launch_select(p.BH, p.n, p.n_kv, budget, nullptr, nullptr, nullptr, 1, 0, false, const_cast<float*>(scores), indices, nullptr,
                               nullptr, nullptr, nullptr, nullptr, nullptr, c.st), 1);
   return RESTKV_OK;
 }
@@ -399,9 +399,11 @@ restkv_status restkv_compact(restkv_handle* h, const restkv_shape* shape, const 
   return RESTKV_OK;
 }
 
+// budgets non-null: per (batch, KV head) budgets on the device; `budget` is then the row stride of the outputs.
 static restkv_status evict_impl(restkv_handle* h, const restkv_shape* shape, const void* Q_obs, const void* K,
                                 const void* V, const float* O_obs, const float* LSE_obs, float ema_decay,
-                                const restkv_pool_params* pool, int budget, float* scores_out, int32_t* indices,
+                                const restkv_pool_params* pool, int budget, const int32_t* budgets, float* scores_out,
+                                int32_t* indices,
                                 void* K_out, void* V_out, void* workspace, size_t workspace_bytes,
                                 restkv_stream stream) {
   if (!h || !Q_obs || !K || !V || !indices || !K_out || !V_out || budget < 1) return RESTKV_ERR_INVALID_ARG;
@@ -425,17 +427,18 @@ static restkv_status evict_impl(restkv_handle* h, const restkv_shape* shape, con
   const int keep_rows = budget < p.n_kv ? budget : p.n_kv;
   FusedSelect sel{keep_rows, pool->width, pool->shift, scores, indices, K_out, V_out};
   bool sel_done = false;
-  if ((s = run_score(c, p, ws, Q_obs, K, V, ema_decay, pool, nullptr, nullptr, adaptive ? nullptr : &sel, &sel_done,
-                     O_obs, LSE_obs)) != RESTKV_OK)
+  if ((s = run_score(c, p, ws, Q_obs, K, V, ema_decay, pool, nullptr, nullptr, (adaptive || budgets) ? nullptr : &sel,
+                     &sel_done, O_obs, LSE_obs)) != RESTKV_OK)
     return s;
   h->last_evict_fused = sel_done;
   if (sel_done) return RESTKV_OK;
   // Pooling (Eq. 13) runs inside the select kernel, which also writes the pooled scores.  So does the gather
   // (Eq. 14) while the select kernel's clusters fit the GPU in one wave; with more (batch, head) rows than that the
   // stand-alone gather, which spreads over every SM, is the faster one.
-  const bool fuse_gather = p.BH * 8 <= h->sm_count;
+  // (with per-head budgets the index rows have unused tails, which only the select kernel's own gather skips)
+  const bool fuse_gather = p.BH * 8 <= h->sm_count || budgets != nullptr;
   RESTKV_LAUNCH(c, RESTKV_KERNEL_SELECT,
-                launch_select(p.BH, p.n, p.n_kv, budget, ws.I_hat, adaptive ? ws.pool : nullptr, pool->width,
+                launch_select(p.BH, p.n, p.n_kv, budget, budgets, ws.I_hat, adaptive ? ws.pool : nullptr, pool->width,
                               pool->shift, p.spatial == RESTKV_SPATIAL_MAX, scores, indices, nullptr,
                               fuse_gather ? &p : nullptr, K, V, K_out, V_out, c.st), 1);
   if (!fuse_gather) {
@@ -450,8 +453,18 @@ restkv_status restkv_evict(restkv_handle* h, const restkv_shape* shape, const vo
                            const void* V, float ema_decay, const restkv_pool_params* pool, int budget,
                            float* scores_out, int32_t* indices, void* K_out, void* V_out, void* workspace,
                            size_t workspace_bytes, restkv_stream stream) {
-  return evict_impl(h, shape, Q_obs, K, V, nullptr, nullptr, ema_decay, pool, budget, scores_out, indices, K_out, V_out,
-                    workspace, workspace_bytes, stream);
+  return evict_impl(h, shape, Q_obs, K, V, nullptr, nullptr, ema_decay, pool, budget, nullptr, scores_out, indices, K_out,
+                    V_out, workspace, workspace_bytes, stream);
+}
+
+restkv_status restkv_evict_budgets(restkv_handle* h, const restkv_shape* shape, const void* Q_obs, const void* K,
+                                   const void* V, float ema_decay, const restkv_pool_params* pool,
+                                   const int32_t* budgets, int max_budget, float* scores_out, int32_t* indices,
+                                   void* K_out, void* V_out, void* workspace, size_t workspace_bytes,
+                                   restkv_stream stream) {
+  if (!budgets) return RESTKV_ERR_INVALID_ARG;
+  return evict_impl(h, shape, Q_obs, K, V, nullptr, nullptr, ema_decay, pool, max_budget, budgets, scores_out, indices,
+                    K_out, V_out, workspace, workspace_bytes, stream);
 }
 
 restkv_status restkv_evict_from_lse(restkv_handle* h, const restkv_shape* shape, const void* Q_obs, const void* K,
@@ -460,8 +473,8 @@ restkv_status restkv_evict_from_lse(restkv_handle* h, const restkv_shape* shape,
                                     void* K_out, void* V_out, void* workspace, size_t workspace_bytes,
                                     restkv_stream stream) {
   if (!O_obs || !LSE_obs || !aligned16(O_obs)) return RESTKV_ERR_INVALID_ARG;
-  return evict_impl(h, shape, Q_obs, K, V, O_obs, LSE_obs, ema_decay, pool, budget, scores_out, indices, K_out, V_out,
-                    workspace, workspace_bytes, stream);
+  return evict_impl(h, shape, Q_obs, K, V, O_obs, LSE_obs, ema_decay, pool, budget, nullptr, scores_out, indices, K_out,
+                    V_out, workspace, workspace_bytes, stream);
 }
 
 restkv_status restkv_evict_host(restkv_handle* h, const restkv_shape* shape, const void* Q_host, const void* K_host,

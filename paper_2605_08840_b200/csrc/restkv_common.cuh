@@ -77,7 +77,7 @@ cudaError_t launch_simt_pass2(const Problem& p, const Workspace& ws, const void*
                               float ema_decay, float* I_raw, cudaStream_t st);
 cudaError_t launch_pool(const Problem& p, const Workspace& ws, const int* pool_dev, int W, int gamma, float* scores,
                         int32_t* pool_used, cudaStream_t st);
-cudaError_t launch_select(int rows, int n, int n_kv, int budget, const float* I_hat, const int* pool_dev, int W,
+cudaError_t launch_select(int rows, int n, int n_kv, int budget, const int* keep_rows, const float* I_hat, const int* pool_dev, int W,
                           int gamma, bool pool_max, float* scores, int32_t* indices, int32_t* pool_used, const Problem* gather,
                           const void* K, const void* V, void* K_out, void* V_out, cudaStream_t st);
 cudaError_t launch_compact(const Problem& p, const void* K, const void* V, const int32_t* indices, int n_sel,
