@@ -506,6 +506,52 @@ def main():
                     "raw_indicator_bytes": 4 * case.batch * case.n_q_heads * case.w * case.n}
         del ws_a
 
+    # ---- eviction again during decoding (Appendix B): the compacted cache plus M generated tokens, the last w of
+    #      them as the window (their own rows are the trailing, causally masked block) ----
+    reevict = None
+    if rank == 0 and case.causal_tail == 0 and case.n > case.budget + 128:
+        M, w, d, G = 128, case.w, case.head_dim, case.group
+        rows = case.budget + M
+        case_r = case.with_(n=rows - w, causal_tail=w)
+        shape_r = rk.make_shape(case_r.batch, case_r.n_q_heads, case_r.n_kv_heads, d, case_r.n_kv, w, w,
+                                rk.BF16 if case.dtype == "bf16" else rk.F32)
+        Kr, Vr = K[:, :, :rows].contiguous(), V[:, :, :rows].contiguous()
+        scale = 1.0 / float(np.sqrt(d))
+        O_r = torch.empty(case.batch, case.n_q_heads, w, d, dtype=torch.float32, device="cuda")
+        L_r = torch.empty(case.batch, case.n_q_heads, w, dtype=torch.float32, device="cuda")
+        ii = torch.arange(w, device="cuda").repeat(G)[:, None]
+        jj = torch.arange(rows, device="cuda")[None, :] - (rows - w)
+        for bi in range(case.batch):          # what the decode calls would have left behind (not timed)
+            for h in range(case.n_kv_heads):
+                qf = Q[bi, h * G:(h + 1) * G].float().reshape(G * w, d)
+                sc = (scale * (qf @ Kr[bi, h].float().T)).masked_fill(jj > ii, float("-inf"))
+                lse = torch.logsumexp(sc, dim=-1)
+                O_r[bi, h * G:(h + 1) * G] = (torch.exp(sc - lse[:, None]) @ Vr[bi, h].float()).view(G, w, d)
+                L_r[bi, h * G:(h + 1) * G] = lse.view(G, w)
+        ws_r = torch.empty(handle.workspace_bytes(shape_r, case.budget), dtype=torch.uint8, device="cuda")
+
+        def time_reevict(fn):
+            tr = []
+            for it in range(23):
+                flush.zero_()
+                ev0.record()
+                fn()
+                ev1.record()
+                torch.cuda.synchronize()
+                if it >= 3:
+                    tr.append(ev0.elapsed_time(ev1))
+            assert handle.poll_status() == rk.RESTKV_OK
+            return float(np.median(tr))
+
+        ms_a = time_reevict(lambda: handle.evict(shape_r, Q, Kr, Vr, case.ema_decay, pool, case.budget, indices, K_out,
+                                                 V_out, ws_r))
+        ms_b = time_reevict(lambda: handle.evict_from_lse(shape_r, Q, Kr, Vr, O_r, L_r, case.ema_decay, pool,
+                                                          case.budget, indices, K_out, V_out, ws_r))
+        reevict = {"note": "one re-eviction of a cache of budget + %d rows back to the budget, window = the last %d "
+                           "generated tokens (causal_tail = w)" % (M, w),
+                   "rows": rows, "evict_us": ms_a * 1e3, "evict_from_decode_statistics_us": ms_b * 1e3}
+        del Kr, Vr, O_r, L_r, ws_r
+
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----
     e2e = None
     if not args.no_e2e:
@@ -578,7 +624,7 @@ def main():
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roofline, "path_roofline": path_roofline, "kernels_ms": kmean,
         "kernels_ms_selection_as_own_kernel": kmean_split, "decode": decode, "from_lse": from_lse,
-        "variants": variants, "adaptive_window": adaptive,
+        "variants": variants, "adaptive_window": adaptive, "reevict": reevict,
     }
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(inp, case.budget)

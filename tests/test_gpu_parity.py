@@ -850,6 +850,67 @@ def test_budgets_per_head_with_the_adaptive_window(handle):
         assert np.all(idx[0, h, keep:] == -1)
 
 
+# ------------------------------------------------------------------ eviction again while decoding (Appendix B)
+@pytest.mark.parametrize("use_decode_statistics", [True, False])
+def test_reeviction_after_m_generated_tokens(handle, use_decode_statistics):
+    """Evict at prefill, decode M tokens over the compacted cache while appending their K/V, then evict again with the
+    last w decode queries as the window.  With use_decode_statistics the second eviction reads the outputs and
+    log-sum-exps that the decode calls themselves produced (restkv_evict_from_lse), as the paper suggests; otherwise
+    it recomputes them (restkv_evict).  Both rounds are held against the oracle run on the same caches."""
+    import torch
+    from paper_2605_08840_b200.inputs import Inputs
+    case = CONFIGS["cfg2"].with_(n=4096, budget=512)
+    B, w, M = case.budget, case.w, 48
+    tol = TOL["bf16"]
+    inp = make_inputs(case)
+    run = GpuRun(handle, inp)
+    scores1, idx1, _, _ = run.evict()
+    ref1 = oracle_scores(inp)
+    assert_scores_close(scores1, ref1.scores, tol)
+    assert_selection_valid(idx1, ref1.scores, B, tol)
+    take = idx1[..., None].astype(np.int64)
+    fresh = make_inputs(case.with_(n=M, recipe="normal"), seed=case.seed + 17)
+    K2 = np.ascontiguousarray(np.concatenate([np.take_along_axis(inp.K, take, axis=2), fresh.K], axis=2))
+    V2 = np.ascontiguousarray(np.concatenate([np.take_along_axis(inp.V, take, axis=2), fresh.V], axis=2))
+    queries = np.stack([make_decode_query(inp, seed=100 + t) for t in range(M)], axis=2)      # [b, Hq, M, d]
+    # decode step t sees the compacted rows and the appended rows up to its own
+    dK2, dV2 = (torch_dev(round_to_bf16_bits(a).view(np.int16), "bf16") for a in (K2, V2))
+    outs = torch.empty((M, case.batch, case.n_q_heads, case.head_dim), dtype=torch.float32, device="cuda")
+    lses = torch.empty((M, case.batch, case.n_q_heads), dtype=torch.float32, device="cuda")
+    for t in range(M):
+        rows = B + t + 1
+        qd = torch_dev(round_to_bf16_bits(queries[:, :, t]).view(np.int16), "bf16")
+        handle.decode(run.shape, qd, dK2[:, :, :rows].contiguous(), dV2[:, :, :rows].contiguous(), rows, outs[t],
+                      run.ws, lse=lses[t])
+    torch.cuda.synchronize()
+    t_chk = M - 1
+    ref_o, ref_l = oracle.decode(queries[:, :, t_chk], K2, V2)
+    assert_decode_close(outs[t_chk].cpu().numpy(), ref_o, queries[:, :, t_chk], K2, V2, "bf16")
+    np.testing.assert_allclose(lses[t_chk].cpu().numpy(), ref_l, rtol=0, atol=2e-3)
+    # second eviction: the last w generated tokens are the window; their own rows are the cache's last w rows
+    case2 = case.with_(name="reevict", n=B + M - w, causal_tail=w, recipe="normal")
+    inp2 = Inputs(case2, np.ascontiguousarray(queries[:, :, M - w:]), K2, V2)
+    run2 = GpuRun(handle, inp2)
+    if use_decode_statistics:
+        O_obs = outs[M - w:].permute(1, 2, 0, 3).contiguous()          # [b, Hq, w, d]
+        L_obs = lses[M - w:].permute(1, 2, 0).contiguous()             # [b, Hq, w]
+        handle.evict_from_lse(run2.shape, run2.Q, run2.K, run2.V, O_obs, L_obs, case2.ema_decay, run2.pool(), B,
+                              run2.indices, run2.K_out, run2.V_out, run2.ws, scores_out=run2.scores)
+    else:
+        handle.evict(run2.shape, run2.Q, run2.K, run2.V, case2.ema_decay, run2.pool(), B, run2.indices, run2.K_out,
+                     run2.V_out, run2.ws, scores_out=run2.scores)
+    torch.cuda.synchronize()
+    assert handle.poll_status() == rk.RESTKV_OK
+    ref2 = oracle_scores(inp2)
+    idx2 = run2.indices.cpu().numpy()
+    assert_scores_close(run2.scores.cpu().numpy(), ref2.scores, tol)
+    assert_selection_valid(idx2, ref2.scores, B, tol)
+    assert np.array_equal(idx2[..., -w:], np.broadcast_to(np.arange(B + M - w, B + M), idx2.shape[:2] + (w,)))
+    _, kbits, vbits = inp2.device_arrays()
+    assert_compaction_exact(idx2, kbits, run2._bits(run2.K_out))
+    assert_compaction_exact(idx2, vbits, run2._bits(run2.V_out))
+
+
 # ------------------------------------------------------------------ a device-side wait that runs out
 def test_wait_limit_runs_out_and_the_handle_recovers(handle):
     """With a wait limit of one SM clock the first CTA to reach a group barrier of the persistent score kernel gives
