@@ -18,11 +18,13 @@ def attention_output(q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: float) 
 
 
 def indicator_by_deletion(Q: np.ndarray, K: np.ndarray, V: np.ndarray, *, causal_tail: int = 0,
-                          scale: float | None = None) -> np.ndarray:
+                          scale: float | None = None, W_O: np.ndarray | None = None) -> np.ndarray:
     """I[b, hq, i, j] = || out(full) - out(without pair j) ||_2 for every scored row j < n (Eq. 6).
 
     Q [b,Hq,w,d]; K,V [b,Hkv,n_kv,d]; with causal_tail = w query i also sees trailing rows
     n..n+i (its own and earlier window tokens) and only prefix rows j < n are deleted.
+    W_O [Hq, d, d_model]: the head outputs are projected before they are compared (Eq. 4: the head's share of
+    the layer output is z W_O).
     """
     b, Hq, w, d = Q.shape
     _, Hkv, n_kv, _ = K.shape
@@ -45,5 +47,8 @@ def indicator_by_deletion(Q: np.ndarray, K: np.ndarray, V: np.ndarray, *, causal
                         out[bi, hq, i, j] = 0.0
                         continue
                     part = attention_output(Q[bi, hq, i], Kv[keep], Vv[keep], scale)
-                    out[bi, hq, i, j] = np.linalg.norm(full - part)
+                    diff = full - part
+                    if W_O is not None:
+                        diff = diff @ W_O[hq].astype(np.float64)
+                    out[bi, hq, i, j] = np.linalg.norm(diff)
     return out

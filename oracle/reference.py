@@ -51,7 +51,7 @@ def _load():
         lib.restkv_oracle_score_variant.argtypes = (
             [c_f, c_f, c_f] + [ctypes.c_int] * 7 + [ctypes.c_double, ctypes.c_double]
             + [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_double, ctypes.c_int]
-            + [ctypes.c_int] * 6
+            + [ctypes.c_int] * 6 + [c_f, ctypes.c_int]
             + [c_d, c_d, c_d, c_d, c_i, c_d, c_d]
         )
         lib.restkv_oracle_select.restype = ctypes.c_int
@@ -102,12 +102,13 @@ class ScoreResult:
 def score(Q, K, V, *, causal_tail: int = 0, scale: Optional[float] = None, ema_decay: float = 0.7,
           pool_mode: int = 0, width: int = 1, shift: int = 0, beta: float = 2000.0, base_width: int = 1,
           budget: int = 0, literal_gamma: bool = False, group_mode: int = 0,
-          indicator_mode: int = 0, temporal_mode: int = 0, spatial_mode: int = 0,
+          indicator_mode: int = 0, temporal_mode: int = 0, spatial_mode: int = 0, W_O=None,
           want_I_hat: bool = True, want_I_raw: bool = False, want_A: bool = False,
           want_O: bool = False) -> ScoreResult:
     """Steps Eq. 3 -> Eq. 7 -> Eq. 8-9 -> (Eq. 10-12) -> Eq. 13.  Q [b,Hq,w,d], K,V [b,Hkv,n_kv,d].
 
-    The three `*_mode` switches pick the ablation variants of Appendix G (0 = the method as printed)."""
+    The three `*_mode` switches pick the ablation variants of Appendix G (0 = the method as printed).
+    W_O [Hq, d, d_model] float32: the output projection of Eq. 4, one d x d_model slice per query head."""
     Q, K, V = _f32(Q), _f32(K), _f32(V)
     b, Hq, w, d = Q.shape
     b2, Hkv, n_kv, d2 = K.shape
@@ -125,13 +126,21 @@ def score(Q, K, V, *, causal_tail: int = 0, scale: Optional[float] = None, ema_d
     D = np.zeros((b, Hkv, 2), np.float64) if pool_mode == 1 else None
     variant = (int(indicator_mode), int(temporal_mode), int(spatial_mode))
     lib = _load()
-    fn = lib.restkv_oracle_score if variant == (0, 0, 0) else lib.restkv_oracle_score_variant
+    plain = variant == (0, 0, 0) and W_O is None
+    fn = lib.restkv_oracle_score if plain else lib.restkv_oracle_score_variant
+    extra = ()
+    if not plain:
+        if W_O is not None:
+            W_O = _f32(W_O)
+            if W_O.ndim != 3 or W_O.shape[:2] != (Hq, d):
+                raise ValueError("W_O must be [Hq, d, d_model]")
+        extra = variant + (_ptr(W_O, ctypes.c_float), 0 if W_O is None else int(W_O.shape[2]))
     rc = fn(
         _ptr(Q, ctypes.c_float), _ptr(K, ctypes.c_float), _ptr(V, ctypes.c_float),
         b, Hq, Hkv, d, n_kv, w, causal_tail, float(scale), float(ema_decay),
         int(pool_mode), int(width), int(shift), float(beta), int(base_width),
         int(budget), int(bool(literal_gamma)), int(group_mode),
-        *(() if variant == (0, 0, 0) else variant),
+        *extra,
         _ptr(A, ctypes.c_double), _ptr(O, ctypes.c_double), _ptr(I_raw, ctypes.c_double),
         _ptr(I_hat, ctypes.c_double), _ptr(pool, ctypes.c_int), _ptr(D, ctypes.c_double),
         _ptr(scores, ctypes.c_double))

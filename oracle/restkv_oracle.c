@@ -16,7 +16,7 @@
  *
  * Steps and where the paper defines them:
  *   logits, softmax, output        Eq. 3   (Section 3.1)
- *   reconstruction indicator       Eq. 7   (Section 3.2), W_O taken as identity
+ *   reconstruction indicator       Eq. 7   (Section 3.2), W_O the identity unless one is given (Eq. 4)
  *   EMA temporal smoothing         Eq. 8-9 (Section 3.3), recursion as written
  *   adaptive window parameters     Eq. 10-12
  *   box pooling (final indicator)  Eq. 13
@@ -111,6 +111,8 @@ static int top_indices(const double* x, int n, int count, int* out) {
  *                  indicator alone   (Appendix G.2)
  *  spatial_mode    0 = box mean of Eq. 13;  1 = maximum over the same box, taps outside the scored rows count
  *                  as 0 as they do in the mean   (Appendix G.2)
+ *  W_O, d_model    the output projection of Eq. 4 as [Hq, d, d_model] (query head hq owns rows hq*d .. hq*d+d-1 of
+ *                  the model's W_O); Eq. 7 then measures || (z_t - v_j) W_O^(hq) ||_2.  NULL: identity.
  *
  * Optional outputs (NULL to skip):
  *  A_out     [batch, Hq, w, n_kv]  attention weights (Eq. 3)
@@ -127,9 +129,11 @@ int restkv_oracle_score_variant(const float* Q, const float* K, const float* V,
                         int pool_mode, int width, int shift, double beta, int base_width,
                         int budget, int literal_gamma, int group_mode,
                         int indicator_mode, int temporal_mode, int spatial_mode,
+                        const float* W_O, int d_model,
                         double* A_out, double* O_out, double* I_raw, double* I_hat,
                         int* pool_out, double* D_out, double* scores) {
   if (!Q || !K || !V || !scores) return ORACLE_BAD_ARG;
+  if (W_O && d_model < 1) return ORACLE_BAD_ARG;
   if (indicator_mode < 0 || indicator_mode > 2 || temporal_mode < 0 || temporal_mode > 3) return ORACLE_BAD_ARG;
   if (spatial_mode < 0 || spatial_mode > 1) return ORACLE_BAD_ARG;
   if (batch < 1 || Hq < 1 || Hkv < 1 || d < 1 || w < 1 || n_kv < 1) return ORACLE_BAD_ARG;
@@ -181,12 +185,23 @@ int restkv_oracle_score_variant(const float* Q, const float* K, const float* V,
         for (int k = 0; k < d; ++k) o[k] = 0.0;
         for (int j = 0; j < visible; ++j)
           for (int k = 0; k < d; ++k) o[k] += a[j] * (double)Vh[(size_t)j * d + k]; /* z_t = A_t V */
-        /* Eq. 7 with W_O = identity: I[j] = A[j] / (1 - A[j]) * || z_t - v_j ||_2 */
+        /* Eq. 7: I[j] = A[j] / (1 - A[j]) * || (z_t - v_j) W_O ||_2, W_O the head's d x d_model slice
+         * (Eq. 4) or the identity */
         for (int j = 0; j < n && indicator_mode == 0; ++j) {
           double ss = 0.0;
-          for (int k = 0; k < d; ++k) {
-            double df = o[k] - (double)Vh[(size_t)j * d + k];
-            ss += df * df;
+          if (W_O) {
+            const float* Wh = W_O + (size_t)hq * d * d_model;
+            for (int mcol = 0; mcol < d_model; ++mcol) {
+              double y = 0.0;
+              for (int k = 0; k < d; ++k)
+                y += (o[k] - (double)Vh[(size_t)j * d + k]) * (double)Wh[(size_t)k * d_model + mcol];
+              ss += y * y;
+            }
+          } else {
+            for (int k = 0; k < d; ++k) {
+              double df = o[k] - (double)Vh[(size_t)j * d + k];
+              ss += df * df;
+            }
           }
           double one_minus = 1.0 - a[j];
           /* a single visible row has A = 1 and nothing to redistribute to: define I = 0 */
@@ -299,7 +314,7 @@ int restkv_oracle_score(const float* Q, const float* K, const float* V,
                         int* pool_out, double* D_out, double* scores) {
   return restkv_oracle_score_variant(Q, K, V, batch, Hq, Hkv, d, n_kv, w, causal_tail, scale, ema_decay,
                                      pool_mode, width, shift, beta, base_width, budget, literal_gamma, group_mode,
-                                     0, 0, 0, A_out, O_out, I_raw, I_hat, pool_out, D_out, scores);
+                                     0, 0, 0, NULL, 0, A_out, O_out, I_raw, I_hat, pool_out, D_out, scores);
 }
 
 /* Eq. 14: per row of `scores` [rows, n_kv], the min(budget, n_kv) largest entries

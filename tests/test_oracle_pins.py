@@ -479,3 +479,51 @@ def test_variant_modes_are_validated():
     for bad in (dict(indicator_mode=3), dict(temporal_mode=4), dict(spatial_mode=2), dict(indicator_mode=-1)):
         with pytest.raises(RuntimeError):
             oracle.score(Q, K, V, **bad)
+
+
+# ---------------------------------------------------------------- Eq. 4 / Eq. 7 with the output projection
+@pytest.mark.parametrize("d_model", [5, 8, 13])
+@pytest.mark.parametrize("causal_tail", [0, 3])
+def test_projected_closed_form_equals_projected_token_deletion(d_model, causal_tail):
+    w = 3
+    Q, K, V = _qkv(b=1, Hq=4, Hkv=2, w=w, d=8, n_kv=20 + causal_tail, seed=21, kscale=3.0)
+    W = _rand((4, 8, d_model), 22)
+    res = oracle.score(Q, K, V, causal_tail=causal_tail, W_O=W, want_I_raw=True)
+    brute = bruteforce.indicator_by_deletion(Q, K, V, causal_tail=causal_tail, W_O=W)
+    np.testing.assert_allclose(res.I_raw, brute, rtol=1e-9, atol=1e-12)
+    plain = oracle.score(Q, K, V, causal_tail=causal_tail, want_I_raw=True).I_raw
+    assert not np.allclose(res.I_raw, plain, rtol=1e-2)
+
+
+def test_projection_by_identity_or_by_orthonormal_rows_changes_nothing():
+    Q, K, V = _qkv(b=1, Hq=4, Hkv=2, w=3, d=8, n_kv=20, seed=23, kscale=2.0)
+    plain = oracle.score(Q, K, V).scores
+    eye = np.broadcast_to(np.eye(8, dtype=np.float32), (4, 8, 8)).copy()
+    np.testing.assert_allclose(oracle.score(Q, K, V, W_O=eye).scores, plain, rtol=1e-12)
+    # rows of W orthonormal (d_model = 11 > d): || x W || = || x ||
+    rng = np.random.default_rng(24)
+    W = np.stack([np.linalg.qr(rng.standard_normal((11, 8)))[0].T for _ in range(4)]).astype(np.float32)
+    np.testing.assert_allclose(oracle.score(Q, K, V, W_O=W).scores, plain, rtol=1e-6)
+
+
+def test_projected_indicator_is_the_plain_indicator_on_projected_values():
+    # (z - v) W = z' - v' with V' = V W, and the attention weights do not depend on V: per query head, the projected
+    # indicator equals the plain one computed on that head's projected values
+    Q, K, V = _qkv(b=1, Hq=4, Hkv=2, w=3, d=8, n_kv=20, seed=25, kscale=2.0)
+    W = _rand((4, 8, 8), 26)
+    got = oracle.score(Q, K, V, W_O=W, want_I_raw=True).I_raw
+    for hq in range(4):
+        h = hq // 2
+        Vp = (V[:, h:h + 1].astype(np.float64) @ W[hq].astype(np.float64))
+        # the product is not float32-exact: compare against the oracle run on its float32 rounding, loosely
+        alone = oracle.score(np.ascontiguousarray(Q[:, hq:hq + 1]), np.ascontiguousarray(K[:, h:h + 1]),
+                             Vp.astype(np.float32), want_I_raw=True).I_raw
+        np.testing.assert_allclose(got[:, hq], alone[:, 0], rtol=1e-5)
+
+
+def test_projection_scale_scales_the_scores():
+    Q, K, V = _qkv(b=1, Hq=2, Hkv=1, w=3, d=8, n_kv=20, seed=27, kscale=2.0)
+    W = _rand((2, 8, 6), 28)
+    a = oracle.score(Q, K, V, W_O=W, width=3).scores
+    b = oracle.score(Q, K, V, W_O=(W * np.float32(4.0)), width=3).scores
+    np.testing.assert_allclose(b, 4.0 * a, rtol=1e-12)
