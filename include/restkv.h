@@ -328,6 +328,29 @@ typedef struct {
 } restkv_variant;
 restkv_status restkv_set_variant(restkv_handle* h, const restkv_variant* v);   /* v: host pointer, read during the call */
 
+/*
+ * The output projection inside the indicator (Eq. 4 and Eq. 7 as printed: || (o_t - v_j) W_O ||_2, where W_O is the
+ * query head's d x d_model slice of the layer's output projection).  A handle starts without one: W_O = identity.
+ *
+ * restkv_prepare_output_projection -- once per layer: from W_O, device [n_q_heads * head_dim, d_model] row-major
+ *   (rows hq*head_dim .. of query head hq; dtype bf16 or f32), fill the caller-owned device buffer `factor`
+ *   (256-byte aligned, restkv_output_projection_bytes(n_q_heads, head_dim) bytes) with what the kernels read: per
+ *   query head M = W W^T (fp32), a Cholesky factor of M rounded to bf16 and the product of the rounded factor with
+ *   its transpose.  Two kernels on `stream`.  head_dim a multiple of 16, at most 128 (else RESTKV_ERR_UNSUPPORTED);
+ *   RESTKV_ERR_WORKSPACE if `factor` is misaligned or too small.  A singular M (d_model < head_dim) is accepted;
+ *   its null directions get no weight.
+ * restkv_set_output_projection -- every later restkv_score / restkv_evict / ..._from_lse / ..._budgets /
+ *   restkv_evict_host call through the handle measures Eq. 7's norm through this factor (the buffer must stay
+ *   alive and unchanged; NULL returns to the identity).  A call whose shape has other n_q_heads or head_dim than
+ *   the factor returns RESTKV_ERR_INVALID_ARG.  The attention-weight indicators of restkv_set_variant have no norm
+ *   of an output difference and ignore it.
+ */
+size_t restkv_output_projection_bytes(int n_q_heads, int head_dim);
+restkv_status restkv_prepare_output_projection(restkv_handle* h, int n_q_heads, int head_dim, int d_model,
+                                               restkv_dtype dtype, const void* W_O, void* factor,
+                                               size_t factor_bytes, restkv_stream stream);
+restkv_status restkv_set_output_projection(restkv_handle* h, const void* factor, int n_q_heads, int head_dim);
+
 #ifdef __cplusplus
 }
 #endif

@@ -26,6 +26,7 @@ EXPORTS = [
     "restkv_poll_status", "restkv_launch_count", "restkv_last_cuda_error", "restkv_error_string",
     "restkv_set_kernel_path", "restkv_set_profile_events", "restkv_set_wait_limit", "restkv_set_fused_select", "restkv_last_evict_fused_select",
     "restkv_set_variant", "restkv_evict_budgets",
+    "restkv_output_projection_bytes", "restkv_prepare_output_projection", "restkv_set_output_projection",
 ]
 KERNEL_NONE, KERNEL_PASS1, KERNEL_COMBINE, KERNEL_PASS2, KERNEL_POOL, KERNEL_SELECT, KERNEL_COMPACT = range(7)
 
@@ -107,6 +108,10 @@ def load_library() -> ctypes.CDLL:
     lib.restkv_set_fused_select.argtypes = [vp, ci]
     lib.restkv_last_evict_fused_select.argtypes = [vp]
     lib.restkv_set_variant.argtypes = [vp, ctypes.POINTER(Variant)]
+    lib.restkv_output_projection_bytes.argtypes = [ci, ci]
+    lib.restkv_output_projection_bytes.restype = sz
+    lib.restkv_prepare_output_projection.argtypes = [vp, ci, ci, ci, ci, vp, vp, sz, vp]
+    lib.restkv_set_output_projection.argtypes = [vp, vp, ci, ci]
     _lib = lib
     return lib
 
@@ -267,6 +272,18 @@ class Handle:
     def set_variant(self, indicator: int = 0, temporal: int = 0, spatial: int = 0, group: int = 0):
         v = Variant(int(indicator), int(temporal), int(spatial), int(group))
         self._check(self._lib.restkv_set_variant(self._h, ctypes.byref(v)), "restkv_set_variant")
+
+    def output_projection_bytes(self, n_q_heads: int, head_dim: int) -> int:
+        return int(self._lib.restkv_output_projection_bytes(int(n_q_heads), int(head_dim)))
+
+    def prepare_output_projection(self, n_q_heads, head_dim, d_model, dtype, W_O, factor, stream=None):
+        self._check(self._lib.restkv_prepare_output_projection(
+            self._h, int(n_q_heads), int(head_dim), int(d_model), int(dtype), _ptr(W_O), _ptr(factor),
+            factor.numel() * factor.element_size(), _stream_ptr(stream)), "restkv_prepare_output_projection")
+
+    def set_output_projection(self, factor=None, n_q_heads: int = 0, head_dim: int = 0):
+        self._check(self._lib.restkv_set_output_projection(self._h, _ptr(factor), int(n_q_heads), int(head_dim)),
+                    "restkv_set_output_projection")
 
     def set_wait_limit(self, sm_clocks: int):
         self._check(self._lib.restkv_set_wait_limit(self._h, int(sm_clocks)), "restkv_set_wait_limit")

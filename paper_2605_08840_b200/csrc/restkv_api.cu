@@ -18,6 +18,8 @@ struct restkv_handle {
   bool last_evict_fused;      // whether the last restkv_evict did
   long long wait_limit;       // SM clocks a device-side wait may last
   restkv_variant variant;     // ablation variant of the score calls (all 0: the method as printed)
+  const void* proj_factor;    // output-projection factor of the score calls (null: identity), caller-owned
+  int proj_heads, proj_dim;   // the shape it was prepared for
   cudaEvent_t prof_start[7], prof_stop[7];   // per restkv_kernel_id, null = not timed
 };
 
@@ -73,6 +75,8 @@ size_t plan_workspace(const Problem& p, int budget, int sm_count, bool adaptive,
   w.O_m2 = (__nv_bfloat16*)take(BH * R * d * sizeof(__nv_bfloat16));
   w.aug = (__nv_bfloat16*)take(BH * R * 64 * sizeof(__nv_bfloat16));
   w.I_hat = (float*)take(BH * (size_t)p.n * sizeof(float));
+  w.O_proj = (float*)take(BH * R * d * sizeof(float));
+  w.vmv = (float*)take(BH * (size_t)p.G * (size_t)p.n_kv * sizeof(float));
   w.scores = (float*)take(BH * (size_t)p.n_kv * sizeof(float));
   w.pool = (int*)take(BH * 2 * sizeof(int));
   w.dec_part = (float*)take(BH * (size_t)kDecodeMaxSplits * p.G * (d + 2) * sizeof(float));
@@ -150,9 +154,18 @@ static restkv_status make_problem(const restkv_shape* s, bool need_kv, Problem* 
   return RESTKV_OK;
 }
 
-static void apply_variant(const restkv_handle* h, Problem* p) {
+// The handle's variant and output projection become part of the problem; false if the projection was prepared
+// for another shape.
+static bool apply_variant(const restkv_handle* h, Problem* p) {
   p->indicator = h->variant.indicator; p->temporal = h->variant.temporal;
   p->spatial = h->variant.spatial; p->group = h->variant.group;
+  p->proj = Projection{};
+  if (h->proj_factor) {
+    if (h->proj_heads != p->Hq || h->proj_dim != p->d) return false;
+    // only Eq. 7 has the projected norm
+    if (p->indicator == RESTKV_INDICATOR_RECONSTRUCTION) p->proj = projection_view(h->proj_factor, p->Hq, p->d);
+  }
+  return true;
 }
 
 static restkv_status check_pool(const restkv_pool_params* pp, const Problem& p) {
@@ -207,6 +220,7 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
   bool use_tc = tc_supported(p) && c.h->tc_state != nullptr && !(adaptive && O_given) &&
                 tc_variant_supported(p, ema_decay);
   if (p.n_kv == 1 && p.indicator != RESTKV_INDICATOR_RECONSTRUCTION) use_tc = false;
+  if (p.proj.M && !tc_vmv_supported(p)) use_tc = false;
   if (c.h->kernel_path == 1) use_tc = false;
   if (c.h->kernel_path >= 2 && !use_tc) return RESTKV_ERR_UNSUPPORTED;
   if (!use_tc && !simt_supported(p)) return RESTKV_ERR_UNSUPPORTED;
@@ -220,6 +234,9 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
   } else if (O_given) {
     // the window rows' outputs and log-sum-exps come from the caller: pass 1 and the merge are not needed
     RESTKV_LAUNCH(c, RESTKV_KERNEL_COMBINE, launch_from_lse_prep(p, ws, O_given, LSE_given, use_tc, c.st), 1);
+    if (use_tc && p.proj.M)
+      RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS1,
+                    launch_tc_vmv(c.h->tc_state, p, V, ws.vmv, c.h->sm_count, c.h->wait_limit, c.h->dev_status, c.st), 1);
     if (use_tc) {
       const bool with_sel = sel && c.h->fused_select &&
                             tc_fused_select_supported(p, c.h->sm_count, false, sel->keep, sel->W, sel->gamma);
@@ -230,6 +247,7 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
     } else {
       Workspace wsl = ws;
       wsl.O_f32 = const_cast<float*>(O_given);
+      if (p.proj.M) RESTKV_LAUNCH(c, RESTKV_KERNEL_COMBINE, launch_projection_rows(p, O_given, ws.O_proj, c.st), 1);
       RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2,
                     launch_simt_pass2(p, wsl, Q, K, V, ema_decay, adaptive ? ws.I_raw : nullptr, c.st), 1);
     }
@@ -237,6 +255,9 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
     // pass 1, merge and pass 2 in one persistent launch (timed as "pass 2"); path 3 keeps only as many heads in
     // flight as fit in L2 so that pass 2 re-reads K and V from there
     const bool reuse_l2 = c.h->kernel_path == 3;
+    if (p.proj.M)   // the tokens' own terms under the output projection, by a kernel of its own (timed as "pass 1")
+      RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS1,
+                    launch_tc_vmv(c.h->tc_state, p, V, ws.vmv, c.h->sm_count, c.h->wait_limit, c.h->dev_status, c.st), 1);
     const bool with_sel = sel && c.h->fused_select &&
                           tc_fused_select_supported(p, c.h->sm_count, reuse_l2, sel->keep, sel->W, sel->gamma);
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2,
@@ -247,6 +268,7 @@ static restkv_status run_score(Call& c, const Problem& p, const Workspace& ws, c
   } else {
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS1, launch_simt_pass1(p, ws, Q, K, V, c.st), 1);
     RESTKV_LAUNCH(c, RESTKV_KERNEL_COMBINE, launch_combine(p, ws, c.st), 1);
+    if (p.proj.M) RESTKV_LAUNCH(c, RESTKV_KERNEL_COMBINE, launch_projection_rows(p, ws.O_f32, ws.O_proj, c.st), 1);
     RESTKV_LAUNCH(c, RESTKV_KERNEL_PASS2, launch_simt_pass2(p, ws, Q, K, V, ema_decay, adaptive ? ws.I_raw : nullptr, c.st), 1);
   }
   if (adaptive) {
@@ -294,6 +316,8 @@ restkv_status restkv_create(restkv_handle** out) {
   h->fused_select = true;
   h->last_evict_fused = false;
   h->variant = restkv_variant{0, 0, 0, 0};
+  h->proj_factor = nullptr;
+  h->proj_heads = h->proj_dim = 0;
   h->launches = 0;
   h->last_cuda_error = 0;
   h->kernel_path = 0;
@@ -339,7 +363,7 @@ restkv_status restkv_score(restkv_handle* h, const restkv_shape* shape, const vo
   Problem p;
   restkv_status s = make_problem(shape, true, &p);
   if (s != RESTKV_OK) return s;
-  apply_variant(h, &p);
+  if (!apply_variant(h, &p)) return RESTKV_ERR_INVALID_ARG;
   if ((s = check_pool(pool, p)) != RESTKV_OK) return s;
   Workspace ws;
   const bool adaptive = pool->mode == RESTKV_POOL_ADAPTIVE;
@@ -361,7 +385,7 @@ restkv_status restkv_score_from_lse(restkv_handle* h, const restkv_shape* shape,
   Problem p;
   restkv_status s = make_problem(shape, true, &p);
   if (s != RESTKV_OK) return s;
-  apply_variant(h, &p);
+  if (!apply_variant(h, &p)) return RESTKV_ERR_INVALID_ARG;
   if ((s = check_pool(pool, p)) != RESTKV_OK) return s;
   Workspace ws;
   const bool adaptive = pool->mode == RESTKV_POOL_ADAPTIVE;
@@ -414,7 +438,7 @@ static restkv_status evict_impl(restkv_handle* h, const restkv_shape* shape, con
   Problem p;
   restkv_status s = make_problem(shape, true, &p);
   if (s != RESTKV_OK) return s;
-  apply_variant(h, &p);
+  if (!apply_variant(h, &p)) return RESTKV_ERR_INVALID_ARG;
   if ((s = check_pool(pool, p)) != RESTKV_OK) return s;
   Workspace ws;
   const bool adaptive = pool->mode == RESTKV_POOL_ADAPTIVE;
@@ -632,6 +656,40 @@ restkv_status restkv_set_variant(restkv_handle* h, const restkv_variant* v) {
   if (v->spatial < 0 || v->spatial > RESTKV_SPATIAL_MAX) return RESTKV_ERR_INVALID_ARG;
   if (v->group < 0 || v->group > RESTKV_GROUP_MAX) return RESTKV_ERR_INVALID_ARG;
   h->variant = *v;
+  return RESTKV_OK;
+}
+
+size_t restkv_output_projection_bytes(int n_q_heads, int head_dim) {
+  if (n_q_heads < 1 || head_dim < 16 || head_dim > 128 || head_dim % 16 != 0) return 0;
+  return projection_factor_bytes(n_q_heads, head_dim);
+}
+
+restkv_status restkv_prepare_output_projection(restkv_handle* h, int n_q_heads, int head_dim, int d_model,
+                                               restkv_dtype dtype, const void* W_O, void* factor,
+                                               size_t factor_bytes, restkv_stream stream) {
+  if (!h || !W_O || !factor || n_q_heads < 1 || d_model < 1) return RESTKV_ERR_INVALID_ARG;
+  if (dtype != RESTKV_BF16 && dtype != RESTKV_F32) return RESTKV_ERR_INVALID_ARG;
+  if (head_dim < 16 || head_dim > 128 || head_dim % 16 != 0) return RESTKV_ERR_UNSUPPORTED;
+  if (((uintptr_t)factor & 255u) != 0 || factor_bytes < projection_factor_bytes(n_q_heads, head_dim))
+    return RESTKV_ERR_WORKSPACE;
+  Call c{h, (cudaStream_t)stream};
+  RESTKV_LAUNCH(c, RESTKV_KERNEL_NONE,
+                launch_projection_prepare(n_q_heads, head_dim, d_model, dtype, W_O, factor, c.st), 2);
+  return RESTKV_OK;
+}
+
+restkv_status restkv_set_output_projection(restkv_handle* h, const void* factor, int n_q_heads, int head_dim) {
+  if (!h) return RESTKV_ERR_INVALID_ARG;
+  if (!factor) {
+    h->proj_factor = nullptr;
+    h->proj_heads = h->proj_dim = 0;
+    return RESTKV_OK;
+  }
+  if (n_q_heads < 1 || head_dim < 16 || head_dim > 128 || head_dim % 16 != 0 || ((uintptr_t)factor & 255u) != 0)
+    return RESTKV_ERR_INVALID_ARG;
+  h->proj_factor = factor;
+  h->proj_heads = n_q_heads;
+  h->proj_dim = head_dim;
   return RESTKV_OK;
 }
 

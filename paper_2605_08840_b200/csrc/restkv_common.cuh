@@ -16,6 +16,13 @@ enum : unsigned int {
   kDevBadIndex = 2u,     // an index outside [0, n_kv) reached the gather
 };
 
+// The output projection of Eq. 4 as quadratic forms, one per query head (all null: identity).
+struct Projection {
+  const float* M;            // [Hq, d, d]  W W^T
+  const float* Mt;           // [Hq, d, d]  L L^T of the bf16-rounded Cholesky factor L of M
+  const __nv_bfloat16* LT;   // [Hq, d, d]  that factor, transposed
+};
+
 struct Problem {
   int batch, Hq, Hkv, G, d;
   int n_kv, n, w, tail;   // n = scored prefix rows, tail = causal_tail
@@ -25,6 +32,7 @@ struct Problem {
   long long ksb, ksh, ksn, vsb, vsh, vsn;  // element strides
   restkv_dtype dtype;
   int indicator, temporal, spatial, group;   // restkv_variant; all 0 = the method as the paper prints it
+  Projection proj;
 };
 
 // Workspace carve-up (all offsets 256-byte aligned).
@@ -46,6 +54,8 @@ struct Workspace {
   __nv_bfloat16* O_m2;    // [BH, R, d]   -2 * bf16(O)
   __nv_bfloat16* aug;     // [BH, R, 64]  per-row constants as bf16 pieces (see combine_kernel)
   float* I_hat;           // [BH, n]
+  float* O_proj;          // [BH, R, d]   M o_r, with an output projection only
+  float* vmv;             // [BH, G, n_kv] v_j^T Mt v_j, with an output projection on the tensor-core path only
   float* scores;          // [BH, n_kv] (used when the caller passes no scores buffer)
   int* pool;              // [BH, 2] (W, gamma)
   float* dec_part;        // decode partials
@@ -87,6 +97,13 @@ cudaError_t launch_decode(const Problem& p, const void* q, const void* Kc, const
 cudaError_t launch_adaptive_params(const Problem& p, const Workspace& ws, int budget, float beta, int base_width,
                                    cudaStream_t st, int* n_launches);
 
+// Output projection (Eq. 4): the caller-owned factor buffer and the per-call projected rows.
+size_t projection_factor_bytes(int n_q_heads, int d);
+Projection projection_view(const void* factor, int n_q_heads, int d);
+cudaError_t launch_projection_prepare(int n_q_heads, int d, int d_model, restkv_dtype dtype, const void* W_O,
+                                      void* factor, cudaStream_t st);
+cudaError_t launch_projection_rows(const Problem& p, const float* O, float* O_proj, cudaStream_t st);
+
 // Tensor-core (tcgen05 / TMEM / TMA) score kernels.  `supported` says whether the shape qualifies.
 bool tc_supported(const Problem& p);
 cudaError_t tc_init(void** state);   // resolves the driver entry point for tensor-map encoding
@@ -100,6 +117,10 @@ cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, 
 // normalisers; otherwise fin_m = LSE, fin_l = 1.
 cudaError_t launch_from_lse_prep(const Problem& p, const Workspace& ws, const float* O, const float* LSE,
                                  bool tensor_core, cudaStream_t st);
+// Output projection on the tensor-core path: the tokens' own terms v^T Mt v, [BH, G, n_kv], by a kernel of its own.
+bool tc_vmv_supported(const Problem& p);
+cudaError_t launch_tc_vmv(void* state, const Problem& p, const void* V, float* out, int sm_count, long long wait_limit,
+                          unsigned int* dev_status, cudaStream_t st);
 // Whether the tensor-core kernel's temporal chain can carry the variant's weights for this decay and window.
 bool tc_variant_supported(const Problem& p, float ema_decay);
 bool tc_fused_select_supported(const Problem& p, int sm_count, bool reuse_l2, int keep, int W, int gamma);

@@ -150,13 +150,15 @@ __global__ void combine_kernel(int R, int d, int splits, const float* __restrict
 template <typename T>
 __global__ void simt_pass2_kernel(Problem p, const T* __restrict__ Q, const T* __restrict__ K,
                                   const T* __restrict__ V, const float* __restrict__ fin_m,
-                                  const float* __restrict__ fin_l, const float* __restrict__ O_f32, float ema_decay,
+                                  const float* __restrict__ fin_l, const float* __restrict__ O_f32,
+                                  const float* __restrict__ O_proj, float ema_decay,
                                   float* __restrict__ I_hat, float* __restrict__ I_raw, int GP) {
   extern __shared__ float smem[];
   const int d = p.d, ld = d + 1;
   float* Kt = smem;
   float* Vt = Kt + (size_t)kP2Tile * ld;
   float* red = Vt + (size_t)kP2Tile * ld;
+  float* MVs = red + (size_t)GP * kP2Tile;   // [GP * kP2Tile][ld]: M v_j of each thread, with a projection only
 
   const int bh = blockIdx.y, b = bh / p.Hkv, h = bh % p.Hkv;
   const int j0 = blockIdx.x * kP2Tile;
@@ -188,6 +190,17 @@ __global__ void simt_pass2_kernel(Problem p, const T* __restrict__ Q, const T* _
     }
     for (int g = slot; g < p.G; g += GP) {
       float ema = 0.f, pw = 1.f;   // pw = ema_decay^i for the inverted EMA
+      // Eq. 7 with the projection of Eq. 4: (o - v)^T M (o - v) = (o - v) . (M o - M v); M v is formed once per
+      // token and query head, M o comes in
+      float* mv = MVs + (size_t)threadIdx.x * ld;
+      if (p.proj.M && p.indicator == RESTKV_INDICATOR_RECONSTRUCTION) {
+        const float* Mg = p.proj.M + (long long)(h * p.G + g) * d * d;
+        for (int i = 0; i < d; ++i) {
+          float acc = 0.f;
+          for (int k = 0; k < d; ++k) acc = fmaf(Mg[i * d + k], vr[k], acc);
+          mv[i] = acc;
+        }
+      }
       for (int i = 0; i < p.w; ++i) {
         // without temporal smoothing only the newest query counts (the raw indicators still want every query)
         if (p.temporal == RESTKV_TEMPORAL_NONE && i != p.w - 1 && !I_raw) continue;
@@ -195,10 +208,19 @@ __global__ void simt_pass2_kernel(Problem p, const T* __restrict__ Q, const T* _
         const T* qr = Qh + (long long)r * d;
         const float* orow = Oh + (long long)r * d;
         float s = 0.f, ss = 0.f;
-        for (int k = 0; k < d; ++k) {
-          s = fmaf(to_f32<T>(qr[k]), kr[k], s);
-          const float df = orow[k] - vr[k];
-          ss = fmaf(df, df, ss);
+        if (p.proj.M) {
+          const float* oprow = O_proj + ((long long)bh * p.R + r) * d;
+          for (int k = 0; k < d; ++k) {
+            s = fmaf(to_f32<T>(qr[k]), kr[k], s);
+            ss = fmaf(orow[k] - vr[k], oprow[k] - mv[k], ss);
+          }
+          ss = fmaxf(ss, 0.f);
+        } else {
+          for (int k = 0; k < d; ++k) {
+            s = fmaf(to_f32<T>(qr[k]), kr[k], s);
+            const float df = orow[k] - vr[k];
+            ss = fmaf(df, df, ss);
+          }
         }
         const long long ri = (long long)bh * p.R + r;
         const float l = fin_l[ri];
@@ -279,19 +301,20 @@ cudaError_t launch_simt_pass2(const Problem& p, const Workspace& ws, const void*
                               float ema_decay, float* I_raw, cudaStream_t st) {
   int GP = p.G < 4 ? p.G : 4;
   const int threads = kP2Tile * GP;
-  const size_t smem = ((size_t)2 * kP2Tile * (p.d + 1) + (size_t)GP * kP2Tile) * sizeof(float);
+  size_t smem = ((size_t)2 * kP2Tile * (p.d + 1) + (size_t)GP * kP2Tile) * sizeof(float);
+  if (p.proj.M) smem += (size_t)GP * kP2Tile * (p.d + 1) * sizeof(float);
   dim3 grid((p.n + kP2Tile - 1) / kP2Tile, p.BH);
   cudaError_t e;
   if (p.dtype == RESTKV_BF16) {
     if ((e = allow_smem(simt_pass2_kernel<__nv_bfloat16>, smem)) != cudaSuccess) return e;
     simt_pass2_kernel<__nv_bfloat16><<<grid, threads, smem, st>>>(
         p, (const __nv_bfloat16*)Q, (const __nv_bfloat16*)K, (const __nv_bfloat16*)V, ws.fin_m, ws.fin_l, ws.O_f32,
-        ema_decay, ws.I_hat, I_raw, GP);
+        ws.O_proj, ema_decay, ws.I_hat, I_raw, GP);
   } else {
     if ((e = allow_smem(simt_pass2_kernel<float>, smem)) != cudaSuccess) return e;
     simt_pass2_kernel<float><<<grid, threads, smem, st>>>(p, (const float*)Q, (const float*)K, (const float*)V,
-                                                          ws.fin_m, ws.fin_l, ws.O_f32, ema_decay, ws.I_hat, I_raw,
-                                                          GP);
+                                                          ws.fin_m, ws.fin_l, ws.O_f32, ws.O_proj, ema_decay,
+                                                          ws.I_hat, I_raw, GP);
   }
   return cudaGetLastError();
 }

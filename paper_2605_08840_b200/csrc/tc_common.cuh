@@ -58,6 +58,41 @@ __device__ __forceinline__ float exact_dist2_warp(const float* __restrict__ o_ro
   return ss;
 }
 
+// The same under the output projection: (o - v)^T Mt (o - v) = (o - v) . (Mt o - Mt v), Mt symmetric [128 x 128] fp32,
+// Mt o given (op_row).  Row k of Mt is read by the whole warp (coalesced) and weighted with v_k, which lane k / 4 holds.
+__device__ __forceinline__ float exact_proj_dist2_warp(const float* __restrict__ o_row, const float* __restrict__ op_row,
+                                                       const __nv_bfloat16* __restrict__ v_row,
+                                                       const float* __restrict__ Mt, int lane) {
+  const float4 o = *reinterpret_cast<const float4*>(o_row + lane * 4);
+  const float4 op = *reinterpret_cast<const float4*>(op_row + lane * 4);
+  const uint2 vv = *reinterpret_cast<const uint2*>(v_row + lane * 4);
+  const float v[4] = {__uint_as_float(vv.x << 16), __uint_as_float(vv.x & 0xFFFF0000u), __uint_as_float(vv.y << 16),
+                      __uint_as_float(vv.y & 0xFFFF0000u)};
+  float4 mv = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 2
+  for (int src = 0; src < 32; ++src) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float vk = __shfl_sync(0xffffffffu, v[e], src);
+      const float4 m = __ldg(reinterpret_cast<const float4*>(Mt + (src * 4 + e) * kHeadDim + lane * 4));
+      mv.x = fmaf(m.x, vk, mv.x); mv.y = fmaf(m.y, vk, mv.y); mv.z = fmaf(m.z, vk, mv.z); mv.w = fmaf(m.w, vk, mv.w);
+    }
+  }
+  float ss = ((o.x - v[0]) * (op.x - mv.x) + (o.y - v[1]) * (op.y - mv.y)) +
+             ((o.z - v[2]) * (op.z - mv.z) + (o.w - v[3]) * (op.w - mv.w));
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+  return fmaxf(ss, 0.f);
+}
+
+// After a wait has failed: wait (bounded, whatever the abort flag says) for a bulk copy or an MMA that this thread
+// itself set in motion, so that nothing is still writing this CTA's shared or tensor memory when it returns.
+__device__ __forceinline__ void wait_issued(uint64_t* bar, uint32_t parity) {
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity & 1u))
+    if (clock64() - t0 > 4000000000ll) return;
+}
+
 constexpr uint32_t kAugBytes = kBoxBytes;     // [128 rows x 64 bf16], only K steps 0 (S') and 1 (C') are used
 constexpr uint32_t kOnesBytes = 1024;         // one 8-row group of ones, shared by all 16 groups (stride 0)
 constexpr float kHeavyA = 0.125f;             // attention weight above which ||o - v||^2 is recomputed exactly

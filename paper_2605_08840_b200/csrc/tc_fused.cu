@@ -56,6 +56,12 @@ struct FusedArgs {
                                      //  Eq. 10-12; every tile then takes the slower epilogue that holds them
   const __nv_bfloat16* V;
   long long vsb, vsh, vsn;
+  // Output projection of Eq. 4 (all null without one): Eq. 7's squared norm becomes the quadratic form of Mt, the
+  // per-head matrices [Hq, 128, 128]; vmv [BH, G, n_kv] holds the tokens' own terms v^T Mt v (in place of ||v||^2),
+  // O_proj [BH, 128, 128] receives Mt o of the window rows.
+  const float* proj_Mt;
+  const float* vmv;
+  float* O_proj;
   unsigned int* counters;            // [groups] (at most 256), zero at launch
   unsigned int* dev_status;
   long long wait_limit;              // SM clocks a wait may last
@@ -98,14 +104,6 @@ __device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p) {
   unsigned int v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
-}
-
-// After a wait has failed: wait (bounded, whatever the abort flag says) for a bulk copy or an MMA that this thread
-// itself set in motion, so that nothing is still writing this CTA's shared or tensor memory when it returns.
-__device__ __forceinline__ void wait_issued(uint64_t* bar, uint32_t parity) {
-  const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity & 1u))
-    if (clock64() - t0 > 4000000000ll) return;
 }
 
 // (Re)initialises every mbarrier of the CTA for one phase.  Called by one thread between two __syncthreads.
@@ -491,6 +489,19 @@ __device__ void phase_a_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
   tc_fence_before();
 }
 
+// (Mt x) for a 128-vector x held in shared memory, Mt symmetric [128 x 128] fp32 in global memory: lane L returns
+// elements 4L .. 4L+3 (row k of Mt is read as a whole by the warp: coalesced).
+__device__ __forceinline__ float4 project_row_warp(const float* __restrict__ Mt, const float* x, int lane) {
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
+  for (int k = 0; k < kHeadDim; ++k) {
+    const float4 m = __ldg(reinterpret_cast<const float4*>(Mt + k * kHeadDim + lane * 4));
+    const float xk = x[k];
+    acc.x = fmaf(m.x, xk, acc.x); acc.y = fmaf(m.y, xk, acc.y); acc.z = fmaf(m.z, xk, acc.z); acc.w = fmaf(m.w, xk, acc.w);
+  }
+  return acc;
+}
+
 // x = hi + mid + lo with three bf16 pieces (24 significant bits).
 __device__ __forceinline__ void split3(float x, __nv_bfloat16* out) {
   const __nv_bfloat16 hi = __float2bfloat16_rn(x);
@@ -565,16 +576,32 @@ __device__ void combine_rows(const FusedArgs& a, int bh, int group, int r, int s
   const float4 o = make_float4(acc.x * inv_l, acc.y * inv_l, acc.z * inv_l, acc.w * inv_l);
   const long long ri = (long long)bh * kRows + r;
   *reinterpret_cast<float4*>(a.O_f32 + ri * kHeadDim + lane * 4) = o;
-  const __nv_bfloat16 b0 = __float2bfloat16_rn(o.x), b1 = __float2bfloat16_rn(o.y), b2 = __float2bfloat16_rn(o.z),
-                      b3 = __float2bfloat16_rn(o.w);
-  const float f0 = __bfloat162float(b0), f1 = __bfloat162float(b1), f2 = __bfloat162float(b2),
-              f3 = __bfloat162float(b3);
-  __nv_bfloat16* om = a.O_m2 + ri * kHeadDim + lane * 4;   // -2 x is exact for a bf16 x
-  om[0] = __float2bfloat16_rn(-2.f * f0);
-  om[1] = __float2bfloat16_rn(-2.f * f1);
-  om[2] = __float2bfloat16_rn(-2.f * f2);
-  om[3] = __float2bfloat16_rn(-2.f * f3);
-  float on = (f0 * f0 + f1 * f1) + (f2 * f2 + f3 * f3);
+  __nv_bfloat16* om = a.O_m2 + ri * kHeadDim + lane * 4;
+  float on;
+  if (a.proj_Mt) {
+    // with the output projection: the row of the third contraction is -2 bf16(Mt o), its constant o^T Mt o
+    __syncwarp();
+    *reinterpret_cast<float4*>(&xch[wq][lane * 4]) = o;   // the warp's own slot: its partials were merged above
+    __syncwarp();
+    const float4 mo = project_row_warp(a.proj_Mt + (long long)((bh % a.Hkv) * (kRows / a.w) + r / a.w) * kHeadDim * kHeadDim,
+                                       xch[wq], lane);
+    *reinterpret_cast<float4*>(a.O_proj + ri * kHeadDim + lane * 4) = mo;
+    om[0] = __float2bfloat16_rn(-2.f * mo.x);
+    om[1] = __float2bfloat16_rn(-2.f * mo.y);
+    om[2] = __float2bfloat16_rn(-2.f * mo.z);
+    om[3] = __float2bfloat16_rn(-2.f * mo.w);
+    on = (o.x * mo.x + o.y * mo.y) + (o.z * mo.z + o.w * mo.w);
+  } else {
+    const __nv_bfloat16 b0 = __float2bfloat16_rn(o.x), b1 = __float2bfloat16_rn(o.y), b2 = __float2bfloat16_rn(o.z),
+                        b3 = __float2bfloat16_rn(o.w);
+    const float f0 = __bfloat162float(b0), f1 = __bfloat162float(b1), f2 = __bfloat162float(b2),
+                f3 = __bfloat162float(b3);
+    om[0] = __float2bfloat16_rn(-2.f * f0);   // -2 x is exact for a bf16 x
+    om[1] = __float2bfloat16_rn(-2.f * f1);
+    om[2] = __float2bfloat16_rn(-2.f * f2);
+    om[3] = __float2bfloat16_rn(-2.f * f3);
+    on = (f0 * f0 + f1 * f1) + (f2 * f2 + f3 * f3);
+  }
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) on += __shfl_xor_sync(0xffffffffu, on, off);
   __nv_bfloat16* arow = a.aug + ri * 64;
@@ -753,7 +780,17 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
   };
   const float* O_head = a.O_f32 + (long long)bh * kRows * kHeadDim;
   const __nv_bfloat16* V_head = a.V + (long long)b * a.vsb + (long long)h * a.vsh;
-  const float* vn_head = a.vnorm + (long long)bh * a.n_kv;
+  // with the output projection the token's own term is v^T Mt v of the query head that this warpgroup's 32 columns
+  // belong to (w >= 32 there), and the exact distances go through that head's Mt
+  const int g_cols = (cgp * 32) / kW;
+  const float* vn_head = a.vmv ? a.vmv + ((long long)bh * kG + g_cols) * a.n_kv : a.vnorm + (long long)bh * a.n_kv;
+  const float* Mt_g = a.proj_Mt ? a.proj_Mt + (long long)(h * kG + g_cols) * kHeadDim * kHeadDim : nullptr;
+  const float* Op_head = a.proj_Mt ? a.O_proj + (long long)bh * kRows * kHeadDim : nullptr;
+  auto exact_dist2 = [&](int row, int js) {
+    const __nv_bfloat16* v_row = V_head + (long long)js * a.vsn;
+    return Mt_g ? exact_proj_dist2_warp(O_head + row * kHeadDim, Op_head + row * kHeadDim, v_row, Mt_g, lane)
+                : exact_dist2_warp(O_head + row * kHeadDim, v_row, lane);
+  };
   float* I_head = a.I_hat + (long long)bh * n;
   float* raw_head = (a.I_raw && !kLse) ? a.I_raw + (long long)bh * kRows * n : nullptr;
   bool ok = true;
@@ -771,9 +808,12 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
   // from_lse: no phase A has left ||v||^2 and the tiles' row maxima behind; ||v||^2 comes from the control warps
   // through shared memory and a warp finds out from the logits themselves whether its part of a tile is heavy
   constexpr bool from_lse = kLse;
-  if (T > 0 && !from_lse) {
+  const bool vn_global = !from_lse || a.vmv != nullptr;   // the token's own term is read from global memory
+  if (T > 0 && vn_global) {
     const int j = (tile0 + T - 1) * kTile + t;
     vn_next = (j < n) ? vn_head[j] : 1.f;
+  }
+  if (T > 0 && !from_lse) {
 #pragma unroll
     for (int k = 0; k < 4; ++k) tm_next[k] = tm_head[(long long)(tile0 + T - 1) * kRows + k * 32 + lane];
   }
@@ -789,11 +829,13 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
     if (from_lse) {
       ok = ok && mbar_wait(&B->vn_full[it & 3], (uint32_t)(it >> 2) & 1u, abort_flag, dev_status, kDevTimeout, a.wait_limit);
       const int jv = (tile0 + T - 1 - it) * kTile + t;
-      vn = (ok && jv < n) ? cx.vn_s[(it & 3) * kTile + t] : 1.f;
+      if (!vn_global) vn = (ok && jv < n) ? cx.vn_s[(it & 3) * kTile + t] : 1.f;
     }
-    if (it + 1 < T && !from_lse) {   // next tile's ||v||^2 and row maxima, well ahead of their use
+    if (it + 1 < T && vn_global) {   // next tile's ||v||^2 (or v^T Mt v), well ahead of its use
       const int jn = (tile0 + T - 2 - it) * kTile + t;
       vn_next = (jn < n) ? vn_head[jn] : 1.f;
+    }
+    if (it + 1 < T && !from_lse) {   // next tile's row maxima
 #pragma unroll
       for (int k = 0; k < 4; ++k) tm_next[k] = tm_head[(long long)(tile0 + T - 2 - it) * kRows + k * 32 + lane];
     }
@@ -890,8 +932,7 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
                 const int src = __ffs(todo) - 1;
                 todo &= todo - 1;
                 const int js = __shfl_sync(0xffffffffu, j, src);
-                const float d2x = exact_dist2_warp(O_head + (cgp * 32 + c * 8 + u) * kHeadDim,
-                                                   V_head + (long long)js * a.vsn, lane);
+                const float d2x = exact_dist2(cgp * 32 + c * 8 + u, js);
                 if (lane == src) x = d2x;
               }
               I[u] = x * rsqrt_approx(fmaf(x * um, um, 1e-36f));
@@ -927,8 +968,7 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
                 const int src = __ffs(todo) - 1;
                 todo &= todo - 1;
                 const int js = __shfl_sync(0xffffffffu, j, src);
-                const float d2x = exact_dist2_warp(O_head + (cgp * 32 + c * 8 + u) * kHeadDim,
-                                                   V_head + (long long)js * a.vsn, lane);
+                const float d2x = exact_dist2(cgp * 32 + c * 8 + u, js);
                 if (lane == src) x = d2x;
               }
               I[u] = x * rsqrt_approx(fmaf(x * um, um, 1e-36f));
@@ -1410,20 +1450,40 @@ tc_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 // ------------------------------------------------------------------------------------------------
 // The window rows' outputs O and log-sum-exps given by the caller (the prefill attention has them): what phase B
 // would have written for phase C.  One warp per query row, lane = four output dims.
+// With the output projection (proj_Mt non-null): the row becomes -2 bf16(Mt o), the constant o^T Mt o, and Mt o is
+// kept in O_proj.
 __global__ void from_lse_prep_kernel(int rows, float scale, const float* __restrict__ O, const float* __restrict__ LSE,
                                      __nv_bfloat16* __restrict__ O_m2, __nv_bfloat16* __restrict__ aug,
-                                     float* __restrict__ row_M2) {
-  const int ri = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+                                     float* __restrict__ row_M2, const float* __restrict__ proj_Mt,
+                                     float* __restrict__ O_proj, int Hkv, int w) {
+  __shared__ float xs[8][kHeadDim];
+  const int wi = threadIdx.x >> 5;
+  const int ri = blockIdx.x * (blockDim.x >> 5) + wi, lane = threadIdx.x & 31;
   if (ri >= rows) return;
   const float4 o = *reinterpret_cast<const float4*>(O + (long long)ri * kHeadDim + lane * 4);
-  const float f0 = __bfloat162float(__float2bfloat16_rn(o.x)), f1 = __bfloat162float(__float2bfloat16_rn(o.y));
-  const float f2 = __bfloat162float(__float2bfloat16_rn(o.z)), f3 = __bfloat162float(__float2bfloat16_rn(o.w));
-  __nv_bfloat16* om = O_m2 + (long long)ri * kHeadDim + lane * 4;   // -2 x is exact for a bf16 x
-  om[0] = __float2bfloat16_rn(-2.f * f0);
-  om[1] = __float2bfloat16_rn(-2.f * f1);
-  om[2] = __float2bfloat16_rn(-2.f * f2);
-  om[3] = __float2bfloat16_rn(-2.f * f3);
-  float on = (f0 * f0 + f1 * f1) + (f2 * f2 + f3 * f3);
+  __nv_bfloat16* om = O_m2 + (long long)ri * kHeadDim + lane * 4;
+  float on;
+  if (proj_Mt) {
+    *reinterpret_cast<float4*>(&xs[wi][lane * 4]) = o;
+    __syncwarp();
+    const int bh = ri / kRows, r = ri % kRows;
+    const float4 mo = project_row_warp(proj_Mt + (long long)((bh % Hkv) * (kRows / w) + r / w) * kHeadDim * kHeadDim,
+                                       xs[wi], lane);
+    *reinterpret_cast<float4*>(O_proj + (long long)ri * kHeadDim + lane * 4) = mo;
+    om[0] = __float2bfloat16_rn(-2.f * mo.x);
+    om[1] = __float2bfloat16_rn(-2.f * mo.y);
+    om[2] = __float2bfloat16_rn(-2.f * mo.z);
+    om[3] = __float2bfloat16_rn(-2.f * mo.w);
+    on = (o.x * mo.x + o.y * mo.y) + (o.z * mo.z + o.w * mo.w);
+  } else {
+    const float f0 = __bfloat162float(__float2bfloat16_rn(o.x)), f1 = __bfloat162float(__float2bfloat16_rn(o.y));
+    const float f2 = __bfloat162float(__float2bfloat16_rn(o.z)), f3 = __bfloat162float(__float2bfloat16_rn(o.w));
+    om[0] = __float2bfloat16_rn(-2.f * f0);   // -2 x is exact for a bf16 x
+    om[1] = __float2bfloat16_rn(-2.f * f1);
+    om[2] = __float2bfloat16_rn(-2.f * f2);
+    om[3] = __float2bfloat16_rn(-2.f * f3);
+    on = (f0 * f0 + f1 * f1) + (f2 * f2 + f3 * f3);
+  }
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) on += __shfl_xor_sync(0xffffffffu, on, off);
   __nv_bfloat16* arow = aug + (long long)ri * 64;
@@ -1490,7 +1550,8 @@ cudaError_t launch_from_lse_prep(const Problem& p, const Workspace& ws, const fl
                                  bool tensor_core, cudaStream_t st) {
   const int rows = p.BH * p.R;
   if (tensor_core)
-    from_lse_prep_kernel<<<(rows + 7) / 8, 256, 0, st>>>(rows, p.scale, O, LSE, ws.O_m2, ws.aug, ws.row_M2);
+    from_lse_prep_kernel<<<(rows + 7) / 8, 256, 0, st>>>(rows, p.scale, O, LSE, ws.O_m2, ws.aug, ws.row_M2, p.proj.Mt,
+                                                         ws.O_proj, p.Hkv, p.w);
   else
     from_lse_prep_simt_kernel<<<(rows + 255) / 256, 256, 0, st>>>(rows, LSE, ws.fin_m, ws.fin_l);
   return cudaGetLastError();
@@ -1613,6 +1674,9 @@ cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, 
     a.t_decay = 0.f; a.t_seed_first = a.t_seed_last = a.t_scale = 1.f;
   } else if (!temporal_chain(p.temporal, ema_decay, p.w, &a.t_decay, &a.t_seed_first, &a.t_seed_last, &a.t_scale)) {
     return cudaErrorInvalidValue;
+  }
+  if (p.proj.Mt && !attention_only) {
+    a.proj_Mt = p.proj.Mt; a.vmv = ws.vmv; a.O_proj = ws.O_proj;
   }
   a.group_max = p.group == RESTKV_GROUP_MAX ? 1 : 0;
   a.pool_max = p.spatial == RESTKV_SPATIAL_MAX ? 1 : 0;

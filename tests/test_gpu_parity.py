@@ -911,6 +911,163 @@ def test_reeviction_after_m_generated_tokens(handle, use_decode_statistics):
     assert_compaction_exact(idx2, vbits, run2._bits(run2.V_out))
 
 
+# ------------------------------------------------------------------ the output projection inside Eq. 7 (Eq. 4)
+def _make_projection(handle, case, d_model, seed, scale=1.0):
+    """(W float32 [Hq, d, d_model] holding dtype-exact values, factor buffer on the device)."""
+    import torch
+    from paper_2605_08840_b200.inputs import bf16_bits_to_f32
+    rng = np.random.default_rng(seed)
+    W = (rng.standard_normal((case.n_q_heads, case.head_dim, d_model)) * scale / np.sqrt(d_model)).astype(np.float32)
+    if case.dtype == "bf16":
+        bits = round_to_bf16_bits(W)
+        W = bf16_bits_to_f32(bits)
+        dW = torch_dev(bits.view(np.int16).reshape(-1, d_model), "bf16")
+    else:
+        dW = torch.from_numpy(W.reshape(-1, d_model)).cuda()
+    nbytes = handle.output_projection_bytes(case.n_q_heads, case.head_dim)
+    assert nbytes > 0
+    factor = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    handle.prepare_output_projection(case.n_q_heads, case.head_dim, d_model, rk.BF16 if case.dtype == "bf16" else rk.F32,
+                                     dW, factor)
+    torch.cuda.synchronize()
+    return W, factor
+
+
+def projection_check(handle, inp, d_model, path=rk.PATH_AUTO, seed=1, from_lse=False, variant=None, fused=None):
+    import torch
+    c = inp.case
+    W, factor = _make_projection(handle, c, d_model, seed)
+    handle.set_kernel_path(path)
+    handle.set_output_projection(factor, c.n_q_heads, c.head_dim)
+    if variant:
+        handle.set_variant(*variant)
+    try:
+        run = GpuRun(handle, inp)
+        if from_lse:
+            _, O, lse = _window_stats(inp, with_A_check=False)
+            handle.evict_from_lse(run.shape, run.Q, run.K, run.V, torch.from_numpy(O).cuda(),
+                                  torch.from_numpy(lse).cuda(), c.ema_decay, run.pool(), run.budget, run.indices,
+                                  run.K_out, run.V_out, run.ws, scores_out=run.scores)
+            torch.cuda.synchronize()
+            assert handle.poll_status() == rk.RESTKV_OK
+            scores, idx = run.scores.cpu().numpy(), run.indices.cpu().numpy()
+            K_out, V_out = run._bits(run.K_out), run._bits(run.V_out)
+        else:
+            scores, idx, K_out, V_out = run.evict()
+        if fused is not None:
+            assert handle.last_evict_fused_select() == fused
+    finally:
+        handle.set_kernel_path(rk.PATH_AUTO)
+        handle.set_output_projection(None)
+        handle.set_variant()
+    kw = {}
+    if variant:
+        kw = dict(indicator_mode=variant[0], temporal_mode=variant[1], spatial_mode=variant[2], group_mode=variant[3])
+    ref = oracle_scores(inp, W_O=W, **kw)
+    tol = TOL[c.dtype]
+    assert_scores_close(scores, ref.scores, tol)
+    assert_selection_valid(idx, ref.scores, run.budget, tol)
+    _, kbits, vbits = inp.device_arrays()
+    assert_compaction_exact(idx, kbits, K_out)
+    assert_compaction_exact(idx, vbits, V_out)
+    plain = oracle_scores(inp, **kw).scores
+    fin = np.isfinite(plain)
+    assert not np.allclose(ref.scores[fin], plain[fin], rtol=1e-2), "the projection changed nothing"
+    return ref
+
+
+@pytest.mark.parametrize("spec", [("f32", 64, 96), ("bf16", 128, 300), ("f32", 128, 64), ("bf16", 48, 48)])
+def test_projection_factor(handle, spec):
+    """M = W W^T, its Cholesky factor rounded to bf16 (stored transposed) and the product of the rounded factor."""
+    import torch
+    from paper_2605_08840_b200.inputs import bf16_bits_to_f32
+    dtype, d, d_model = spec
+    case = Case("proj", 1, 6, 2, d, 64, 4, 8, 1, 0, 0.9, dtype, 0, "normal", 3)
+    W, factor = _make_projection(handle, case, d_model, seed=9)
+    raw = factor.cpu().numpy()
+    dd = 6 * d * d
+    M = raw[:4 * dd].view(np.float32).reshape(6, d, d)
+    Mt = raw[4 * dd:8 * dd].view(np.float32).reshape(6, d, d)
+    LT = bf16_bits_to_f32(raw[8 * dd:10 * dd].view(np.uint16)).reshape(6, d, d)
+    M_ref = np.einsum("hik,hjk->hij", W.astype(np.float64), W.astype(np.float64))
+    np.testing.assert_allclose(M, M_ref, rtol=0, atol=2e-6 * np.abs(M_ref).max())
+    L = np.swapaxes(LT, 1, 2).astype(np.float64)
+    assert np.all(np.triu(L, 1) == 0)
+    np.testing.assert_allclose(Mt, L @ np.swapaxes(L, 1, 2), rtol=0, atol=2e-6 * np.abs(M_ref).max())
+    # the rounded factor reproduces M to bf16 accuracy, also where M is singular (d_model < d)
+    err = np.linalg.norm(Mt - M_ref, axis=(1, 2)) / np.linalg.norm(M_ref, axis=(1, 2))
+    assert err.max() < 2.0 ** -7
+
+
+@pytest.mark.parametrize("spec", [("cfg1b", "f32", 0, 96), ("cfg1b", "bf16", 32, 64), ("cfg1a", "f32", 0, 40)])
+def test_projection_on_the_simt_kernels(handle, spec):
+    name, dtype, tail, d_model = spec
+    projection_check(handle, make_inputs(CONFIGS[name].with_(dtype=dtype, causal_tail=tail)), d_model)
+
+
+@pytest.mark.parametrize("tail", [0, 32])
+@pytest.mark.parametrize("d_model", [256, 24])
+def test_projection_on_the_tensor_core_kernel(handle, tail, d_model):
+    # workload 2 has planted heavy hitters: entries with A > 1/8 take the exact (projected) distance
+    projection_check(handle, make_inputs(CONFIGS["cfg2"].with_(causal_tail=tail)), d_model, path=rk.PATH_TENSOR_CORE,
+                     fused=True)
+
+
+def test_projection_from_given_window_statistics(handle):
+    projection_check(handle, make_inputs(CONFIGS["cfg2"]), 192, path=rk.PATH_TENSOR_CORE, from_lse=True)
+
+
+@pytest.mark.parametrize("spec", [(4, 2, 64), (2, 2, 128), (16, 2, 16)])
+def test_projection_at_other_window_lengths(handle, spec):
+    """w = 64 and 128 run on the tensor-core kernel (two heads, one head per group); w = 16 has eight query heads per
+    KV head, more than the tensor-core path's four factor tiles, and runs on the SIMT kernels."""
+    Hq, Hkv, w = spec
+    case = Case("proj_w%d" % w, 2, Hq, Hkv, 128, 3000, w, 200, 5, 0, 0.9, "bf16", 0, "normal", 56)
+    projection_check(handle, make_inputs(case), 160, path=rk.PATH_TENSOR_CORE if w >= 32 else rk.PATH_AUTO)
+
+
+def test_projection_with_a_variant(handle):
+    inp = make_inputs(CONFIGS["cfg2"])
+    projection_check(handle, inp, 128, path=rk.PATH_TENSOR_CORE, variant=(REC, INV, rk.SPATIAL_MAX, rk.GROUP_MAX))
+
+
+def test_projection_is_ignored_by_the_attention_weight_indicators(handle):
+    inp = make_inputs(CONFIGS["cfg2"])
+    W, factor = _make_projection(handle, inp.case, 64, seed=4)
+    handle.set_output_projection(factor, inp.case.n_q_heads, inp.case.head_dim)
+    handle.set_variant(ATT, MEAN)
+    try:
+        scores, _, _, _ = GpuRun(handle, inp).evict()
+    finally:
+        handle.set_output_projection(None)
+        handle.set_variant()
+    ref = oracle_scores(inp, indicator_mode=ATT, temporal_mode=MEAN)
+    assert_scores_close(scores, ref.scores, TOL["bf16"])
+
+
+def test_projection_at_full_size(handle):
+    """The long-context workload with a rank-8 projection (d_model = 8 keeps the oracle's cost in bounds)."""
+    projection_check(handle, make_inputs(CONFIGS["cfg4"]), 8, fused=True)
+
+
+def test_projection_must_match_the_shape(handle):
+    import torch
+    inp = make_inputs(CONFIGS["cfg1b"])
+    c = inp.case
+    _, factor = _make_projection(handle, c, 32, seed=2)
+    run = GpuRun(handle, inp)
+    handle.set_output_projection(factor, c.n_q_heads + 8, c.head_dim)
+    try:
+        with pytest.raises(rk.RestKVError) as e:
+            handle.evict(run.shape, run.Q, run.K, run.V, 0.9, run.pool(), run.budget, run.indices, run.K_out, run.V_out,
+                         run.ws)
+        assert e.value.status == rk.ERR_INVALID_ARG
+    finally:
+        handle.set_output_projection(None)
+    assert handle.output_projection_bytes(8, 20) == 0 and handle.output_projection_bytes(8, 256) == 0
+    torch.cuda.synchronize()
+
+
 # ------------------------------------------------------------------ a device-side wait that runs out
 def test_wait_limit_runs_out_and_the_handle_recovers(handle):
     """With a wait limit of one SM clock the first CTA to reach a group barrier of the persistent score kernel gives
