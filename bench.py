@@ -552,6 +552,39 @@ def main():
                    "rows": rows, "evict_us": ms_a * 1e3, "evict_from_decode_statistics_us": ms_b * 1e3}
         del Kr, Vr, O_r, L_r, ws_r
 
+    # ---- the output projection inside Eq. 7's norm (Eq. 4): || (o - v) W_O ||, W_O random [Hq * d, 4096] ----
+    projection = None
+    if rank == 0 and case.dtype == "bf16":
+        d_model = 4096
+        Wp = (torch.randn(case.n_q_heads * case.head_dim, d_model, device="cuda", generator=torch.Generator("cuda").manual_seed(7))
+              / float(np.sqrt(d_model))).to(torch.bfloat16)
+        factor = torch.empty(handle.output_projection_bytes(case.n_q_heads, case.head_dim), dtype=torch.uint8, device="cuda")
+        ev0.record()
+        handle.prepare_output_projection(case.n_q_heads, case.head_dim, d_model, rk.BF16, Wp, factor)
+        ev1.record()
+        torch.cuda.synchronize()
+        prep_ms = ev0.elapsed_time(ev1)
+        handle.set_output_projection(factor, case.n_q_heads, case.head_dim)
+        try:
+            tp = []
+            for it in range(13):
+                flush.zero_()
+                ev0.record()
+                step()
+                ev1.record()
+                torch.cuda.synchronize()
+                if it >= 3:
+                    tp.append(ev0.elapsed_time(ev1))
+            pk = kernel_pass({"value_forms": rk.KERNEL_PASS1, "score_pool_select_compact": rk.KERNEL_PASS2}, 5)
+        finally:
+            handle.set_output_projection(None)
+        assert handle.poll_status() == rk.RESTKV_OK
+        projection = {"note": "restkv_evict with restkv_set_output_projection: the tokens' own quadratic forms v^T M v "
+                              "come from a tensor-core kernel of their own (one more read of V), the rest is the same launch",
+                      "d_model": d_model, "prepare_ms_once_per_layer": prep_ms, "evict_ms": float(np.median(tp)),
+                      "kernels_ms": pk}
+        del Wp, factor
+
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----
     e2e = None
     if not args.no_e2e:
@@ -624,7 +657,7 @@ def main():
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roofline, "path_roofline": path_roofline, "kernels_ms": kmean,
         "kernels_ms_selection_as_own_kernel": kmean_split, "decode": decode, "from_lse": from_lse,
-        "variants": variants, "adaptive_window": adaptive, "reevict": reevict,
+        "variants": variants, "adaptive_window": adaptive, "reevict": reevict, "output_projection": projection,
     }
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(inp, case.budget)

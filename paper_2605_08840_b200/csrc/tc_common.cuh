@@ -35,11 +35,14 @@ __device__ __forceinline__ uint64_t kmajor_desc(uint32_t addr) { return make_sme
 
 // D[128 x 128] (+)= A[128 x 128] * B[128 x 128]^T, both operands K-major 128B-swizzled [128 x 128] bf16 tiles
 // made of two [128 x 64] boxes.  One thread issues the eight K = 16 steps.
+// (The issuing thread's own instruction stream is what bounds a run of small products: the two descriptors are built
+// once and stepped by adding to their address field, which counts 16-byte units.)
 __device__ __forceinline__ void mma_tile_kk(uint32_t tmem_d, uint32_t a_smem, uint32_t b_smem, bool accumulate) {
+  const uint64_t a0 = kmajor_desc(a_smem), b0 = kmajor_desc(b_smem);
 #pragma unroll
   for (int k = 0; k < 8; ++k) {
-    const uint32_t off = (uint32_t)(k >> 2) * kBoxBytes + (uint32_t)(k & 3) * 32u;
-    umma_ss(tmem_d, kmajor_desc(a_smem + off), kmajor_desc(b_smem + off), kIdescKK, accumulate || k > 0);
+    const uint64_t step = (uint64_t)(((uint32_t)(k >> 2) * kBoxBytes + (uint32_t)(k & 3) * 32u) >> 4);
+    umma_ss(tmem_d, a0 + step, b0 + step, kIdescKK, accumulate || k > 0);
   }
 }
 
@@ -83,6 +86,22 @@ __device__ __forceinline__ float exact_proj_dist2_warp(const float* __restrict__
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
   return fmaxf(ss, 0.f);
+}
+
+// The expansion o^T Mt o - 2 (Mt o) . v + v^T Mt v in fp32 with exact dot products (vmv = v^T Mt v given): accurate
+// as long as the three terms do not nearly cancel, i.e. while o stays away from v.
+__device__ __forceinline__ float expanded_proj_dist2_warp(const float* __restrict__ o_row, const float* __restrict__ op_row,
+                                                          const __nv_bfloat16* __restrict__ v_row, float vmv, int lane) {
+  const float4 o = *reinterpret_cast<const float4*>(o_row + lane * 4);
+  const float4 op = *reinterpret_cast<const float4*>(op_row + lane * 4);
+  const uint2 vv = *reinterpret_cast<const uint2*>(v_row + lane * 4);
+  const float v0 = __uint_as_float(vv.x << 16), v1 = __uint_as_float(vv.x & 0xFFFF0000u);
+  const float v2 = __uint_as_float(vv.y << 16), v3 = __uint_as_float(vv.y & 0xFFFF0000u);
+  // o . (Mt o) - 2 v . (Mt o) = (o - 2 v) . (Mt o)
+  float ss = ((o.x - 2.f * v0) * op.x + (o.y - 2.f * v1) * op.y) + ((o.z - 2.f * v2) * op.z + (o.w - 2.f * v3) * op.w);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+  return fmaxf(ss + vmv, 0.f);
 }
 
 // After a wait has failed: wait (bounded, whatever the abort flag says) for a bulk copy or an MMA that this thread

@@ -517,6 +517,7 @@ __device__ __forceinline__ void split3(float x, __nv_bfloat16* out) {
 // `sub` of the row takes partials sub, sub + wpr, ...), whose sums meet in shared memory and are added in a fixed
 // order: the result does not depend on timing.  Written for phase C: O (fp32), -2 bf16(O), and the row's strip
 // of bf16 constant pieces.  Called by all sixteen worker warps; r < 0 means this warp has no row.
+template <bool kProj>
 __device__ void combine_rows(const FusedArgs& a, int bh, int group, int r, int sub, int wpr, int wq, int lane,
                              float (*xch)[kHeadDim + 4]) {
   float m = -INFINITY, l = 0.f;
@@ -578,7 +579,7 @@ __device__ void combine_rows(const FusedArgs& a, int bh, int group, int r, int s
   *reinterpret_cast<float4*>(a.O_f32 + ri * kHeadDim + lane * 4) = o;
   __nv_bfloat16* om = a.O_m2 + ri * kHeadDim + lane * 4;
   float on;
-  if (a.proj_Mt) {
+  if (kProj) {
     // with the output projection: the row of the third contraction is -2 bf16(Mt o), its constant o^T Mt o
     __syncwarp();
     *reinterpret_cast<float4*>(&xch[wq][lane * 4]) = o;   // the warp's own slot: its partials were merged above
@@ -737,12 +738,14 @@ __device__ void phase_c_control(const Ctx& cx, const FusedArgs& a, const CUtenso
   }
 }
 
-// kInd: 0 = Eq. 7; 1 = the attention weight alone; 2 = attention weight times ||v|| (Appendix G.1).
+// kInd: 0 = Eq. 7; 1 = the attention weight alone; 2 = attention weight times ||v|| (Appendix G.1); 3 = Eq. 7 with
+// the output projection of Eq. 4 inside its norm.
 template <int kW, bool kLse, int kInd>
 __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensorMap* tmO, const CUtensorMap* tmAug,
                         const CUtensorMap* tmK, const CUtensorMap* tmV, int bh, int tile0, int T, int pre,
                         float (*red)[4][kTile]) {
   constexpr int kG = kRows / kW;
+  constexpr bool kEq7 = kInd == 0 || kInd == 3, kProj = kInd == 3;
   FusedBars* B = cx.B;
   int* abort_flag = cx.abort_flag;
   unsigned int* dev_status = a.dev_status;
@@ -783,13 +786,17 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
   // with the output projection the token's own term is v^T Mt v of the query head that this warpgroup's 32 columns
   // belong to (w >= 32 there), and the exact distances go through that head's Mt
   const int g_cols = (cgp * 32) / kW;
-  const float* vn_head = a.vmv ? a.vmv + ((long long)bh * kG + g_cols) * a.n_kv : a.vnorm + (long long)bh * a.n_kv;
-  const float* Mt_g = a.proj_Mt ? a.proj_Mt + (long long)(h * kG + g_cols) * kHeadDim * kHeadDim : nullptr;
-  const float* Op_head = a.proj_Mt ? a.O_proj + (long long)bh * kRows * kHeadDim : nullptr;
-  auto exact_dist2 = [&](int row, int js) {
+  const float* vn_head = kProj ? a.vmv + ((long long)bh * kG + g_cols) * a.n_kv : a.vnorm + (long long)bh * a.n_kv;
+  const float* Mt_g = kProj ? a.proj_Mt + (long long)(h * kG + g_cols) * kHeadDim * kHeadDim : nullptr;
+  const float* Op_head = kProj ? a.O_proj + (long long)bh * kRows * kHeadDim : nullptr;
+  // S' above this <=> A > 0.9: under the projection only those entries take the exact quadratic form; the others
+  // above kHeavyA take its expansion in fp32 from exact dot products, which is accurate while 1 - A is not small
+  const float extreme_thr = log2f(1.f / 0.9f) / neg_c2;
+  auto exact_dist2 = [&](int row, int js, bool extreme) {
     const __nv_bfloat16* v_row = V_head + (long long)js * a.vsn;
-    return Mt_g ? exact_proj_dist2_warp(O_head + row * kHeadDim, Op_head + row * kHeadDim, v_row, Mt_g, lane)
-                : exact_dist2_warp(O_head + row * kHeadDim, v_row, lane);
+    if (!kProj) return exact_dist2_warp(O_head + row * kHeadDim, v_row, lane);
+    if (extreme) return exact_proj_dist2_warp(O_head + row * kHeadDim, Op_head + row * kHeadDim, v_row, Mt_g, lane);
+    return expanded_proj_dist2_warp(O_head + row * kHeadDim, Op_head + row * kHeadDim, v_row, vn_head[js], lane);
   };
   float* I_head = a.I_hat + (long long)bh * n;
   float* raw_head = (a.I_raw && !kLse) ? a.I_raw + (long long)bh * kRows * n : nullptr;
@@ -808,7 +815,7 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
   // from_lse: no phase A has left ||v||^2 and the tiles' row maxima behind; ||v||^2 comes from the control warps
   // through shared memory and a warp finds out from the logits themselves whether its part of a tile is heavy
   constexpr bool from_lse = kLse;
-  const bool vn_global = !from_lse || a.vmv != nullptr;   // the token's own term is read from global memory
+  const bool vn_global = !from_lse || kProj;   // the token's own term is read from global memory
   if (T > 0 && vn_global) {
     const int j = (tile0 + T - 1) * kTile + t;
     vn_next = (j < n) ? vn_head[j] : 1.f;
@@ -824,7 +831,7 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
     float vn = vn_next;
     // only Eq. 7 has the factor 1 / (1 - A) and the distance that need the exact form near A = 1
     const bool tile_heavy = raw_head != nullptr ||
-                            (kInd == 0 && __any_sync(0xffffffffu, tm_next[0] > m2r[0] || tm_next[1] > m2r[1] ||
+                            (kEq7 && __any_sync(0xffffffffu, tm_next[0] > m2r[0] || tm_next[1] > m2r[1] ||
                                                                       tm_next[2] > m2r[2] || tm_next[3] > m2r[3]));
     if (from_lse) {
       ok = ok && mbar_wait(&B->vn_full[it & 3], (uint32_t)(it >> 2) & 1u, abort_flag, dev_status, kDevTimeout, a.wait_limit);
@@ -864,10 +871,10 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
       float sv0[16], cv0[16], sv1[16], cv1[16];
       if (!tile_heavy) {
         tmem_ld16(tS, sv0);
-        if (kInd == 0) tmem_ld16(tC, cv0);
+        if (kEq7) tmem_ld16(tC, cv0);
         tmem_wait_ld();
         tmem_ld16(tS + 16, sv1);   // the second half of the columns travels while the first is worked on
-        if (kInd == 0) tmem_ld16(tC + 16, cv1);
+        if (kEq7) tmem_ld16(tC + 16, cv1);
       }
       bool redo_heavy = false;   // from_lse: this warp found a weight above kHeavyA among the logits it holds
       if (!tile_heavy) {
@@ -881,7 +888,7 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&B->acc_empty[s]);
-            if (from_lse && kInd == 0) {
+            if (from_lse && kEq7) {
               // no pass 1 has flagged the tiles with large weights: the warp looks at the logits it now holds in
               // registers (S' above heavy_thr <=> A > kHeavyA) and, if it finds one, does its part of the tile again
               // below with exact distances, from those registers (the accumulators are already released)
@@ -896,7 +903,7 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
           for (int q = 0; q < 8; ++q) {
             const f32x2 nt = f2_mul(f2_make(sv[2 * q], sv[2 * q + 1]), nc2);
             f32x2 Iq;
-            if (kInd == 0) {
+            if (kEq7) {
               const f32x2 um = f2_add(f2_make(ex2_approx(f2_lo(nt)), ex2_approx(f2_hi(nt))), m1);   // 1/A - 1
               const f32x2 x = f2_add(f2_make(cv[2 * q], cv[2 * q + 1]), vn2);                       // ||o - v||^2
               const f32x2 bq = f2_fma(f2_mul(x, um), um, tiny2);                                    // x (1/A - 1)^2
@@ -915,7 +922,7 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
             h2 = f2_make(0.f, 0.f);
           }
         }
-        if (from_lse && kInd == 0 && redo_heavy) {
+        if (from_lse && kEq7 && redo_heavy) {
           tot = 0.f;
           h2 = f2_make(0.f, 0.f);
 #pragma unroll
@@ -932,7 +939,7 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
                 const int src = __ffs(todo) - 1;
                 todo &= todo - 1;
                 const int js = __shfl_sync(0xffffffffu, j, src);
-                const float d2x = exact_dist2(cgp * 32 + c * 8 + u, js);
+                const float d2x = exact_dist2(cgp * 32 + c * 8 + u, js, __shfl_sync(0xffffffffu, sv[u] > extreme_thr, src) != 0);
                 if (lane == src) x = d2x;
               }
               I[u] = x * rsqrt_approx(fmaf(x * um, um, 1e-36f));
@@ -959,7 +966,7 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
           tmem_wait_ld();
 #pragma unroll
           for (int u = 0; u < 8; ++u) {
-            if (kInd == 0) {
+            if (kEq7) {
               const float um = ex2_approx(sv[u] * neg_c2) - 1.f;
               float x = cv[u] + vnb;
               // the whole warp computes the exact distance of each of its lanes' heavy entries in turn
@@ -968,7 +975,7 @@ __device__ void phase_c_worker(const Ctx& cx, const FusedArgs& a, const CUtensor
                 const int src = __ffs(todo) - 1;
                 todo &= todo - 1;
                 const int js = __shfl_sync(0xffffffffu, j, src);
-                const float d2x = exact_dist2(cgp * 32 + c * 8 + u, js);
+                const float d2x = exact_dist2(cgp * 32 + c * 8 + u, js, __shfl_sync(0xffffffffu, sv[u] > extreme_thr, src) != 0);
                 if (lane == src) x = d2x;
               }
               I[u] = x * rsqrt_approx(fmaf(x * um, um, 1e-36f));
@@ -1354,7 +1361,7 @@ __device__ void worker_main(const Ctx& cx, const FusedArgs& a, const Plan& pl, c
       float (*xch)[kHeadDim + 4] = reinterpret_cast<float (*)[kHeadDim + 4]>(cx.gen_base + kOffAug);
       for (int k0 = 0; k0 < rows_max; k0 += rows_at_once) {
         const int r = pl.rank + (k0 + wq / wpr) * a.cpg;
-        combine_rows(a, bh, pl.group, r < kRows ? r : -1, wq % wpr, wpr, wq, cx.lane, xch);
+        combine_rows<kInd == 3>(a, bh, pl.group, r < kRows ? r : -1, wq % wpr, wpr, wq, cx.lane, xch);
         named_barrier_sync(2, kFWorkerWarps * 32);   // the exchange buffer is reused by the next batch of rows
       }
       fence_proxy_async_smem();   // the exchange buffer is overwritten by a TMA load in phase C
@@ -1591,15 +1598,18 @@ template <int kW>
 static FusedKernel pick_fused_w(bool from_lse, int indicator) {
   if (from_lse) {
     if (indicator == 0) return tc_fused_kernel<kW, true, 0>;
+    if (indicator == 3) return tc_fused_kernel<kW, true, 3>;
     return indicator == 1 ? tc_fused_kernel<kW, true, 1> : tc_fused_kernel<kW, true, 2>;
   }
   if (indicator == 0) return tc_fused_kernel<kW, false, 0>;
+  if (indicator == 3) return tc_fused_kernel<kW, false, 3>;
   return indicator == 1 ? tc_fused_kernel<kW, false, 1> : tc_fused_kernel<kW, false, 2>;
 }
 
-// The instantiation for a window length (it only matters to phase C), input form and indicator; null if there is none.
+// The instantiation for a window length (it only matters to phase C), input form and indicator (3: Eq. 7 under the
+// output projection); null if there is none.
 static FusedKernel pick_fused(int w, bool from_lse, int indicator) {
-  if (indicator < 0 || indicator > 2) return nullptr;
+  if (indicator < 0 || indicator > 3) return nullptr;
   switch (w) {
     case 16: return pick_fused_w<16>(from_lse, indicator);
     case 32: return pick_fused_w<32>(from_lse, indicator);
@@ -1614,7 +1624,7 @@ cudaError_t tc_fused_init() {
   const int widths[4] = {16, 32, 64, 128};
   for (int w : widths)
     for (int lse = 0; lse < 2; ++lse)
-      for (int ind = 0; ind < 3; ++ind) {
+      for (int ind = 0; ind < 4; ++ind) {
         FusedKernel kernel = pick_fused(w, lse != 0, ind);
         if (e == cudaSuccess) e = check_launch_regs(kernel);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmem);
@@ -1702,7 +1712,7 @@ cudaError_t launch_tc_fused(void* state, const Problem& p, const Workspace& ws, 
     if (e != cudaSuccess) return e;
   }
   const dim3 grid(a.groups * a.cpg), block(kFThreads);
-  FusedKernel kernel = attention_only ? pick_fused(32, false, 0) : pick_fused(p.w, a.from_lse != 0, p.indicator);
+  FusedKernel kernel = attention_only ? pick_fused(32, false, 0) : pick_fused(p.w, a.from_lse != 0, a.proj_Mt ? 3 : p.indicator);
   if (!kernel) return cudaErrorInvalidValue;
   kernel<<<grid, block, kFSmem, st>>>(tmQ, tmK, tmV, tmO, tmAug, a);
   return cudaGetLastError();

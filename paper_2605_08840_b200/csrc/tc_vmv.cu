@@ -6,9 +6,14 @@
 // 128-column accumulator per query head), then the row sums of squares.  One CTA per SM over an equal, contiguous
 // share of the (head, tile) pairs; CTAs do not wait for one another.
 //   warp 0     TMA: the head's G factor tiles L_g^T [128 x 128] bf16 (reloaded when the share enters a new head),
-//              then the V tiles through a ring of two
-//   warp 1     MMA issue: for each tile G products, each committed to its accumulator's barrier
-//   warps 2-5  read-out: thread = token (tensor-memory lane), 128 columns squared and summed per query head
+//              then the V tiles through a ring that takes the rest of shared memory (three to six tiles: the loads
+//              are latency-bound, so every tile in flight counts)
+//   warp 1     MMA issue: for each tile G products, each committed to its accumulator's barrier.  L_g is lower
+//              triangular: the K step over dims 16 s .. 16 s + 15 only reaches output columns below 16 (s + 1), so
+//              the steps are issued from the last (all 128 columns, which also initialises the accumulator) to
+//              the first (16 columns): 56 % of the full product's tensor cycles
+//   warps 2-17 read-out: thread = token (tensor-memory lane), 128 columns squared and summed; each of the four warps
+//              of a lane quarter takes one query head
 // Every wait is bounded; after a failed wait the roles stop, wait for what they issued and the CTA returns.
 #include "tc_common.cuh"
 
@@ -16,13 +21,14 @@ namespace restkv {
 
 namespace {
 
-constexpr int kVThreads = 192;
-constexpr int kVRing = 2;
+constexpr int kVThreads = 576;
 constexpr int kVMaxG = 4;
-constexpr size_t kVSmem = (size_t)(kVMaxG + kVRing) * kTileBytes + 1024;
+constexpr int kVTiles = 7;                 // factor tiles + ring slots: 224 KB
+constexpr int kVMaxRing = kVTiles - 1;
+constexpr size_t kVSmem = (size_t)kVTiles * kTileBytes + 1024;
 
 struct VmvBars {
-  uint64_t lt_full, v_full[kVRing], v_empty[kVRing], acc_full[kVMaxG], acc_empty[kVMaxG], drain;
+  uint64_t lt_full, v_full[kVMaxRing], v_empty[kVMaxRing], acc_full[kVMaxG], acc_empty[kVMaxG], drain;
 };
 
 struct VmvArgs {
@@ -47,7 +53,8 @@ vmv_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUte
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t off_v = kVMaxG * kTileBytes;   // the ring follows the factor tiles
+  const uint32_t off_v = (uint32_t)a.G * kTileBytes;   // the ring follows the factor tiles
+  const int kVRing = kVTiles - a.G;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   VmvBars* B = &bars;
   unsigned int* dev_status = a.dev_status;
@@ -55,13 +62,13 @@ vmv_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUte
   if (threadIdx.x == 0) {
     abort_flag = 0;
     mbar_init(&B->lt_full, 1);
-    for (int i = 0; i < kVRing; ++i) {
+    for (int i = 0; i < kVMaxRing; ++i) {
       mbar_init(&B->v_full[i], 1);
       mbar_init(&B->v_empty[i], 1);
     }
     for (int g = 0; g < kVMaxG; ++g) {
       mbar_init(&B->acc_full[g], 1);
-      mbar_init(&B->acc_empty[g], 4);   // the four read-out warps
+      mbar_init(&B->acc_empty[g], 4);   // the four read-out warps (one per lane quarter) that take this query head
     }
     mbar_init(&B->drain, 1);
     fence_mbar_init();
@@ -136,8 +143,15 @@ vmv_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUte
             ok = mbar_wait(&B->acc_empty[g], (uint32_t)(it - 1) & 1u, &abort_flag, dev_status, kDevTimeout, a.wait_limit);
           if (!ok) break;
           tc_fence_after();
-          mma_tile_kk(tmem + (uint32_t)g * 128u, smem_base + off_v + (uint32_t)s * kTileBytes,
-                      smem_base + (uint32_t)g * kTileBytes, false);
+          const uint32_t a_smem = smem_base + off_v + (uint32_t)s * kTileBytes, b_smem = smem_base + (uint32_t)g * kTileBytes;
+          // (one thread issues 8 G products per tile: its instruction stream is the bound, so the descriptors are
+          // built once and stepped by adding to their address field, which counts 16-byte units)
+          const uint64_t a0 = kmajor_desc(a_smem), b0 = kmajor_desc(b_smem);
+#pragma unroll
+          for (int k = 7; k >= 0; --k) {
+            const uint64_t step = (uint64_t)(((uint32_t)(k >> 2) * kBoxBytes + (uint32_t)(k & 3) * 32u) >> 4);
+            umma_ss(tmem + (uint32_t)g * 128u, a0 + step, b0 + step, make_idesc_bf16(128, 16 * (k + 1), false), k < 7);
+          }
           umma_commit(&B->acc_full[g]);
         }
         if (ok) umma_commit(&B->v_empty[s]);   // the tile's slot is free once its last product has read it
@@ -149,6 +163,7 @@ vmv_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUte
     }
   } else {
     const int quad = warp & 3;   // the tensor-memory lane quarter this warp may touch
+    const int g_first = (warp - 2) >> 2;
     const int t = quad * 32 + lane;
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
     bool ok = true;
@@ -156,28 +171,25 @@ vmv_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUte
       const long long idx = first + it;
       const int bh = (int)(idx / a.tiles), tile = (int)(idx % a.tiles);
       const int j = tile * kTile + t;
-      for (int g = 0; g < a.G && ok; ++g) {
+      for (int g = g_first; g < a.G && ok; g += 4) {
         ok = mbar_wait(&B->acc_full[g], (uint32_t)it & 1u, &abort_flag, dev_status, kDevTimeout, a.wait_limit);
         float sum = 0.f;
         if (ok) {
           tc_fence_after();
           const uint32_t tY = tmem + lane_base + (uint32_t)g * 128u;
-          float y0[16], y1[16];
-          tmem_ld16(tY, y0);
 #pragma unroll
-          for (int c = 0; c < 8; c += 2) {
+          for (int c = 0; c < 2; ++c) {
+            float y0[32], y1[32];
+            tmem_ld32(tY + (uint32_t)c * 64u, y0);
+            tmem_ld32(tY + (uint32_t)c * 64u + 32u, y1);
             tmem_wait_ld();
-            tmem_ld16(tY + (uint32_t)(c + 1) * 16u, y1);   // travels while y0 is summed
-            float s0 = 0.f, s1 = 0.f;
+            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-            for (int u = 0; u < 16; u += 2) { s0 = fmaf(y0[u], y0[u], s0); s1 = fmaf(y0[u + 1], y0[u + 1], s1); }
-            sum += s0 + s1;
-            tmem_wait_ld();
-            if (c + 2 < 8) tmem_ld16(tY + (uint32_t)(c + 2) * 16u, y0);
-            s0 = 0.f; s1 = 0.f;
-#pragma unroll
-            for (int u = 0; u < 16; u += 2) { s0 = fmaf(y1[u], y1[u], s0); s1 = fmaf(y1[u + 1], y1[u + 1], s1); }
-            sum += s0 + s1;
+            for (int u = 0; u < 32; u += 2) {
+              s0 = fmaf(y0[u], y0[u], s0); s1 = fmaf(y0[u + 1], y0[u + 1], s1);
+              s2 = fmaf(y1[u], y1[u], s2); s3 = fmaf(y1[u + 1], y1[u + 1], s3);
+            }
+            sum += (s0 + s1) + (s2 + s3);
           }
           tc_fence_before();
         }
