@@ -3,15 +3,16 @@
 // without one).  It does not depend on the queries.
 //
 // Per 128-token tile: Y_g = V_tile L_g on the tensor cores (tcgen05, fp32 accumulators in tensor memory, one
-// 128-column accumulator per query head), then the row sums of squares.  One CTA per SM over an equal, contiguous
+// 128-column accumulator per query head; two query heads share one product of N = 256, their factor tiles lying
+// behind one another in shared memory), then the row sums of squares.  One CTA per SM over an equal, contiguous
 // share of the (head, tile) pairs; CTAs do not wait for one another.
 //   warp 0     TMA: the head's G factor tiles L_g^T [128 x 128] bf16 (reloaded when the share enters a new head),
 //              then the V tiles through a ring that takes the rest of shared memory (three to six tiles: the loads
 //              are latency-bound, so every tile in flight counts)
-//   warp 1     MMA issue: for each tile G products, each committed to its accumulator's barrier.  L_g is lower
-//              triangular: the K step over dims 16 s .. 16 s + 15 only reaches output columns below 16 (s + 1), so
-//              the steps are issued from the last (all 128 columns, which also initialises the accumulator) to
-//              the first (16 columns): 56 % of the full product's tensor cycles
+//   warp 1     MMA issue: for each tile one product per pair of query heads (eight K = 16 steps of N = 256; N = 128
+//              with a single head), each committed to the pair's barrier.  A step costs the issuing thread and the
+//              tensor pipe about as much at N = 64 as at N = 128, so fewer, wider steps are what pays (narrowing
+//              the steps to the triangular factor's non-zero columns did not)
 //   warps 2-17 read-out: thread = token (tensor-memory lane), 128 columns squared and summed; each of the four warps
 //              of a lane quarter takes one query head
 // Every wait is bounded; after a failed wait the roles stop, wait for what they issued and the CTA returns.
@@ -55,6 +56,8 @@ vmv_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUte
   uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
   const uint32_t off_v = (uint32_t)a.G * kTileBytes;   // the ring follows the factor tiles
   const int kVRing = kVTiles - a.G;
+  const uint32_t half_stride = a.G >= 2 ? kTileBytes : kBoxBytes;   // distance of a factor operand's two K halves
+  const int pairs = (a.G + 1) / 2;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   VmvBars* B = &bars;
   unsigned int* dev_status = a.dev_status;
@@ -67,8 +70,8 @@ vmv_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUte
       mbar_init(&B->v_empty[i], 1);
     }
     for (int g = 0; g < kVMaxG; ++g) {
-      mbar_init(&B->acc_full[g], 1);
-      mbar_init(&B->acc_empty[g], 4);   // the four read-out warps (one per lane quarter) that take this query head
+      mbar_init(&B->acc_full[g], 1);    // indexed by pair of query heads
+      mbar_init(&B->acc_empty[g], a.G >= 2 ? 8 : 4);   // the read-out warps of the pair: four lane quarters per head
     }
     mbar_init(&B->drain, 1);
     fence_mbar_init();
@@ -102,10 +105,12 @@ vmv_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUte
           if (ok) {
             mbar_arrive_expect_tx(&B->lt_full, (uint32_t)a.G * kTileBytes);
             for (int g = 0; g < a.G; ++g) {
+              // a pair's tiles interleave by K half: [half 0: head 2p, head 2p+1][half 1: head 2p, head 2p+1], so
+              // that each half is one K-major operand of 256 rows
               const int hq = (bh % a.Hkv) * a.G + g;
-              uint8_t* dst = gen_base + (uint32_t)g * kTileBytes;
+              uint8_t* dst = gen_base + (uint32_t)(g >> 1) * 2u * kTileBytes + (uint32_t)(g & 1) * kBoxBytes;
               tma_load_3d(dst, &tmLT, &B->lt_full, 0, 0, hq);
-              tma_load_3d(dst + kBoxBytes, &tmLT, &B->lt_full, 64, 0, hq);
+              tma_load_3d(dst + half_stride, &tmLT, &B->lt_full, 64, 0, hq);
             }
             ++heads_seen;
             prev_bh = bh;
@@ -138,21 +143,23 @@ vmv_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUte
           prev_bh = bh;
         }
         ok = ok && mbar_wait(&B->v_full[s], (uint32_t)(it / kVRing) & 1u, &abort_flag, dev_status, kDevTimeout, a.wait_limit);
-        for (int g = 0; g < a.G && ok; ++g) {
+        for (int pr = 0; pr < pairs && ok; ++pr) {
           if (it > 0)
-            ok = mbar_wait(&B->acc_empty[g], (uint32_t)(it - 1) & 1u, &abort_flag, dev_status, kDevTimeout, a.wait_limit);
+            ok = mbar_wait(&B->acc_empty[pr], (uint32_t)(it - 1) & 1u, &abort_flag, dev_status, kDevTimeout, a.wait_limit);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t a_smem = smem_base + off_v + (uint32_t)s * kTileBytes, b_smem = smem_base + (uint32_t)g * kTileBytes;
-          // (one thread issues 8 G products per tile: its instruction stream is the bound, so the descriptors are
-          // built once and stepped by adding to their address field, which counts 16-byte units)
+          const uint32_t a_smem = smem_base + off_v + (uint32_t)s * kTileBytes;
+          const uint32_t b_smem = smem_base + (uint32_t)pr * 2u * kTileBytes;
+          // the descriptors are built once and stepped by adding to their address field (16-byte units)
           const uint64_t a0 = kmajor_desc(a_smem), b0 = kmajor_desc(b_smem);
+          const uint32_t idesc = a.G >= 2 ? make_idesc_bf16(128, 256, false) : make_idesc_bf16(128, 128, false);
 #pragma unroll
-          for (int k = 7; k >= 0; --k) {
-            const uint64_t step = (uint64_t)(((uint32_t)(k >> 2) * kBoxBytes + (uint32_t)(k & 3) * 32u) >> 4);
-            umma_ss(tmem + (uint32_t)g * 128u, a0 + step, b0 + step, make_idesc_bf16(128, 16 * (k + 1), false), k < 7);
+          for (int k = 0; k < 8; ++k) {
+            const uint64_t a_step = (uint64_t)(((uint32_t)(k >> 2) * kBoxBytes + (uint32_t)(k & 3) * 32u) >> 4);
+            const uint64_t b_step = (uint64_t)(((uint32_t)(k >> 2) * half_stride + (uint32_t)(k & 3) * 32u) >> 4);
+            umma_ss(tmem + (uint32_t)pr * 256u, a0 + a_step, b0 + b_step, idesc, k > 0);
           }
-          umma_commit(&B->acc_full[g]);
+          umma_commit(&B->acc_full[pr]);
         }
         if (ok) umma_commit(&B->v_empty[s]);   // the tile's slot is free once its last product has read it
       }
@@ -172,7 +179,7 @@ vmv_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUte
       const int bh = (int)(idx / a.tiles), tile = (int)(idx % a.tiles);
       const int j = tile * kTile + t;
       for (int g = g_first; g < a.G && ok; g += 4) {
-        ok = mbar_wait(&B->acc_full[g], (uint32_t)it & 1u, &abort_flag, dev_status, kDevTimeout, a.wait_limit);
+        ok = mbar_wait(&B->acc_full[g >> 1], (uint32_t)it & 1u, &abort_flag, dev_status, kDevTimeout, a.wait_limit);
         float sum = 0.f;
         if (ok) {
           tc_fence_after();
@@ -194,7 +201,7 @@ vmv_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUte
           tc_fence_before();
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(&B->acc_empty[g]);
+        if (lane == 0) mbar_arrive(&B->acc_empty[g >> 1]);
         if (ok && j < a.n_kv) a.out[((long long)bh * a.G + g) * a.n_kv + j] = sum;
       }
     }
