@@ -72,7 +72,7 @@ def whole_job_value(tokens_per_rank_step, world, steps, total_ms):
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from an ncu capture
 # of this workload, together with the digest of the kernel sources the capture was taken on: the figure is reported
 # only while those sources are unchanged, otherwise `traffic` is null.
-KERNEL_TRAFFIC = {"cfg4": {"bytes": 1027409664 + 26176256, "sources_sha256": "595146513b8956870b53db3635e0ce99c42d3f6c9114f6dc45ba2ce04fc327a4"}}
+KERNEL_TRAFFIC = {"cfg4": {"bytes": 1024809984 + 27120896, "sources_sha256": "17e3ec72af554e0aebc6eeff775d86a85b19c7550b16ef355da76ebcd708b551"}}
 KERNEL_SOURCES = ("tc_fused.cu", "tc_common.cuh", "sm100_ptx.cuh")
 
 
@@ -249,6 +249,9 @@ def main():
     ap.add_argument("--workload", default="cfg4")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the timings beside the headline that came with the variants, the adaptive window, "
+                         "re-eviction and the output projection (short runs under a profiler)")
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 force SIMT, 2 require tensor cores")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -452,7 +455,7 @@ def main():
 
     # ---- the ablation variants of Appendix G as modes of the same path (beside the headline) ----
     variants = None
-    if rank == 0:
+    if rank == 0 and not args.no_extras:
         labelled = (("attention_weight__mean_over_window", (rk.INDICATOR_ATTENTION, rk.TEMPORAL_MEAN, 0, 0)),
                     ("attention_weight_times_value_norm__ema", (rk.INDICATOR_ATTENTION_VNORM, rk.TEMPORAL_EMA, 0, 0)),
                     ("reconstruction__inverted_ema__max_pool__group_max",
@@ -478,7 +481,7 @@ def main():
 
     # ---- the adaptive window of Eq. 10-12 (per-query top-B of the raw indicator, D_front / D_rear) ----
     adaptive = None
-    if rank == 0:
+    if rank == 0 and not args.no_extras:
         apool = rk.adaptive_pool(2000.0, case.width, case.budget)
         ws_a = torch.empty(handle.workspace_bytes(shape, case.budget, adaptive=True), dtype=torch.uint8, device="cuda")
 
@@ -509,7 +512,7 @@ def main():
     # ---- eviction again during decoding (Appendix B): the compacted cache plus M generated tokens, the last w of
     #      them as the window (their own rows are the trailing, causally masked block) ----
     reevict = None
-    if rank == 0 and case.causal_tail == 0 and case.n > case.budget + 128:
+    if rank == 0 and not args.no_extras and case.causal_tail == 0 and case.n > case.budget + 128:
         M, w, d, G = 128, case.w, case.head_dim, case.group
         rows = case.budget + M
         case_r = case.with_(n=rows - w, causal_tail=w)
@@ -554,7 +557,7 @@ def main():
 
     # ---- the output projection inside Eq. 7's norm (Eq. 4): || (o - v) W_O ||, W_O random [Hq * d, 4096] ----
     projection = None
-    if rank == 0 and case.dtype == "bf16":
+    if rank == 0 and not args.no_extras and case.dtype == "bf16":
         d_model = 4096
         Wp = (torch.randn(case.n_q_heads * case.head_dim, d_model, device="cuda", generator=torch.Generator("cuda").manual_seed(7))
               / float(np.sqrt(d_model))).to(torch.bfloat16)
