@@ -60,7 +60,7 @@ def shape_of(case: Case, **kw):
                          case.causal_tail, rk.BF16 if case.dtype == "bf16" else rk.F32, **kw)
 
 
-class GpuRun:
+class DeviceRun:
     """Device copies of one workload plus output buffers; calls go through the binding only."""
 
     def __init__(self, handle: rk.Handle, inp: Inputs, budget: int | None = None, adaptive_budget: int = 0):

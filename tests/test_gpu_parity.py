@@ -8,7 +8,7 @@ import oracle
 from paper_2605_08840_b200 import binding as rk
 from paper_2605_08840_b200.inputs import CONFIGS, Case, make_inputs, make_decode_query, round_to_bf16_bits
 
-from helpers import (TOL, GpuRun, assert_compaction_exact, assert_decode_close, assert_scores_close, assert_selection_valid,
+from helpers import (TOL, DeviceRun, assert_compaction_exact, assert_decode_close, assert_scores_close, assert_selection_valid,
                      shape_of, torch_dev)
 
 pytestmark = pytest.mark.gpu
@@ -33,7 +33,7 @@ def full_check(handle, inp, budget=None, path=rk.PATH_AUTO, **pool_kw):
     c = inp.case
     handle.set_kernel_path(path)
     try:
-        run = GpuRun(handle, inp, budget=budget)
+        run = DeviceRun(handle, inp, budget=budget)
         scores, idx, K_out, V_out = run.evict(pool=run.pool(**pool_kw))
     finally:
         handle.set_kernel_path(rk.PATH_AUTO)
@@ -58,7 +58,7 @@ def test_config1(handle, name, dtype, tail):
 
 def test_config1_separate_calls_match_fused(handle):
     inp = make_inputs(CONFIGS["cfg1b"])
-    run = GpuRun(handle, inp)
+    run = DeviceRun(handle, inp)
     s_f, i_f, k_f, v_f = run.evict()
     s = run.score()
     i = run.select()
@@ -85,7 +85,7 @@ def test_config1_adaptive_window(handle, tail):
         x = (ref.D[..., 0] - ref.D[..., 1]) / beta
         if np.any(np.abs(x - np.round(x)) < 0.05):
             continue   # too close to a rounding boundary for an fp32-vs-fp64 ranking comparison
-        run = GpuRun(handle, inp, adaptive_budget=B)
+        run = DeviceRun(handle, inp, adaptive_budget=B)
         scores = run.score(pool=rk.adaptive_pool(beta, base, B))
         np.testing.assert_array_equal(run.pool_used.cpu().numpy(), ref.pool)
         assert_scores_close(scores, ref.scores, TOL[case.dtype])
@@ -99,7 +99,7 @@ def test_config2(handle, path):
     inp = make_inputs(CONFIGS["cfg2"])
     worst, exact = full_check(handle, inp, path=path)
     # the planted heavy rows and sinks should be kept (reported, and checked loosely)
-    run = GpuRun(handle, inp)
+    run = DeviceRun(handle, inp)
     _, idx, _, _ = run.evict()
     planted = np.concatenate([inp.heavy_rows, np.broadcast_to(np.arange(4), inp.heavy_rows.shape[:2] + (4,))], -1)
     recall = np.mean([np.isin(planted[0, h], idx[0, h]).mean() for h in range(8)])
@@ -137,7 +137,7 @@ def _adaptive_check(handle, inp, path, base=5, evict=False):
     assert keep.any()
     handle.set_kernel_path(path)
     try:
-        run = GpuRun(handle, inp, adaptive_budget=B)
+        run = DeviceRun(handle, inp, adaptive_budget=B)
         pool = rk.adaptive_pool(beta, base, B)
         if evict:
             scores, idx, K_out, V_out = run.evict(pool=pool)
@@ -175,7 +175,7 @@ def test_adaptive_window_at_full_size(handle):
 
 
 def test_config2_is_deterministic(handle):
-    run = GpuRun(handle, make_inputs(CONFIGS["cfg2"]))
+    run = DeviceRun(handle, make_inputs(CONFIGS["cfg2"]))
     a = run.evict()
     b = run.evict()
     for x, y in zip(a, b):
@@ -189,7 +189,7 @@ def test_selection_inside_the_score_kernel_equals_the_separate_kernel(handle, sp
     switched off the separate kernel does: scores, indices and gathered rows must be identical bit for bit."""
     name, tail, budget, width, shift = spec
     inp = make_inputs(CONFIGS[name].with_(causal_tail=tail))
-    run = GpuRun(handle, inp, budget=budget)
+    run = DeviceRun(handle, inp, budget=budget)
     pool = run.pool(width=width, shift=shift)
     fused = [x.copy() for x in run.evict(pool=pool)]
     handle.set_fused_select(False)
@@ -214,7 +214,7 @@ def test_selection_inside_the_score_kernel_with_ties(handle):
     va, vb = inp.V[:, :, 0:1].copy(), inp.V[:, :, 1:2].copy()
     inp.V[:, :, 0::2] = va
     inp.V[:, :, 1::2] = vb
-    run = GpuRun(handle, inp)
+    run = DeviceRun(handle, inp)
     fused = [x.copy() for x in run.evict()]
     handle.set_fused_select(False)
     try:
@@ -232,7 +232,7 @@ def test_selection_inside_the_score_kernel_with_ties(handle):
 def test_config3_layer(handle, layer):
     case = CONFIGS["cfg3"].with_(seed=3000 + layer)
     inp = make_inputs(case)
-    run = GpuRun(handle, inp)
+    run = DeviceRun(handle, inp)
     scores, idx, K_out, V_out = run.evict()
     ref = oracle_scores(inp)                      # all eight heads of the layer
     assert_scores_close(scores, ref.scores, TOL["bf16"])
@@ -244,7 +244,7 @@ def test_config3_layer(handle, layer):
 
 def test_config3_wide_pooling_changes_the_selection(handle):
     inp = make_inputs(CONFIGS["cfg3"])
-    run = GpuRun(handle, inp)
+    run = DeviceRun(handle, inp)
     _, idx7, _, _ = run.evict()
     idx7 = idx7.copy()
     scores, idx31, _, _ = run.evict(pool=run.pool(width=31))
@@ -262,7 +262,7 @@ def test_config4_full_size(handle):
 
 
 def test_config4_is_deterministic(handle):
-    run = GpuRun(handle, make_inputs(CONFIGS["cfg4"]))
+    run = DeviceRun(handle, make_inputs(CONFIGS["cfg4"]))
     a = run.evict()
     b = run.evict()
     for x, y in zip(a, b):
@@ -282,7 +282,7 @@ def test_config5_sweep(handle, cfg5_inputs, decay, width):
     ref = oracle_scores(inp, ema_decay=decay, width=width).scores     # all 64 (batch, KV head) rows
     _, kbits, vbits = inp.device_arrays()
     for budget in (128, 512, 2048):
-        run = GpuRun(handle, inp, budget=budget)
+        run = DeviceRun(handle, inp, budget=budget)
         scores, idx, K_out, V_out = run.evict(pool=run.pool(width=width), ema_decay=decay)
         assert_scores_close(scores, ref, TOL["bf16"])
         assert_selection_valid(idx, ref, budget, TOL["bf16"])
@@ -292,7 +292,7 @@ def test_config5_sweep(handle, cfg5_inputs, decay, width):
 
 
 def test_config5_is_deterministic(handle, cfg5_inputs):
-    run = GpuRun(handle, cfg5_inputs)
+    run = DeviceRun(handle, cfg5_inputs)
     a = run.evict()
     b = run.evict()
     for x, y in zip(a, b):
@@ -330,7 +330,7 @@ def test_more_heads_than_sms(handle):
     """160 (batch, KV head) pairs: the persistent score kernel runs one CTA per head and two rounds."""
     case = Case("many_heads", 20, 32, 8, 128, 300, 32, 30, 5, 0, 0.8, "bf16", 0, "normal", 33)
     inp = make_inputs(case)
-    run = GpuRun(handle, inp)
+    run = DeviceRun(handle, inp)
     scores, idx, K_out, V_out = run.evict()
     ref = oracle_scores(inp).scores            # all 160 heads
     assert_scores_close(scores, ref, TOL["bf16"])
@@ -365,9 +365,9 @@ def test_strided_kv_layout(handle):
     H, n, d = case.n_kv_heads, case.n_kv, case.head_dim
     strides = (n * H * d, d, H * d)
     shape = shape_of(case, k_strides=strides, v_strides=strides)
-    ref_run = GpuRun(handle, inp)
+    ref_run = DeviceRun(handle, inp)
     s_ref, i_ref, k_ref, v_ref = ref_run.evict()
-    run = GpuRun(handle, inp)
+    run = DeviceRun(handle, inp)
     handle.evict(shape, Q, Kt, Vt, case.ema_decay, run.pool(), case.budget, run.indices, run.K_out, run.V_out, run.ws,
                  scores_out=run.scores)
     torch.cuda.synchronize()
@@ -383,7 +383,7 @@ def test_evict_host_matches_oracle(handle):
     import torch
     case = CONFIGS["cfg2"]
     inp = make_inputs(case)
-    run = GpuRun(handle, inp)
+    run = DeviceRun(handle, inp)
     q, k, v = inp.device_arrays()
     hQ, hK, hV = (torch.from_numpy(np.ascontiguousarray(a)).pin_memory() for a in (q, k, v))
     dQ, dK, dV = (torch.empty_like(t, device="cuda") for t in (hQ, hK, hV))     # staging, filled by the call
@@ -491,7 +491,7 @@ def test_decode_matches_oracle(handle, spec):
 def test_decode_over_compacted_cache_of_config2(handle):
     import torch
     inp = make_inputs(CONFIGS["cfg2"])
-    run = GpuRun(handle, inp)
+    run = DeviceRun(handle, inp)
     _, idx, K_out, V_out = run.evict()
     q = make_decode_query(inp)
     qd = round_to_bf16_bits(q).view(np.int16)
@@ -539,7 +539,7 @@ def test_score_from_lse_matches_oracle(handle, spec):
     name, dtype, tail = spec
     inp = make_inputs(CONFIGS[name].with_(dtype=dtype, causal_tail=tail))
     ref, O, lse = _window_stats(inp)
-    run = GpuRun(handle, inp)
+    run = DeviceRun(handle, inp)
     handle.score_from_lse(run.shape, run.Q, run.K, run.V, torch.from_numpy(O).cuda(), torch.from_numpy(lse).cuda(),
                           inp.case.ema_decay, run.pool(), run.scores, run.ws)
     torch.cuda.synchronize()
@@ -555,7 +555,7 @@ def test_evict_from_lse_matches_oracle(handle, spec):
     inp = make_inputs(CONFIGS[name].with_(causal_tail=tail))
     c = inp.case
     ref, O, lse = _window_stats(inp, with_A_check=False)
-    run = GpuRun(handle, inp)
+    run = DeviceRun(handle, inp)
     handle.evict_from_lse(run.shape, run.Q, run.K, run.V, torch.from_numpy(O).cuda(), torch.from_numpy(lse).cuda(),
                           c.ema_decay, run.pool(), run.budget, run.indices, run.K_out, run.V_out, run.ws,
                           scores_out=run.scores)
@@ -573,7 +573,7 @@ def test_score_from_lse_at_full_size(handle):
     import torch
     inp = make_inputs(CONFIGS["cfg4"])
     ref, O, lse = _window_stats(inp, with_A_check=False)
-    run = GpuRun(handle, inp)
+    run = DeviceRun(handle, inp)
     dO, dL = torch.from_numpy(O).cuda(), torch.from_numpy(lse).cuda()
     handle.score_from_lse(run.shape, run.Q, run.K, run.V, dO, dL, inp.case.ema_decay, run.pool(), run.scores, run.ws)
     torch.cuda.synchronize()
@@ -617,7 +617,7 @@ def variant_check(handle, inp, variant, path=rk.PATH_AUTO, from_lse=False, ema_d
     handle.set_kernel_path(path)
     handle.set_variant(ind, tmp, spa, grp)
     try:
-        run = GpuRun(handle, inp, budget=budget)
+        run = DeviceRun(handle, inp, budget=budget)
         if from_lse:
             _, O, lse = _window_stats(inp, with_A_check=False)
             handle.evict_from_lse(run.shape, run.Q, run.K, run.V, torch.from_numpy(O).cuda(),
@@ -696,7 +696,7 @@ def test_inverted_ema_leaves_the_tensor_core_kernel_when_its_chain_would_overflo
         handle.set_kernel_path(rk.PATH_TENSOR_CORE)
         handle.set_variant(*variant)
         try:
-            run = GpuRun(handle, inp)
+            run = DeviceRun(handle, inp)
             with pytest.raises(rk.RestKVError) as e:
                 handle.evict(run.shape, run.Q, run.K, run.V, decay, run.pool(), run.budget, run.indices, run.K_out,
                              run.V_out, run.ws)
@@ -727,7 +727,7 @@ def test_variants_with_the_adaptive_window(handle, variant):
             continue   # too close to a rounding boundary for an fp32-vs-fp64 ranking comparison
         handle.set_variant(ind, tmp, spa, grp)
         try:
-            run = GpuRun(handle, inp, adaptive_budget=B)
+            run = DeviceRun(handle, inp, adaptive_budget=B)
             scores = run.score(pool=rk.adaptive_pool(beta, base, B))
         finally:
             handle.set_variant()
@@ -744,7 +744,7 @@ def test_variants_score_a_single_row_cache(handle):
     for ind, expect in ((REC, None), (ATT, 1.0), (ATTV, None)):
         handle.set_variant(ind)
         try:
-            got = GpuRun(handle, inp).score()
+            got = DeviceRun(handle, inp).score()
         finally:
             handle.set_variant()
         ref = oracle.score(inp.Q, inp.K, inp.V, ema_decay=case.ema_decay, width=1, indicator_mode=ind).scores
@@ -773,7 +773,7 @@ def test_set_variant_validates_its_fields(handle):
 def _budgets_check(handle, inp, budgets, max_budget, pool=None, oracle_kw=None):
     import torch
     c = inp.case
-    run = GpuRun(handle, inp, budget=max_budget)
+    run = DeviceRun(handle, inp, budget=max_budget)
     S = run.keep                                           # min(max_budget, n_kv)
     dB = torch.from_numpy(np.ascontiguousarray(budgets, dtype=np.int32)).cuda()
     sentinel = 0x7B7B if c.dtype == "bf16" else None
@@ -836,7 +836,7 @@ def test_budgets_per_head_with_the_adaptive_window(handle):
         pytest.skip("a head sits on a rounding boundary of Eq. 11")
     import torch
     c = inp.case
-    run = GpuRun(handle, inp, budget=B, adaptive_budget=B)
+    run = DeviceRun(handle, inp, budget=B, adaptive_budget=B)
     dB = torch.tensor([[100, 17]], dtype=torch.int32, device="cuda")
     handle.evict_budgets(run.shape, run.Q, run.K, run.V, c.ema_decay, rk.adaptive_pool(beta, 3, B), dB, B, run.indices,
                          run.K_out, run.V_out, run.ws, scores_out=run.scores)
@@ -863,7 +863,7 @@ def test_reeviction_after_m_generated_tokens(handle, use_decode_statistics):
     B, w, M = case.budget, case.w, 48
     tol = TOL["bf16"]
     inp = make_inputs(case)
-    run = GpuRun(handle, inp)
+    run = DeviceRun(handle, inp)
     scores1, idx1, _, _ = run.evict()
     ref1 = oracle_scores(inp)
     assert_scores_close(scores1, ref1.scores, tol)
@@ -890,7 +890,7 @@ def test_reeviction_after_m_generated_tokens(handle, use_decode_statistics):
     # second eviction: the last w generated tokens are the window; their own rows are the cache's last w rows
     case2 = case.with_(name="reevict", n=B + M - w, causal_tail=w, recipe="normal")
     inp2 = Inputs(case2, np.ascontiguousarray(queries[:, :, M - w:]), K2, V2)
-    run2 = GpuRun(handle, inp2)
+    run2 = DeviceRun(handle, inp2)
     if use_decode_statistics:
         O_obs = outs[M - w:].permute(1, 2, 0, 3).contiguous()          # [b, Hq, w, d]
         L_obs = lses[M - w:].permute(1, 2, 0).contiguous()             # [b, Hq, w]
@@ -942,7 +942,7 @@ def projection_check(handle, inp, d_model, path=rk.PATH_AUTO, seed=1, from_lse=F
     if variant:
         handle.set_variant(*variant)
     try:
-        run = GpuRun(handle, inp)
+        run = DeviceRun(handle, inp)
         if from_lse:
             _, O, lse = _window_stats(inp, with_A_check=False)
             handle.evict_from_lse(run.shape, run.Q, run.K, run.V, torch.from_numpy(O).cuda(),
@@ -1037,7 +1037,7 @@ def test_projection_is_ignored_by_the_attention_weight_indicators(handle):
     handle.set_output_projection(factor, inp.case.n_q_heads, inp.case.head_dim)
     handle.set_variant(ATT, MEAN)
     try:
-        scores, _, _, _ = GpuRun(handle, inp).evict()
+        scores, _, _, _ = DeviceRun(handle, inp).evict()
     finally:
         handle.set_output_projection(None)
         handle.set_variant()
@@ -1055,7 +1055,7 @@ def test_projection_must_match_the_shape(handle):
     inp = make_inputs(CONFIGS["cfg1b"])
     c = inp.case
     _, factor = _make_projection(handle, c, 32, seed=2)
-    run = GpuRun(handle, inp)
+    run = DeviceRun(handle, inp)
     handle.set_output_projection(factor, c.n_q_heads + 8, c.head_dim)
     try:
         with pytest.raises(rk.RestKVError) as e:
@@ -1076,7 +1076,7 @@ def test_wait_limit_runs_out_and_the_handle_recovers(handle):
     handle and workspace then give the oracle's scores."""
     case = Case("timeout", 1, 4, 1, 128, 2000, 32, 100, 5, 0, 0.9, "bf16", 0, "normal", 123)
     inp = make_inputs(case)
-    run = GpuRun(handle, inp)
+    run = DeviceRun(handle, inp)
     handle.set_kernel_path(rk.PATH_TENSOR_CORE)
     try:
         handle.set_wait_limit(1)
@@ -1096,7 +1096,7 @@ def test_api_rejects_bad_arguments(handle):
     import torch
     case = CONFIGS["cfg1b"]
     inp = make_inputs(case)
-    run = GpuRun(handle, inp)
+    run = DeviceRun(handle, inp)
 
     def status_of(fn):
         try:
