@@ -72,7 +72,7 @@ def whole_job_value(tokens_per_rank_step, world, steps, total_ms):
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from an ncu capture
 # of this workload, together with the digest of the kernel sources the capture was taken on: the figure is reported
 # only while those sources are unchanged, otherwise `traffic` is null.
-KERNEL_TRAFFIC = {"cfg4": {"bytes": 1024809984 + 27120896, "sources_sha256": "17e3ec72af554e0aebc6eeff775d86a85b19c7550b16ef355da76ebcd708b551"}}
+KERNEL_TRAFFIC = {"cfg4": {"bytes": 1024809984 + 27120896, "sources_sha256": "c2a2d5d570c4642c49dda616763660c7e2819fce2c4e152d8a36ee85e09c58ec"}}
 KERNEL_SOURCES = ("tc_fused.cu", "tc_common.cuh", "sm100_ptx.cuh")
 
 
