@@ -1068,6 +1068,80 @@ def test_projection_must_match_the_shape(handle):
     torch.cuda.synchronize()
 
 
+# ------------------------------------------------------------------ nothing is written outside the buffers
+class _Guarded:
+    """One device allocation carved into buffers with 4 KB bands of a fixed byte pattern before and after each: a
+    write past either end of a buffer shows up as a changed band (reads cannot be seen this way)."""
+    BAND = 4096
+
+    def __init__(self, sizes):
+        import torch
+        self.torch = torch
+        self.offsets, off = [], self.BAND
+        for nbytes in sizes:
+            self.offsets.append((off, nbytes))
+            off += (nbytes + self.BAND - 1) // self.BAND * self.BAND + self.BAND
+        self.raw = torch.full((off,), 0xA5, dtype=torch.uint8, device="cuda")
+
+    def view(self, i, dtype, shape):
+        off, nbytes = self.offsets[i]
+        return self.raw[off:off + nbytes].view(dtype).view(shape)
+
+    def bands_intact(self):
+        mask = self.torch.ones_like(self.raw, dtype=self.torch.bool)
+        for off, nbytes in self.offsets:
+            mask[off:off + nbytes] = False
+        return bool((self.raw[mask] == 0xA5).all())
+
+
+GUARD_CASES = [
+    ("tc_ragged", Case("g1", 2, 8, 2, 128, 1000, 32, 64, 5, 0, 0.8, "bf16", 0, "normal", 91), rk.PATH_AUTO, False),
+    ("tc_tail_fused", CONFIGS["cfg2"].with_(causal_tail=32), rk.PATH_TENSOR_CORE, False),
+    ("tc_one_over_tile", Case("g2", 1, 4, 1, 128, 129, 32, 130, 3, 0, 0.7, "bf16", 0, "normal", 92), rk.PATH_AUTO, False),
+    ("head_sequential", Case("g3", 3, 4, 1, 128, 700, 32, 50, 7, 2, 0.9, "bf16", 0, "normal", 93), rk.PATH_HEAD_SEQUENTIAL, False),
+    ("simt_f32", CONFIGS["cfg1b"].with_(causal_tail=32), rk.PATH_AUTO, False),
+    ("simt_odd", Case("g4", 2, 6, 3, 72, 333, 5, 40, 3, -1, 0.6, "f32", 0, "normal", 94), rk.PATH_AUTO, False),
+    ("many_heads", Case("g5", 20, 32, 8, 128, 300, 32, 30, 5, 0, 0.8, "bf16", 0, "normal", 95), rk.PATH_AUTO, False),
+    ("adaptive_tc", CONFIGS["cfg2"].with_(n=2000, budget=200), rk.PATH_AUTO, True),
+    ("adaptive_simt", CONFIGS["cfg1b"], rk.PATH_AUTO, True),
+]
+
+
+@pytest.mark.parametrize("spec", GUARD_CASES, ids=[g[0] for g in GUARD_CASES])
+def test_no_write_lands_outside_a_buffer(handle, spec):
+    import torch
+    _, case, path, adaptive = spec
+    inp = make_inputs(case)
+    c = inp.case
+    keep = min(c.budget, c.n_kv)
+    BH = c.batch * c.n_kv_heads
+    esize = 2 if c.dtype == "bf16" else 4
+    shape = shape_of(c)
+    ws_bytes = handle.workspace_bytes(shape, c.budget, adaptive=adaptive)
+    g = _Guarded([BH * c.n_kv * 4, BH * keep * 4, BH * keep * c.head_dim * esize, BH * keep * c.head_dim * esize, ws_bytes])
+    el = torch.bfloat16 if c.dtype == "bf16" else torch.float32
+    scores = g.view(0, torch.float32, (c.batch, c.n_kv_heads, c.n_kv))
+    indices = g.view(1, torch.int32, (c.batch, c.n_kv_heads, keep))
+    K_out = g.view(2, el, (c.batch, c.n_kv_heads, keep, c.head_dim))
+    V_out = g.view(3, el, (c.batch, c.n_kv_heads, keep, c.head_dim))
+    ws = g.view(4, torch.uint8, (ws_bytes,))
+    q, k, v = (torch_dev(a, c.dtype) for a in inp.device_arrays())
+    pool = rk.adaptive_pool(50.0, 3, c.budget) if adaptive else rk.fixed_pool(c.width, c.shift)
+    handle.set_kernel_path(path)
+    try:
+        handle.evict(shape, q, k, v, c.ema_decay, pool, c.budget, indices, K_out, V_out, ws, scores_out=scores)
+        handle.score(shape, q, k, v, c.ema_decay, pool, scores, ws)
+        handle.select(shape, scores, c.budget, indices, ws)
+        handle.compact(shape, k, v, indices, keep, K_out, V_out)
+        torch.cuda.synchronize()
+    finally:
+        handle.set_kernel_path(rk.PATH_AUTO)
+    assert handle.poll_status() == rk.RESTKV_OK
+    assert g.bands_intact()
+    idx = indices.cpu().numpy()
+    assert idx.min() >= 0 and idx.max() < c.n_kv
+
+
 # ------------------------------------------------------------------ a device-side wait that runs out
 def test_wait_limit_runs_out_and_the_handle_recovers(handle):
     """With a wait limit of one SM clock the first CTA to reach a group barrier of the persistent score kernel gives
