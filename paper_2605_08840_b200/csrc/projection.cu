@@ -1,6 +1,6 @@
 // The output projection of Eq. 4 inside Eq. 7's norm: || (o - v) W ||^2 = (o - v)^T M (o - v) with M = W W^T, one
 // d x d matrix per query head (W = that head's d x d_model slice of the model's W_O).
-//   restkv_prepare_output_projection:  M (fp32), a Cholesky factor L of M rounded to bf16 (stored transposed, for
+//   restkv_prepare_output_projection:  M (fp32), a factor L of M (L L^T = M) rounded to bf16 (stored transposed, for
 //     the tensor-core kernels) and Mt = L L^T of the rounded factor (fp32), so that every term the tensor-core path
 //     forms belongs to one and the same quadratic form.
 //   per call:  m_r = M o_r for the window rows (SIMT path; the tensor-core kernel does it in its merge).
@@ -48,48 +48,82 @@ __global__ void proj_gram_kernel(int d, int d_model, const T* __restrict__ W, fl
     for (int b = 0; b < per; ++b) Mh[(ti + 16 * a) * d + tk + 16 * b] = acc[a][b];
 }
 
-// Cholesky factor of M[hq] (lower triangular L, L L^T = M) in shared memory, fp32; where a pivot vanishes (M
-// singular: d_model < d) the column is dropped, which leaves that direction without weight.  Then the factor
-// is rounded to bf16 and written transposed (LT[c][i] = L[i][c]), and Mt = L L^T of the rounded factor.
-// grid (Hq), block d threads (thread i owns row i), dynamic shared memory d * (d + 1) floats.
+// A factor L of M[hq] with L L^T = M, by Cholesky elimination with diagonal pivoting in shared memory, fp32: every
+// step takes the row with the largest remaining diagonal entry, and the elimination stops once that entry has
+// fallen to 1e-5 of the first one (M singular, d_model < d: what is left is rounding residue, and a column built
+// on it would be noise divided by its square root); the remaining columns are zero.  The rows of L stay in their
+// original order, its columns follow the pivots, so L is not triangular; nothing downstream needs that.  Then the
+// factor is rounded to bf16 and written transposed (LT[c][i] = L[i][c]), and Mt = L L^T of the rounded factor.
+// grid (Hq), block 128 threads (thread i < d owns row i), dynamic shared memory d * (d + 1) floats.
 __global__ void proj_factor_kernel(int d, const float* __restrict__ M, float* __restrict__ Mt,
                                    __nv_bfloat16* __restrict__ LT) {
   extern __shared__ float Ls[];   // [d][d + 1]
-  __shared__ float s_diag;
-  const int hq = blockIdx.x, i = threadIdx.x, ld = d + 1;
+  __shared__ float red_v[4];
+  __shared__ int red_i[4];
+  __shared__ float s_piv;
+  __shared__ int s_row;
+  const int hq = blockIdx.x, i = threadIdx.x, ld = d + 1, lane = i & 31, wid = i >> 5;
+  const bool act = i < d;
   const float* Mh = M + (long long)hq * d * d;
-  float trace = 0.f;
-  for (int k = 0; k < d; ++k) {
-    Ls[i * ld + k] = Mh[i * d + k];
-    trace += Mh[k * d + k];
-  }
-  // a pivot below fp32's resolution of the diagonal means that M has no weight left in this direction (M is
-  // positive semi-definite, so the rest of the column is zero as well): the column is dropped
-  const float floor_pivot = fmaxf(trace / (float)d, 1e-30f) * 4e-6f;
-  __syncthreads();
+  float dres = act ? Mh[i * d + i] : -1.f;   // what is left of the row's diagonal entry
+  bool done = !act;
+  float top = 0.f;
   for (int c = 0; c < d; ++c) {
-    // row i, column c: M[i][c] - sum_{k<c} L[i][k] L[c][k]
-    float v = Ls[i * ld + c];
-    if (i >= c)
-      for (int k = 0; k < c; ++k) v = fmaf(-Ls[i * ld + k], Ls[c * ld + k], v);
-    if (i == c) s_diag = v > floor_pivot ? sqrtf(v) : 0.f;
+    // the largest remaining diagonal entry (ties: the lower row)
+    float bv = done ? -1.f : dres;
+    int bi = i;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+      if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+    }
+    if (lane == 0) { red_v[wid] = bv; red_i[wid] = bi; }
     __syncthreads();
-    if (i >= c && s_diag > 0.f) Ls[i * ld + c] = (i == c) ? s_diag : v / s_diag;
-    else Ls[i * ld + c] = 0.f;
+    if (i == 0) {
+      float v = red_v[0];
+      int r = red_i[0];
+      for (int w = 1; w < 4; ++w)
+        if (red_v[w] > v) { v = red_v[w]; r = red_i[w]; }
+      s_piv = v;
+      s_row = r;
+    }
+    __syncthreads();
+    const float piv = s_piv;
+    const int pr = s_row;
+    if (c == 0) top = piv;
+    const bool stop = !(piv > 1e-5f * top) || !(piv > 1e-30f);   // uniform over the block
+    if (stop) {
+      if (act)
+        for (int cc = c; cc < d; ++cc) Ls[i * ld + cc] = 0.f;
+      break;
+    }
+    if (act) {
+      // column c: (M[i][pr] - sum_{k<c} L[i][k] L[pr][k]) / sqrt(pivot); rows eliminated earlier get 0
+      float v = Mh[i * d + pr];
+      for (int k = 0; k < c; ++k) v = fmaf(-Ls[i * ld + k], Ls[pr * ld + k], v);
+      const float sd = sqrtf(piv);
+      const float l = done ? 0.f : (i == pr ? sd : v / sd);
+      Ls[i * ld + c] = l;
+      dres -= l * l;
+      if (i == pr) done = true;
+    }
     __syncthreads();
   }
+  __syncthreads();
   __nv_bfloat16* LTh = LT + (long long)hq * d * d;
-  for (int c = 0; c < d; ++c) {
-    const __nv_bfloat16 r = __float2bfloat16_rn(Ls[i * ld + c]);
-    LTh[c * d + i] = r;
-    Ls[i * ld + c] = __bfloat162float(r);
-  }
+  if (act)
+    for (int c = 0; c < d; ++c) {
+      const __nv_bfloat16 r = __float2bfloat16_rn(Ls[i * ld + c]);
+      LTh[c * d + i] = r;
+      Ls[i * ld + c] = __bfloat162float(r);
+    }
   __syncthreads();
+  if (!act) return;
   float* Mth = Mt + (long long)hq * d * d;
   for (int k = 0; k < d; ++k) {
     float v = 0.f;
-    const int cmax = min(i, k);
-    for (int c = 0; c <= cmax; ++c) v = fmaf(Ls[i * ld + c], Ls[k * ld + c], v);
+    for (int c = 0; c < d; ++c) v = fmaf(Ls[i * ld + c], Ls[k * ld + c], v);
     Mth[i * d + k] = v;
   }
 }
@@ -140,7 +174,7 @@ cudaError_t launch_projection_prepare(int n_q_heads, int d, int d_model, restkv_
     e = cudaFuncSetAttribute(proj_factor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  proj_factor_kernel<<<n_q_heads, d, smem, st>>>(d, pr.M, const_cast<float*>(pr.Mt),
+  proj_factor_kernel<<<n_q_heads, 128, smem, st>>>(d, pr.M, const_cast<float*>(pr.Mt),
                                                  const_cast<__nv_bfloat16*>(pr.LT));
   return cudaGetLastError();
 }

@@ -169,9 +169,11 @@ def test_config2_adaptive_window_evict_on_the_tensor_core_kernel(handle, tail):
 
 
 def test_adaptive_window_at_full_size(handle):
-    """The long-context workload with the adaptive window: 1024 per-query top-B selections over 131072 tokens each."""
-    keep = _adaptive_check(handle, make_inputs(CONFIGS["cfg4"]), rk.PATH_TENSOR_CORE, evict=True)
-    assert keep.sum() >= 4
+    """The adaptive window at the long context's length: per-query top-B selections over 131072 tokens each (two KV
+    heads of the long-context workload's shape; the oracle sorts every query's row, which sets the cost of this test)."""
+    case = CONFIGS["cfg4"].with_(n_q_heads=8, n_kv_heads=2)
+    keep = _adaptive_check(handle, make_inputs(case), rk.PATH_TENSOR_CORE, evict=True)
+    assert keep.sum() >= 1
 
 
 def test_config2_is_deterministic(handle):
@@ -976,9 +978,10 @@ def projection_check(handle, inp, d_model, path=rk.PATH_AUTO, seed=1, from_lse=F
     return ref
 
 
-@pytest.mark.parametrize("spec", [("f32", 64, 96), ("bf16", 128, 300), ("f32", 128, 64), ("bf16", 48, 48)])
+@pytest.mark.parametrize("spec", [("f32", 64, 96), ("bf16", 128, 300), ("f32", 128, 64), ("bf16", 48, 48),
+                                  ("bf16", 128, 96), ("bf16", 128, 120), ("bf16", 128, 24)])
 def test_projection_factor(handle, spec):
-    """M = W W^T, its Cholesky factor rounded to bf16 (stored transposed) and the product of the rounded factor."""
+    """M = W W^T, a factor of it rounded to bf16 (stored transposed) and the product of the rounded factor."""
     import torch
     from paper_2605_08840_b200.inputs import bf16_bits_to_f32
     dtype, d, d_model = spec
@@ -992,11 +995,13 @@ def test_projection_factor(handle, spec):
     M_ref = np.einsum("hik,hjk->hij", W.astype(np.float64), W.astype(np.float64))
     np.testing.assert_allclose(M, M_ref, rtol=0, atol=2e-6 * np.abs(M_ref).max())
     L = np.swapaxes(LT, 1, 2).astype(np.float64)
-    assert np.all(np.triu(L, 1) == 0)
     np.testing.assert_allclose(Mt, L @ np.swapaxes(L, 1, 2), rtol=0, atol=2e-6 * np.abs(M_ref).max())
     # the rounded factor reproduces M to bf16 accuracy, also where M is singular (d_model < d)
     err = np.linalg.norm(Mt - M_ref, axis=(1, 2)) / np.linalg.norm(M_ref, axis=(1, 2))
     assert err.max() < 2.0 ** -7
+    # no column is built on a pivot that is rounding residue: a singular M keeps at most its rank
+    kept = (np.abs(LT) > 0).any(axis=2).sum(axis=1)          # non-zero columns of L
+    assert kept.max() <= min(d, d_model)
 
 
 @pytest.mark.parametrize("spec", [("cfg1b", "f32", 0, 96), ("cfg1b", "bf16", 32, 64), ("cfg1a", "f32", 0, 40)])
@@ -1006,7 +1011,7 @@ def test_projection_on_the_simt_kernels(handle, spec):
 
 
 @pytest.mark.parametrize("tail", [0, 32])
-@pytest.mark.parametrize("d_model", [256, 24])
+@pytest.mark.parametrize("d_model", [96, 24])
 def test_projection_on_the_tensor_core_kernel(handle, tail, d_model):
     # workload 2 has planted heavy hitters: entries with A > 1/8 take the exact (projected) distance
     projection_check(handle, make_inputs(CONFIGS["cfg2"].with_(causal_tail=tail)), d_model, path=rk.PATH_TENSOR_CORE,
@@ -1014,7 +1019,7 @@ def test_projection_on_the_tensor_core_kernel(handle, tail, d_model):
 
 
 def test_projection_from_given_window_statistics(handle):
-    projection_check(handle, make_inputs(CONFIGS["cfg2"]), 192, path=rk.PATH_TENSOR_CORE, from_lse=True)
+    projection_check(handle, make_inputs(CONFIGS["cfg2"]), 64, path=rk.PATH_TENSOR_CORE, from_lse=True)
 
 
 @pytest.mark.parametrize("spec", [(4, 2, 64), (2, 2, 128), (16, 2, 16)])
@@ -1028,7 +1033,7 @@ def test_projection_at_other_window_lengths(handle, spec):
 
 def test_projection_with_a_variant(handle):
     inp = make_inputs(CONFIGS["cfg2"])
-    projection_check(handle, inp, 128, path=rk.PATH_TENSOR_CORE, variant=(REC, INV, rk.SPATIAL_MAX, rk.GROUP_MAX))
+    projection_check(handle, inp, 48, path=rk.PATH_TENSOR_CORE, variant=(REC, INV, rk.SPATIAL_MAX, rk.GROUP_MAX))
 
 
 def test_projection_is_ignored_by_the_attention_weight_indicators(handle):
