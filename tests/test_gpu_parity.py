@@ -1209,6 +1209,84 @@ def test_random_shapes_and_settings(handle, seed):
         assert_compaction_exact(idx, vbits, V_out)
 
 
+@pytest.mark.parametrize("seed", [21, 22])
+def test_random_shapes_through_the_other_entry_points(handle, seed):
+    """Fifty seeded draws per seed of shape and settings through restkv_score_from_lse, restkv_evict_from_lse,
+    restkv_evict_budgets and the adaptive window, each against the oracle."""
+    import torch
+    rng = np.random.default_rng(seed)
+    for _ in range(50):
+        if rng.random() < 0.7:
+            w = int(rng.choice([16, 32, 64, 128])); G = 128 // w; d = 128; dtype = "bf16"
+        else:
+            w = int(rng.integers(1, 20)); G = int(rng.choice([1, 2, 3, 4])); d = int(rng.choice([16, 32, 64, 72, 128]))
+            dtype = str(rng.choice(["f32", "bf16"]))
+        Hkv, b = int(rng.integers(1, 4)), int(rng.integers(1, 3))
+        tail = int(rng.choice([0, w]))
+        n = int(rng.choice([2, 5, 127, 128, 129, 300, 1000, 2500, 4097])) + int(rng.integers(0, 3))
+        budget = int(rng.choice([1, 7, 64, 200, 5000]))
+        width, shift = int(rng.choice([1, 3, 7, 21, 31])), int(rng.choice([0, 0, 2, -5, 40]))
+        decay = float(rng.choice([0.0, 0.3, 0.7, 0.9, 0.99, 1.0]))
+        recipe = "normal" if (dtype == "f32" and n < 50) else str(rng.choice(["normal", "planted"]))
+        mode = str(rng.choice(["lse_score", "lse_evict", "budgets", "adaptive"]))
+        case = Case("sweep2", b, Hkv * G, Hkv, d, n, w, budget, width, shift, decay, dtype, tail, recipe,
+                    int(rng.integers(0, 10000)))
+        what = "%s %s" % (mode, case)
+        inp = make_inputs(case)
+        tol = TOL[dtype]
+        _, kbits, vbits = inp.device_arrays()
+        if mode in ("lse_score", "lse_evict"):
+            ref, O, lse = _window_stats(inp, with_A_check=False)
+            run = DeviceRun(handle, inp)
+            dO, dL = torch.from_numpy(O).cuda(), torch.from_numpy(lse).cuda()
+            if mode == "lse_score":
+                handle.score_from_lse(run.shape, run.Q, run.K, run.V, dO, dL, decay, run.pool(), run.scores, run.ws)
+            else:
+                handle.evict_from_lse(run.shape, run.Q, run.K, run.V, dO, dL, decay, run.pool(), run.budget,
+                                      run.indices, run.K_out, run.V_out, run.ws, scores_out=run.scores)
+            torch.cuda.synchronize()
+            assert handle.poll_status() == rk.RESTKV_OK, what
+            assert_scores_close(run.scores.cpu().numpy(), ref.scores, tol, what)
+            if mode == "lse_evict":
+                idx = run.indices.cpu().numpy()
+                assert_selection_valid(idx, ref.scores, run.budget, tol)
+                assert_compaction_exact(idx, kbits, run._bits(run.K_out))
+                assert_compaction_exact(idx, vbits, run._bits(run.V_out))
+        elif mode == "budgets":
+            ref = oracle_scores(inp)
+            run = DeviceRun(handle, inp)
+            bud = rng.integers(0, budget + 3, size=(b, Hkv)).astype(np.int32)
+            run.indices.fill_(-7)
+            handle.evict_budgets(run.shape, run.Q, run.K, run.V, decay, run.pool(), torch.from_numpy(bud).cuda(),
+                                 budget, run.indices, run.K_out, run.V_out, run.ws, scores_out=run.scores)
+            torch.cuda.synchronize()
+            assert handle.poll_status() == rk.RESTKV_OK, what
+            idx, K_out = run.indices.cpu().numpy(), run._bits(run.K_out)
+            assert_scores_close(run.scores.cpu().numpy(), ref.scores, tol, what)
+            for bi in range(b):
+                for hh in range(Hkv):
+                    keep = min(max(int(bud[bi, hh]), 1), run.keep)
+                    assert_selection_valid(idx[bi, hh, :keep], ref.scores[bi, hh], keep, tol)
+                    assert np.all(idx[bi, hh, keep:] == -1), what
+                    assert np.array_equal(K_out[bi, hh, :keep], kbits[bi, hh][idx[bi, hh, :keep]]), what
+        else:
+            Bp = max(1, min(budget, 300)) + tail
+            probe = oracle_scores(inp, pool_mode=1, beta=1e9, base_width=1, budget=Bp)
+            delta = abs(probe.D[..., 0] - probe.D[..., 1]).min()
+            if not delta > 0:
+                continue
+            beta, base = float(delta / 1.5), int(rng.choice([1, 3, 5]))
+            ref = oracle_scores(inp, pool_mode=1, beta=beta, base_width=base, budget=Bp)
+            x = (ref.D[..., 0] - ref.D[..., 1]) / beta
+            keepm = np.abs(x - np.round(x)) >= 0.05
+            run = DeviceRun(handle, inp, budget=Bp, adaptive_budget=Bp)
+            sc = run.score(pool=rk.adaptive_pool(beta, base, Bp))
+            assert handle.poll_status() == rk.RESTKV_OK, what
+            assert np.array_equal(run.pool_used.cpu().numpy()[keepm], ref.pool[keepm]), what
+            for bi, hh in zip(*np.nonzero(keepm)):
+                assert_scores_close(sc[bi, hh], ref.scores[bi, hh], tol, what)
+
+
 # ------------------------------------------------------------------ a device-side wait that runs out
 def test_wait_limit_runs_out_and_the_handle_recovers(handle):
     """With a wait limit of one SM clock the first CTA to reach a group barrier of the persistent score kernel gives
