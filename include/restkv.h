@@ -192,7 +192,8 @@ restkv_status restkv_evict_host(restkv_handle* h, const restkv_shape* shape, con
  * RESTKV_BF16 with head_dim 128 and up to 128 query heads per KV head runs as plain attention on the tensor-core
  * kernel (the softmax weights are rounded to bf16 before they meet V) when the workspace has the ~10 MB it needs,
  * which every restkv_workspace_bytes() result has; everything else runs on fp32 SIMT kernels, which need
- * batch * n_kv_heads * 64 * group * (head_dim + 2) floats.
+ * batch * n_kv_heads * 64 * group * (head_dim + 2) floats and take 1, 2, 4 or 8 query heads per KV head and rows of
+ * 32, 64, ..., 1024 bytes (head_dim * element size a power of two); other shapes return RESTKV_ERR_UNSUPPORTED.
  */
 restkv_status restkv_decode(restkv_handle* h, const restkv_shape* shape, const void* q, const void* Kc,
                             const void* Vc, int n_rows, float* out, float* lse, void* workspace,
