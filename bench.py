@@ -455,7 +455,7 @@ def main():
 
     # ---- the ablation variants of Appendix G as modes of the same path (beside the headline) ----
     variants = None
-    if rank == 0 and not args.no_extras:
+    if rank == 0 and world == 1 and not args.no_extras:
         labelled = (("attention_weight__mean_over_window", (rk.INDICATOR_ATTENTION, rk.TEMPORAL_MEAN, 0, 0)),
                     ("attention_weight_times_value_norm__ema", (rk.INDICATOR_ATTENTION_VNORM, rk.TEMPORAL_EMA, 0, 0)),
                     ("reconstruction__inverted_ema__max_pool__group_max",
@@ -481,7 +481,7 @@ def main():
 
     # ---- the adaptive window of Eq. 10-12 (per-query top-B of the raw indicator, D_front / D_rear) ----
     adaptive = None
-    if rank == 0 and not args.no_extras:
+    if rank == 0 and world == 1 and not args.no_extras:
         apool = rk.adaptive_pool(2000.0, case.width, case.budget)
         ws_a = torch.empty(handle.workspace_bytes(shape, case.budget, adaptive=True), dtype=torch.uint8, device="cuda")
 
@@ -512,7 +512,7 @@ def main():
     # ---- eviction again during decoding (Appendix B): the compacted cache plus M generated tokens, the last w of
     #      them as the window (their own rows are the trailing, causally masked block) ----
     reevict = None
-    if rank == 0 and not args.no_extras and case.causal_tail == 0 and case.n > case.budget + 128:
+    if rank == 0 and world == 1 and not args.no_extras and case.causal_tail == 0 and case.n > case.budget + 128:
         M, w, d, G = 128, case.w, case.head_dim, case.group
         rows = case.budget + M
         case_r = case.with_(n=rows - w, causal_tail=w)
@@ -557,7 +557,7 @@ def main():
 
     # ---- the output projection inside Eq. 7's norm (Eq. 4): || (o - v) W_O ||, W_O random [Hq * d, 4096] ----
     projection = None
-    if rank == 0 and not args.no_extras and case.dtype == "bf16":
+    if rank == 0 and world == 1 and not args.no_extras and case.dtype == "bf16":
         d_model = 4096
         Wp = (torch.randn(case.n_q_heads * case.head_dim, d_model, device="cuda", generator=torch.Generator("cuda").manual_seed(7))
               / float(np.sqrt(d_model))).to(torch.bfloat16)
